@@ -1,0 +1,223 @@
+/*
+ * medverse_attn.h -- C ABI of the B200-native topology-aware (DAG) attention library.
+ *
+ * The library implements the attention of DAG-structured parallel decoding: every active
+ * branch of a request's reasoning DAG (a Petri-net transition, Sec. 3.2) decodes at the same time
+ * against one shared paged KV cache; a query token attends to the shared prefix, the nodes on its
+ * own path and itself, never to a concurrently running sibling (Eq. 3), and its rotary position
+ * continues from its fork or join point instead of the flattened sequence offset (Sec. 4.2,
+ * "Adaptive Position Indices").
+ *
+ * Conventions for every call
+ *   - extern "C", plain pointers and sizes.  "host" / "device" is stated per argument.
+ *   - Ownership: the caller owns every device buffer (Q/K/V/O, page pools, workspace, the plan's
+ *     device table buffer).  The library never allocates or frees device memory.  An mv_plan owns
+ *     only host memory (its tables, kept in page-locked memory so that uploads are asynchronous).
+ *   - Streams: `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     The three kernel calls and mv_plan_upload are asynchronous; they return the launch status only.
+ *   - Errors: an mv_status is returned; argument errors are found on the host before any launch.
+ *     Kernels never trap.  mv_status_string() names a status.
+ *   - Layouts: q, k, v, q_rot, out are [tokens][heads][head_dim], row-major, element type
+ *     mv_attn_geom.dtype.  The K and V page pools are separate buffers, each
+ *     [num_pages][n_kv_heads][page_size][head_dim] of the same element type.
+ *   - Order: "new tokens" (rows) are ordered (request, node index, token index) ascending.
+ *   - Supported geometry: head_dim 64 or 128; n_q_heads a multiple of n_kv_heads; page_size 16.
+ *     Anything else returns MV_ERR_UNSUPPORTED.  There is no CPU fallback.
+ */
+#ifndef MEDVERSE_ATTN_H_
+#define MEDVERSE_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MV_OK = 0,
+  MV_ERR_INVALID_ARG = 1,      /* null pointer, negative size, inconsistent offsets, bad enum          */
+  MV_ERR_NOT_TOPOLOGICAL = 2,  /* a parent index is not smaller than its child's index (or a cycle)     */
+  MV_ERR_PAGE_CAPACITY = 3,    /* a node's page list is too short for node_len + node_new tokens        */
+  MV_ERR_UNSUPPORTED = 4,      /* head_dim / dtype / group size / batch shape the kernel does not take  */
+  MV_ERR_WORKSPACE = 5,        /* workspace or table buffer missing, too small or misaligned            */
+  MV_ERR_CUDA = 6,             /* a CUDA runtime call failed (launch error, copy error)                 */
+  MV_ERR_TIMEOUT = 7           /* reserved for bounded device-side waits                                */
+} mv_status;
+
+/* Which nodes a token may attend to.  The paper states the mask twice, differently (Eq. 3 masks only
+ * same-frontier siblings; Sec. 3.2 / 4.3 let a branch inherit the history of its own path only). */
+typedef enum {
+  MV_VIS_ANCESTORS = 0,  /* prefix + transitive ancestors + the node itself (Sec. 3.2, Sec. 4.3 Join) */
+  MV_VIS_LAYERWISE = 1   /* Eq. 3 literally: every node of an earlier frontier layer + the node itself */
+} mv_vis_mode;
+
+/* Where a node's position indices start (Sec. 4.2). */
+typedef enum {
+  MV_POS_MAX_PARENT_END = 0,  /* right after the largest index used by any parent (fork alignment and
+                                 the join rule, applied node by node)                                   */
+  MV_POS_FRONTIER_ALIGNED = 1 /* one start for a whole frontier layer: the largest end of the previous
+                                 layer (the sentence on fork alignment read literally)                  */
+} mv_pos_mode;
+
+typedef enum { MV_F32 = 0, MV_BF16 = 1 } mv_dtype;
+
+/* A batch of request DAGs.  HOST memory, caller-owned, read only during mv_plan_dag.
+ * A node is one reasoning step (one Petri-net transition); node 0 of a request is normally the shared
+ * prefix (prompt + linear plan, Sec. 4.3 Phase I).  Node indices inside a request are local. */
+typedef struct {
+  int32_t n_req;
+  const int32_t* node_off;   /* [n_req+1]   CSR over nodes                                             */
+  const int32_t* node_len;   /* [n_nodes]   tokens of the node already in the KV pool                  */
+  const int32_t* node_new;   /* [n_nodes]   tokens appended by this step (decode: 1 on frontier nodes,
+                                            0 elsewhere; prefill: the node's length)                   */
+  const int32_t* parent_off; /* [n_nodes+1] CSR over parent lists                                      */
+  const int32_t* parent_idx; /* local parent indices, each < its child's local index                   */
+  const int32_t* page_off;   /* [n_nodes+1] CSR over page lists                                        */
+  const int32_t* page_idx;   /* physical page ids; a node's pages hold only that node's tokens; the
+                                last page may be partial; ceil((len+new)/page_size) pages are required */
+  int32_t page_size;         /* 16 */
+  int32_t vis_mode;          /* mv_vis_mode */
+  int32_t pos_mode;          /* mv_pos_mode */
+  int32_t chunk_tokens;      /* decode split-KV chunk length in tokens (multiple of page_size); 0 = automatic */
+} mv_dag_batch;
+
+typedef struct {
+  int32_t n_q_heads, n_kv_heads, head_dim, page_size;
+  int64_t num_pages;   /* pages in each of the K and V pools */
+  int32_t dtype;       /* mv_dtype of q/k/v/out and of the pools */
+  float sm_scale;      /* softmax scale; 0 means 1/sqrt(head_dim) */
+  double rope_base;    /* theta_i = rope_base^(-2i/head_dim) */
+} mv_attn_geom;
+
+typedef struct mv_plan mv_plan;
+
+/* Canonical integer tables of a plan (host memory, owned by the plan, valid until the plan is
+ * re-planned or destroyed).  "q-node" = a node that receives new tokens in this step. */
+typedef enum {
+  MV_TAB_LAYER = 0,         /* int32 [n_nodes]      frontier layer: 0 for roots, else 1 + max over parents (Eq. 1) */
+  MV_TAB_POS_START = 1,     /* int32 [n_nodes]      first position index of the node (Sec. 4.2)                 */
+  MV_TAB_POS_ID = 2,        /* int32 [n_new_tokens] position index of every new token                           */
+  MV_TAB_SLOT = 3,          /* int64 [n_new_tokens] pool slot = page_id * page_size + offset in page            */
+  MV_TAB_QNODE = 4,         /* int32 [n_qnodes]     global node index of every q-node, ascending                 */
+  MV_TAB_QNODE_TOK_OFF = 5, /* int32 [n_qnodes+1]   offsets of each q-node's new tokens                          */
+  MV_TAB_SEG_OFF = 6,       /* int32 [n_qnodes+1]   CSR over the q-node's visible segments                       */
+  MV_TAB_SEG_NODE = 7,      /* int32 [n_segs]       global node index of the segment (ascending in a q-node)     */
+  MV_TAB_SEG_LEN = 8,       /* int32 [n_segs]       node_len + node_new of that node                             */
+  MV_TAB_KV_LEN = 9         /* int64 [n_qnodes]     tokens visible to the last new token of the q-node           */
+} mv_plan_table_id;
+
+typedef struct {
+  int64_t n_nodes, n_new_tokens, n_qnodes, n_segs;
+  int64_t decode_ready;        /* 1 if every q-node has exactly one new token (mv_dag_decode_attn applies) */
+  int64_t prefill_ready;       /* 1 if no node holds older tokens (mv_dag_prefill_attn applies)            */
+  int64_t n_items;             /* decode: (KV chunk, row set) work items per KV head                        */
+  int64_t n_partials;          /* decode: split-KV partial results per query head                          */
+  int64_t chunk_tokens;        /* decode: chunk length used                                                 */
+  int64_t unique_kv_tokens;    /* tokens of every node at least one row sees, each once                    */
+  int64_t per_row_kv_tokens;   /* sum over rows of visible tokens                                          */
+  int64_t n_q_tiles;           /* prefill: query tiles                                                      */
+  int64_t visible_pairs;       /* prefill: allowed (query, key) pairs                                      */
+  int64_t tile_pairs;          /* prefill: (query, key) pairs inside the KV ranges the kernel walks,
+                                  rounded up to whole 128x64 tiles                                         */
+  int64_t max_page_id;         /* largest page id referenced                                                */
+} mv_plan_stats;
+
+enum { MV_OP_ROPE_WRITE_KV = 0, MV_OP_DECODE_ATTN = 1, MV_OP_PREFILL_ATTN = 2 };
+
+/* DAG -> segment planner (Eq. 1 layering; Eq. 3 / Sec. 4.3 visibility; Sec. 4.2 positions; Sec. 3.2 KV index
+ * lists).  Host only, integers only, deterministic.
+ *   batch  host, read during the call only.
+ *   plan   in/out: if *plan is NULL a new plan is created; otherwise the existing plan is re-planned in
+ *          place and its host buffers are reused (no allocation once they are large enough).  The caller
+ *          must not re-plan while an mv_plan_upload of the same plan is still in flight on a stream.
+ * Errors: MV_ERR_INVALID_ARG, MV_ERR_NOT_TOPOLOGICAL, MV_ERR_PAGE_CAPACITY.  On error *plan is unchanged
+ * if it was NULL and left in an unusable-but-destroyable state otherwise. */
+mv_status mv_plan_dag(const mv_dag_batch* batch, mv_plan** plan);
+
+/* Canonical table access for parity checks.  *host_ptr points into the plan; *count is in elements. */
+mv_status mv_plan_table(const mv_plan* plan, int which, const void** host_ptr, int64_t* count);
+
+mv_status mv_plan_get_stats(const mv_plan* plan, mv_plan_stats* stats);
+
+/* Bytes of device memory the plan's kernel tables need (positions, slots, page ids, work lists). */
+size_t mv_plan_device_bytes(const mv_plan* plan);
+
+/* Asynchronous host->device copy of the plan's kernel tables into `device_buf` (device, caller-owned,
+ * 256-byte aligned, at least mv_plan_device_bytes(plan) bytes).  The plan remembers device_buf; the
+ * kernel calls below read the tables from there, so device_buf must stay valid and unmodified while
+ * calls that use this plan are in flight.  Errors: MV_ERR_WORKSPACE, MV_ERR_CUDA. */
+mv_status mv_plan_upload(mv_plan* plan, void* device_buf, size_t device_buf_bytes, void* cuda_stream);
+
+void mv_plan_destroy(mv_plan* plan);
+
+/* Workspace bytes (device, caller-owned, 256-byte aligned) an op needs for this plan and geometry.
+ * MV_OP_DECODE_ATTN: split-KV partial outputs and softmax statistics.  The other ops need none (0). */
+size_t mv_workspace_bytes(const mv_plan* plan, const mv_attn_geom* geom, int op);
+
+/* RoPE with adaptive positions fused into the KV-cache write (P(i) of Eq. 2 at the indices of Sec. 4.2).
+ * For new token t (n = n_new_tokens of the plan):
+ *   q_rot[t] = RoPE(q[t], pos_id[t]);  k_pages[slot[t]] = RoPE(k[t], pos_id[t]);  v_pages[slot[t]] = v[t].
+ * RoPE pairs element i with i + head_dim/2; the angle pos * rope_base^(-2i/head_dim) and its cos / sin are
+ * evaluated in double precision and rounded to float; the rotation is float; results are stored in `dtype`.
+ *   q       device [n][n_q_heads][head_dim]   raw queries, or NULL (then q_rot is not written)
+ *   k, v    device [n][n_kv_heads][head_dim]  raw keys / values
+ *   q_rot   device [n][n_q_heads][head_dim]   out (may alias q), or NULL with q
+ *   k_pages, v_pages  device pools, updated in place at the new tokens' slots
+ * Requires mv_plan_upload first.  Errors: MV_ERR_INVALID_ARG, MV_ERR_UNSUPPORTED, MV_ERR_CUDA. */
+mv_status mv_rope_write_kv(const mv_plan* plan, const mv_attn_geom* geom, const void* q, const void* k,
+                           const void* v, void* q_rot, void* k_pages, void* v_pages, void* cuda_stream);
+
+/* Multi-branch decode attention (Eq. 2 with the DAG mask of Eq. 3 over a shared paged cache, Sec. 4.3
+ * Fork / Join): for every row r (the single new token of a frontier node v) and query head h,
+ *   out[r][h] = sum_j softmax_j(sm_scale * <q_rot[r][h], K_j>) V_j
+ * over all tokens j of the nodes visible to v, the row's own just-written token included, so
+ * mv_rope_write_kv must precede this call in stream order.  Pages shared by several rows of a request
+ * (prefix, common ancestors) are read once per KV head and serve all those rows and the whole GQA group.
+ *   q_rot   device [n_rows][n_q_heads][head_dim]  bf16
+ *   k_pages, v_pages  device pools, bf16
+ *   out     device [n_rows][n_q_heads][head_dim]  bf16
+ *   workspace device, mv_workspace_bytes(plan, geom, MV_OP_DECODE_ATTN) bytes; contents are scratch
+ * dtype must be MV_BF16 and the plan decode_ready, else MV_ERR_UNSUPPORTED. */
+mv_status mv_dag_decode_attn(const mv_plan* plan, const mv_attn_geom* geom, const void* q_rot,
+                             const void* k_pages, const void* v_pages, void* out, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream);
+
+/* Topology-masked prefill attention over a flattened DAG sequence (Eq. 3; the training-time layout of
+ * Sec. 4.2 and the engine's re-prefill): all tokens of the batch are new and contiguous in
+ * (request, node, token) order;
+ *   out[i][h] = sum_j softmax_j(sm_scale * <q_rot[i][h], k_rot[j]> + M_ij) v[j],
+ * M_ij = 0 iff token j belongs to a node visible to node(i) and, inside node(i) itself, j <= i.
+ * Key/value ranges no query of a tile may see are never visited (tile skipping).
+ *   q_rot  device [T][n_q_heads][head_dim]   position-embedded queries
+ *   k_rot  device [T][n_kv_heads][head_dim]  position-embedded keys
+ *   v      device [T][n_kv_heads][head_dim]
+ *   out    device [T][n_q_heads][head_dim]
+ * dtype MV_F32 runs a float32 SIMT kernel, MV_BF16 the tensor-core kernel (float32 accumulation).
+ * The plan must be prefill_ready, else MV_ERR_UNSUPPORTED.  workspace may be NULL (none needed). */
+mv_status mv_dag_prefill_attn(const mv_plan* plan, const mv_attn_geom* geom, const void* q_rot,
+                              const void* k_rot, const void* v, void* out, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream);
+
+/* One decode step with HOST inputs and outputs (the end-to-end form of the path: Sec. 4.3 Phase II, one
+ * frontier step).  Copies q, k, v (host, preferably page-locked, [n_rows][heads][head_dim]) to the device
+ * staging buffer, uploads the plan, runs mv_rope_write_kv and mv_dag_decode_attn on `cuda_stream`, copies
+ * `out` back to host memory and returns after enqueueing everything (asynchronous; synchronise the stream
+ * before reading out_host).
+ *   staging  device, caller-owned, mv_decode_step_staging_bytes(plan, geom) bytes, 256-byte aligned; holds
+ *            the plan tables, q/k/v/out device copies and the decode workspace
+ *   k_pages, v_pages  device pools (the resident KV cache) */
+size_t mv_decode_step_staging_bytes(const mv_plan* plan, const mv_attn_geom* geom);
+mv_status mv_decode_step_host(mv_plan* plan, const mv_attn_geom* geom, const void* q_host, const void* k_host,
+                              const void* v_host, void* out_host, void* k_pages, void* v_pages, void* staging,
+                              size_t staging_bytes, void* cuda_stream);
+
+const char* mv_status_string(mv_status s);
+
+/* Number of kernel launches the library has issued in this process since load (diagnostic counter). */
+int64_t mv_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MEDVERSE_ATTN_H_ */

@@ -1,0 +1,224 @@
+"""Thin ctypes binding over the C ABI of ``libmedverse_attn.so`` (argument marshalling only).
+
+Every step of the path runs inside the library; PyTorch is used for device memory and streams.
+Importing this module loads the library and raises if it has not been built: there is no fallback.
+Function names mirror the C entry points declared in ``include/medverse_attn.h``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmedverse_attn.so")
+
+MV_OK = 0
+STATUS_NAMES = {0: "MV_OK", 1: "MV_ERR_INVALID_ARG", 2: "MV_ERR_NOT_TOPOLOGICAL", 3: "MV_ERR_PAGE_CAPACITY",
+                4: "MV_ERR_UNSUPPORTED", 5: "MV_ERR_WORKSPACE", 6: "MV_ERR_CUDA", 7: "MV_ERR_TIMEOUT"}
+MV_F32, MV_BF16 = 0, 1
+OP_ROPE_WRITE_KV, OP_DECODE_ATTN, OP_PREFILL_ATTN = 0, 1, 2
+TABLES = {"layer": (0, np.int32), "pos_start": (1, np.int32), "pos_id": (2, np.int32), "slot": (3, np.int64),
+          "qnode": (4, np.int32), "qnode_tok_off": (5, np.int32), "seg_off": (6, np.int32),
+          "seg_node": (7, np.int32), "seg_len": (8, np.int32), "kv_len": (9, np.int64)}
+
+EXPORTS = ["mv_plan_dag", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_bytes", "mv_plan_upload",
+           "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
+           "mv_dag_prefill_attn", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_status_string",
+           "mv_launch_count"]
+
+
+class MvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class _DagBatch(C.Structure):
+    _fields_ = [("n_req", C.c_int32), ("node_off", C.c_void_p), ("node_len", C.c_void_p), ("node_new", C.c_void_p),
+                ("parent_off", C.c_void_p), ("parent_idx", C.c_void_p), ("page_off", C.c_void_p),
+                ("page_idx", C.c_void_p), ("page_size", C.c_int32), ("vis_mode", C.c_int32), ("pos_mode", C.c_int32),
+                ("chunk_tokens", C.c_int32)]
+
+
+class _Geom(C.Structure):
+    _fields_ = [("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("page_size", C.c_int32),
+                ("num_pages", C.c_int64), ("dtype", C.c_int32), ("sm_scale", C.c_float), ("rope_base", C.c_double)]
+
+
+class _Stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "n_nodes", "n_new_tokens", "n_qnodes", "n_segs", "decode_ready", "prefill_ready", "n_items", "n_partials",
+        "chunk_tokens", "unique_kv_tokens", "per_row_kv_tokens", "n_q_tiles", "visible_pairs", "tile_pairs",
+        "max_page_id")]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_07529_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+    lib.mv_plan_dag.argtypes = [C.POINTER(_DagBatch), C.POINTER(vp)]
+    lib.mv_plan_table.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(i64)]
+    lib.mv_plan_get_stats.argtypes = [vp, C.POINTER(_Stats)]
+    lib.mv_plan_device_bytes.argtypes = [vp]
+    lib.mv_plan_device_bytes.restype = sz
+    lib.mv_plan_upload.argtypes = [vp, vp, sz, vp]
+    lib.mv_plan_destroy.argtypes = [vp]
+    lib.mv_plan_destroy.restype = None
+    lib.mv_workspace_bytes.argtypes = [vp, C.POINTER(_Geom), C.c_int]
+    lib.mv_workspace_bytes.restype = sz
+    lib.mv_rope_write_kv.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 7
+    lib.mv_dag_decode_attn.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp, sz, vp]
+    lib.mv_dag_prefill_attn.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp, sz, vp]
+    lib.mv_decode_step_staging_bytes.argtypes = [vp, C.POINTER(_Geom)]
+    lib.mv_decode_step_staging_bytes.restype = sz
+    lib.mv_decode_step_host.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 7 + [sz, vp]
+    lib.mv_status_string.argtypes = [C.c_int]
+    lib.mv_status_string.restype = C.c_char_p
+    lib.mv_launch_count.argtypes = []
+    lib.mv_launch_count.restype = i64
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if fn.restype is C.c_int and name not in ("mv_plan_destroy",):
+            fn.restype = C.c_int
+    return lib
+
+
+lib = _load()
+
+
+def _check(status: int, where: str):
+    if status != MV_OK:
+        raise MvError(int(status), where)
+
+
+def _i32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _ptr(t):
+    """Device (or host) pointer of a torch tensor / numpy array / None / int."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def make_geom(n_q_heads, n_kv_heads, head_dim, num_pages, dtype, page_size=16, sm_scale=0.0, rope_base=10000.0) -> _Geom:
+    code = {"f32": MV_F32, "bf16": MV_BF16}[dtype] if isinstance(dtype, str) else int(dtype)
+    return _Geom(n_q_heads, n_kv_heads, head_dim, page_size, int(num_pages), code, float(sm_scale), float(rope_base))
+
+
+def geom_of(workload) -> _Geom:
+    g = workload.geom
+    return make_geom(g.n_q_heads, g.n_kv_heads, g.head_dim, workload.batch.num_pages, g.dtype, g.page_size, 0.0, g.rope_base)
+
+
+class Plan:
+    """Owner of an ``mv_plan*``.  ``Plan(batch)`` plans; ``plan.replan(batch)`` recycles the same object."""
+
+    def __init__(self, batch=None, chunk_tokens: int = 0):
+        self._h = C.c_void_p(None)
+        self._keep = None
+        if batch is not None:
+            self.replan(batch, chunk_tokens)
+
+    def replan(self, batch, chunk_tokens: int = 0):
+        arrs = [_i32(getattr(batch, n)) for n in ("node_off", "node_len", "node_new", "parent_off", "parent_idx",
+                                                   "page_off", "page_idx")]
+        self._keep = arrs
+        b = _DagBatch(int(batch.n_req), *[a.ctypes.data for a in arrs], int(batch.page_size), int(batch.vis_mode),
+                      int(batch.pos_mode), int(chunk_tokens))
+        _check(lib.mv_plan_dag(C.byref(b), C.byref(self._h)), "mv_plan_dag")
+        return self
+
+    @property
+    def handle(self):
+        return self._h
+
+    def table(self, name: str) -> np.ndarray:
+        which, dt = TABLES[name]
+        p, n = C.c_void_p(), C.c_int64()
+        _check(lib.mv_plan_table(self._h, which, C.byref(p), C.byref(n)), "mv_plan_table")
+        if n.value == 0:
+            return np.zeros(0, dt)
+        buf = (C.c_char * (n.value * np.dtype(dt).itemsize)).from_address(p.value)
+        return np.frombuffer(buf, dtype=dt).copy()
+
+    def stats(self) -> dict:
+        s = _Stats()
+        _check(lib.mv_plan_get_stats(self._h, C.byref(s)), "mv_plan_get_stats")
+        return {n: int(getattr(s, n)) for n, _ in _Stats._fields_}
+
+    def device_bytes(self) -> int:
+        return int(lib.mv_plan_device_bytes(self._h))
+
+    def upload(self, device_buf, stream=None):
+        _check(lib.mv_plan_upload(self._h, _ptr(device_buf), device_buf.numel() * device_buf.element_size(),
+                                  _stream_ptr(stream)), "mv_plan_upload")
+
+    def workspace_bytes(self, geom: _Geom, op: int) -> int:
+        return int(lib.mv_workspace_bytes(self._h, C.byref(geom), op))
+
+    def destroy(self):
+        if self._h:
+            lib.mv_plan_destroy(self._h)
+            self._h = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def mv_plan_dag(batch, chunk_tokens: int = 0) -> Plan:
+    return Plan(batch, chunk_tokens)
+
+
+def mv_rope_write_kv(plan: Plan, geom: _Geom, q, k, v, q_rot, k_pages, v_pages, stream=None):
+    _check(lib.mv_rope_write_kv(plan.handle, C.byref(geom), _ptr(q), _ptr(k), _ptr(v), _ptr(q_rot), _ptr(k_pages),
+                                _ptr(v_pages), _stream_ptr(stream)), "mv_rope_write_kv")
+
+
+def mv_dag_decode_attn(plan: Plan, geom: _Geom, q_rot, k_pages, v_pages, out, workspace, stream=None):
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.mv_dag_decode_attn(plan.handle, C.byref(geom), _ptr(q_rot), _ptr(k_pages), _ptr(v_pages), _ptr(out),
+                                  _ptr(workspace), nbytes, _stream_ptr(stream)), "mv_dag_decode_attn")
+
+
+def mv_dag_prefill_attn(plan: Plan, geom: _Geom, q_rot, k_rot, v, out, workspace=None, stream=None):
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.mv_dag_prefill_attn(plan.handle, C.byref(geom), _ptr(q_rot), _ptr(k_rot), _ptr(v), _ptr(out),
+                                   _ptr(workspace), nbytes, _stream_ptr(stream)), "mv_dag_prefill_attn")
+
+
+def mv_decode_step_staging_bytes(plan: Plan, geom: _Geom) -> int:
+    return int(lib.mv_decode_step_staging_bytes(plan.handle, C.byref(geom)))
+
+
+def mv_decode_step_host(plan: Plan, geom: _Geom, q_host, k_host, v_host, out_host, k_pages, v_pages, staging, stream=None):
+    _check(lib.mv_decode_step_host(plan.handle, C.byref(geom), _ptr(q_host), _ptr(k_host), _ptr(v_host), _ptr(out_host),
+                                   _ptr(k_pages), _ptr(v_pages), _ptr(staging),
+                                   staging.numel() * staging.element_size(), _stream_ptr(stream)), "mv_decode_step_host")
+
+
+def mv_launch_count() -> int:
+    return int(lib.mv_launch_count())
+
+
+def mv_status_string(status: int) -> str:
+    return lib.mv_status_string(int(status)).decode()

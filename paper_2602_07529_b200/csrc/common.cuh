@@ -1,0 +1,74 @@
+// Shared device / launcher helpers of the library (sm_100a only).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+
+#include "plan_internal.h"
+
+namespace mv {
+
+extern std::atomic<int64_t> g_launches;  // kernels launched by this library since load
+
+inline mv_status check_geom(const mv_attn_geom* g) {
+  if (!g) return MV_ERR_INVALID_ARG;
+  if (g->n_q_heads <= 0 || g->n_kv_heads <= 0 || g->num_pages < 0) return MV_ERR_INVALID_ARG;
+  if (g->dtype != MV_F32 && g->dtype != MV_BF16) return MV_ERR_INVALID_ARG;
+  if (g->head_dim != 64 && g->head_dim != 128) return MV_ERR_UNSUPPORTED;
+  if (g->page_size != 16) return MV_ERR_UNSUPPORTED;
+  if (g->n_q_heads % g->n_kv_heads != 0) return MV_ERR_UNSUPPORTED;
+  return MV_OK;
+}
+
+inline float softmax_scale(const mv_attn_geom* g) {
+  return g->sm_scale != 0.f ? g->sm_scale : 1.0f / sqrtf(float(g->head_dim));
+}
+
+template <typename T>
+inline const T* table(const mv_plan* p, size_t off) {
+  return reinterpret_cast<const T*>(static_cast<const char*>(p->device_buf) + off);
+}
+
+// ---- small PTX wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+// 16-byte asynchronous global->shared copy; src_bytes < 16 zero-fills the remainder (0 = all zeros).
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+// D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+
+}  // namespace mv

@@ -1,0 +1,430 @@
+// DAG -> segment planner: host only, integers only, deterministic.
+//
+// Turns each request's node graph into (i) frontier layers (Eq. 1: a transition fires once all of its
+// input places are marked), (ii) visibility sets (Eq. 3 mask / Sec. 3.2 path history / Sec. 4.3 Join
+// as a set union), (iii) adaptive position indices (Sec. 4.2), (iv) the KV index list of every active
+// branch as segment + page tables (the `k` of a Petri-net token, Sec. 3.2), and (v) the private work
+// lists of the decode and prefill kernels.
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <numeric>
+
+#include "plan_internal.h"
+
+namespace {
+
+using mv::ItemRow;
+using mv::KvRange;
+using mv::QTile;
+using mv::WorkItem;
+
+struct Bits {  // dense bitset rows, n_words per node
+  int n_words = 0;
+  std::vector<uint64_t> w;
+  void reset(int n_nodes) {
+    n_words = (n_nodes + 63) / 64;
+    w.assign(size_t(n_nodes) * n_words, 0);
+  }
+  uint64_t* row(int v) { return w.data() + size_t(v) * n_words; }
+  const uint64_t* row(int v) const { return w.data() + size_t(v) * n_words; }
+  void set(int v, int u) { row(v)[u >> 6] |= (uint64_t(1) << (u & 63)); }
+  bool get(int v, int u) const { return (row(v)[u >> 6] >> (u & 63)) & 1; }
+};
+
+size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+mv_status check_batch(const mv_dag_batch* b) {
+  if (!b || b->n_req < 0) return MV_ERR_INVALID_ARG;
+  if (!b->node_off) return MV_ERR_INVALID_ARG;
+  if (b->page_size != 16) return MV_ERR_INVALID_ARG;
+  if (b->vis_mode != MV_VIS_ANCESTORS && b->vis_mode != MV_VIS_LAYERWISE) return MV_ERR_INVALID_ARG;
+  if (b->pos_mode != MV_POS_MAX_PARENT_END && b->pos_mode != MV_POS_FRONTIER_ALIGNED) return MV_ERR_INVALID_ARG;
+  if (b->chunk_tokens < 0 || (b->chunk_tokens % b->page_size) != 0) return MV_ERR_INVALID_ARG;
+  if (b->node_off[0] != 0) return MV_ERR_INVALID_ARG;
+  for (int r = 0; r < b->n_req; ++r)
+    if (b->node_off[r + 1] < b->node_off[r]) return MV_ERR_INVALID_ARG;
+  const int n_nodes = b->node_off[b->n_req];
+  if (n_nodes > 0 && (!b->node_len || !b->node_new || !b->parent_off || !b->page_off)) return MV_ERR_INVALID_ARG;
+  if (n_nodes == 0) return MV_OK;
+  if (b->parent_off[0] != 0 || b->page_off[0] != 0) return MV_ERR_INVALID_ARG;
+  for (int g = 0; g < n_nodes; ++g) {
+    if (b->node_len[g] < 0 || b->node_new[g] < 0) return MV_ERR_INVALID_ARG;
+    if (b->parent_off[g + 1] < b->parent_off[g] || b->page_off[g + 1] < b->page_off[g]) return MV_ERR_INVALID_ARG;
+  }
+  if (b->parent_off[n_nodes] > 0 && !b->parent_idx) return MV_ERR_INVALID_ARG;
+  if (b->page_off[n_nodes] > 0 && !b->page_idx) return MV_ERR_INVALID_ARG;
+  return MV_OK;
+}
+
+}  // namespace
+
+extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
+  if (!out) return MV_ERR_INVALID_ARG;
+  mv_status st = check_batch(b);
+  if (st != MV_OK) return st;
+
+  const int ps = b->page_size;
+  const int n_nodes = b->node_off[b->n_req];
+
+  // ---- validation that needs the graph: topological numbering, page capacity, page ids
+  int64_t max_page = -1;
+  for (int r = 0; r < b->n_req; ++r) {
+    const int lo = b->node_off[r], hi = b->node_off[r + 1];
+    for (int g = lo; g < hi; ++g) {
+      for (int e = b->parent_off[g]; e < b->parent_off[g + 1]; ++e) {
+        const int p = b->parent_idx[e];
+        if (p < 0 || p >= g - lo) return MV_ERR_NOT_TOPOLOGICAL;
+      }
+      const int64_t tot = int64_t(b->node_len[g]) + b->node_new[g];
+      const int64_t n_pages = b->page_off[g + 1] - b->page_off[g];
+      if (n_pages * ps < tot) return MV_ERR_PAGE_CAPACITY;
+      for (int e = b->page_off[g]; e < b->page_off[g + 1]; ++e) {
+        if (b->page_idx[e] < 0) return MV_ERR_INVALID_ARG;
+        max_page = std::max<int64_t>(max_page, b->page_idx[e]);
+      }
+    }
+  }
+
+  mv_plan* P = *out;
+  const bool created = (P == nullptr);
+  if (created) {
+    P = new (std::nothrow) mv_plan();
+    if (!P) return MV_ERR_INVALID_ARG;
+  }
+  P->valid = false;
+  P->device_buf = nullptr;
+  P->page_size = ps;
+  P->layer.assign(n_nodes, 0);
+  P->pos_start.assign(n_nodes, 0);
+  P->pos_id.clear(); P->slot.clear(); P->qnode.clear();
+  P->qnode_tok_off.assign(1, 0);
+  P->seg_off.assign(1, 0);
+  P->seg_node.clear(); P->seg_len.clear(); P->kv_len.clear();
+  P->items.clear(); P->item_rows.clear(); P->row_part_off.clear();
+  P->q_tiles.clear(); P->kv_ranges.clear();
+  P->page_idx.assign(b->page_idx, b->page_idx + (n_nodes ? b->page_off[n_nodes] : 0));
+  mv_plan_stats S{};
+  S.n_nodes = n_nodes;
+  S.max_page_id = max_page;
+
+  bool decode_ready = true, prefill_ready = true;
+  for (int g = 0; g < n_nodes; ++g) {
+    if (b->node_new[g] > 1) decode_ready = false;
+    if (b->node_len[g] != 0) prefill_ready = false;
+  }
+
+  // ---- pass 1 (per request): layers, visibility, positions, canonical tables
+  Bits vis;
+  std::vector<int32_t> pos_end, layer_end;
+  std::vector<int64_t> node_tok_start(n_nodes, 0);  // flattened index of a node's first NEW token
+  std::vector<std::vector<int32_t>> rows_of_node;    // decode: rows that see each node (request local)
+  struct PendingItem { int32_t page_begin, n_tokens, row_begin, n_rows; };
+  int64_t unique_tokens = 0, per_row_tokens = 0, visible_pairs = 0, tile_pairs = 0;
+  std::vector<int32_t> row_parts;  // per row: number of partials
+  std::vector<std::vector<int32_t>> item_row_lists;  // parallel to P->items before sorting
+
+  // automatic chunk length: aim for a few work items per CTA slot, assuming 8 KV heads
+  int chunk = b->chunk_tokens;
+  if (chunk == 0 && decode_ready) {
+    int64_t total_unique = 0;
+    for (int r = 0; r < b->n_req; ++r) {
+      // cheap upper bound: all nodes with tokens in requests that have a frontier
+      const int lo = b->node_off[r], hi = b->node_off[r + 1];
+      bool has_new = false;
+      for (int g = lo; g < hi; ++g) has_new |= b->node_new[g] > 0;
+      if (!has_new) continue;
+      for (int g = lo; g < hi; ++g) total_unique += b->node_len[g] + b->node_new[g];
+    }
+    int64_t c = (total_unique * 8) / (148 * 2 * 6);
+    c = ((c + 63) / 64) * 64;
+    chunk = int(std::min<int64_t>(1024, std::max<int64_t>(256, c)));
+  }
+  if (chunk == 0) chunk = 256;
+  S.chunk_tokens = chunk;
+
+  int64_t new_tok_count = 0;
+  for (int r = 0; r < b->n_req; ++r) {
+    const int lo = b->node_off[r], hi = b->node_off[r + 1], n = hi - lo;
+    if (n == 0) continue;
+    int32_t* layer = P->layer.data() + lo;
+    int32_t* pstart = P->pos_start.data() + lo;
+    // Eq. 1: layer(v) = 0 for roots, else 1 + max over parents
+    int max_layer = 0;
+    for (int v = 0; v < n; ++v) {
+      int L = 0;
+      for (int e = b->parent_off[lo + v]; e < b->parent_off[lo + v + 1]; ++e)
+        L = std::max(L, layer[b->parent_idx[e]] + 1);
+      layer[v] = L;
+      max_layer = std::max(max_layer, L);
+    }
+    // visibility sets
+    vis.reset(n);
+    if (b->vis_mode == MV_VIS_ANCESTORS) {
+      for (int v = 0; v < n; ++v) {
+        uint64_t* rv = vis.row(v);
+        for (int e = b->parent_off[lo + v]; e < b->parent_off[lo + v + 1]; ++e) {
+          const uint64_t* rp = vis.row(b->parent_idx[e]);
+          for (int w = 0; w < vis.n_words; ++w) rv[w] |= rp[w];
+        }
+        vis.set(v, v);
+      }
+    } else {
+      for (int v = 0; v < n; ++v) {
+        for (int u = 0; u < n; ++u)
+          if (layer[u] < layer[v]) vis.set(v, u);
+        vis.set(v, v);
+      }
+    }
+    // Sec. 4.2 positions
+    pos_end.assign(n, 0);
+    if (b->pos_mode == MV_POS_MAX_PARENT_END) {
+      for (int v = 0; v < n; ++v) {
+        int32_t s = 0;
+        for (int e = b->parent_off[lo + v]; e < b->parent_off[lo + v + 1]; ++e)
+          s = std::max(s, pos_end[b->parent_idx[e]]);
+        pstart[v] = s;
+        pos_end[v] = s + b->node_len[lo + v] + b->node_new[lo + v];
+      }
+    } else {
+      layer_end.assign(max_layer + 2, 0);
+      for (int L = 0; L <= max_layer; ++L) {
+        int32_t e_max = 0;
+        for (int v = 0; v < n; ++v) {
+          if (layer[v] != L) continue;
+          pstart[v] = layer_end[L];
+          pos_end[v] = pstart[v] + b->node_len[lo + v] + b->node_new[lo + v];
+          e_max = std::max(e_max, pos_end[v]);
+        }
+        layer_end[L + 1] = e_max;
+      }
+    }
+    // canonical per-token and per-q-node tables
+    const int64_t first_row_of_req = new_tok_count;
+    rows_of_node.assign(n, {});
+    std::vector<char> seen_by_frontier(n, 0);
+    for (int v = 0; v < n; ++v) {
+      const int g = lo + v;
+      node_tok_start[g] = new_tok_count;
+      const int nl = b->node_len[g], nn = b->node_new[g];
+      if (nn == 0) continue;
+      for (int t = nl; t < nl + nn; ++t) {
+        P->pos_id.push_back(pstart[v] + t);
+        const int64_t page = b->page_idx[b->page_off[g] + t / ps];
+        P->slot.push_back(page * ps + t % ps);
+      }
+      P->qnode.push_back(g);
+      int64_t kv = 0;
+      for (int u = 0; u < n; ++u) {
+        if (!vis.get(v, u)) continue;
+        const int32_t ln = b->node_len[lo + u] + b->node_new[lo + u];
+        P->seg_node.push_back(lo + u);
+        P->seg_len.push_back(ln);
+        kv += ln;
+        seen_by_frontier[u] = 1;
+        if (decode_ready) rows_of_node[u].push_back(int32_t(new_tok_count));
+      }
+      P->seg_off.push_back(int32_t(P->seg_node.size()));
+      P->kv_len.push_back(kv);
+      per_row_tokens += kv;  // decode: exactly the row's visible tokens
+      new_tok_count += nn;
+      P->qnode_tok_off.push_back(int32_t(new_tok_count));
+    }
+    for (int u = 0; u < n; ++u)
+      if (seen_by_frontier[u]) unique_tokens += b->node_len[lo + u] + b->node_new[lo + u];
+
+    // ---- decode work items of this request: (node chunk) x (rows that see the node)
+    if (decode_ready) {
+      const int64_t n_rows_req = new_tok_count - first_row_of_req;
+      row_parts.resize(size_t(new_tok_count), 0);
+      (void)n_rows_req;
+      for (int u = 0; u < n; ++u) {
+        const auto& rows = rows_of_node[u];
+        const int32_t L = b->node_len[lo + u] + b->node_new[lo + u];
+        if (rows.empty() || L == 0) continue;
+        const int n_pages = (L + ps - 1) / ps;
+        const int n_chunks = (L + chunk - 1) / chunk;
+        const int pages_per_chunk = (n_pages + n_chunks - 1) / n_chunks;
+        for (int c = 0; c * pages_per_chunk < n_pages; ++c) {
+          const int pb = c * pages_per_chunk;
+          const int pe = std::min(n_pages, pb + pages_per_chunk);
+          WorkItem it;
+          it.page_begin = b->page_off[lo + u] + pb;
+          it.n_tokens = std::min(L, pe * ps) - pb * ps;
+          it.row_begin = 0;
+          it.n_rows = int32_t(rows.size());
+          P->items.push_back(it);
+          std::vector<int32_t> rl;
+          rl.reserve(rows.size() * 2);
+          for (int32_t row : rows) {
+            rl.push_back(row);
+            rl.push_back(row_parts[row]++);  // partial index local to the row, made global below
+          }
+          item_row_lists.push_back(std::move(rl));
+        }
+      }
+    }
+
+    // ---- prefill tiles of this request
+    if (prefill_ready) {
+      // flattened start of every node of the request
+      for (int v = 0; v < n; ++v) {
+        const int g = lo + v;
+        const int32_t len_v = b->node_new[g];
+        if (len_v == 0) continue;
+        const int64_t v_start = node_tok_start[g];
+        // visible ranges in flattened order, adjacent ones merged
+        std::vector<KvRange> base;
+        int64_t vis_before = 0;  // visible tokens outside the node itself
+        for (int u = 0; u < n; ++u) {
+          if (u == v || !vis.get(v, u) || b->node_new[lo + u] == 0) continue;
+          const int32_t us = int32_t(node_tok_start[lo + u]);
+          const int32_t ul = b->node_new[lo + u];
+          vis_before += ul;
+          if (!base.empty() && base.back().kv_start + base.back().kv_len == us) base.back().kv_len += ul;
+          else base.push_back(KvRange{us, ul, 0, 0});
+        }
+        visible_pairs += vis_before * len_v + int64_t(len_v) * (len_v + 1) / 2;
+        for (int32_t q0 = 0; q0 < len_v; q0 += mv::kPrefillQTile) {
+          const int32_t ql = std::min<int32_t>(mv::kPrefillQTile, len_v - q0);
+          QTile qt;
+          qt.q_start = int32_t(v_start + q0);
+          qt.q_len = ql;
+          qt.range_begin = int32_t(P->kv_ranges.size());
+          // own causal range [v_start, q_start + q_len), placed in flattened order.  A fully visible
+          // range that ends exactly where the node starts is folded into it: every key before the
+          // node start precedes every query of the tile, so the causal test is vacuous there.
+          KvRange own{int32_t(v_start), q0 + ql, 1, 0};
+          size_t k = 0;
+          for (; k < base.size() && base[k].kv_start < own.kv_start; ++k) {
+            if (base[k].kv_start + base[k].kv_len == own.kv_start) {
+              own.kv_start = base[k].kv_start;
+              own.kv_len += base[k].kv_len;
+            } else {
+              P->kv_ranges.push_back(base[k]);
+            }
+          }
+          P->kv_ranges.push_back(own);
+          for (; k < base.size(); ++k) P->kv_ranges.push_back(base[k]);
+          qt.range_count = int32_t(P->kv_ranges.size()) - qt.range_begin;
+          for (int i = qt.range_begin; i < qt.range_begin + qt.range_count; ++i) {
+            const int64_t kl = P->kv_ranges[i].kv_len;
+            tile_pairs += int64_t(mv::kPrefillQTile) * (((kl + mv::kPrefillKvTile - 1) / mv::kPrefillKvTile) * mv::kPrefillKvTile);
+          }
+          P->q_tiles.push_back(qt);
+        }
+      }
+    }
+  }
+
+  // ---- decode: global partial slots, longest-first item order
+  if (decode_ready) {
+    const int64_t n_rows = new_tok_count;
+    row_parts.resize(size_t(n_rows), 0);
+    P->row_part_off.assign(size_t(n_rows) + 1, 0);
+    for (int64_t r = 0; r < n_rows; ++r) P->row_part_off[r + 1] = P->row_part_off[r] + row_parts[r];
+    std::vector<int32_t> order(P->items.size());
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t c) {
+      return P->items[a].n_tokens > P->items[c].n_tokens;
+    });
+    std::vector<WorkItem> sorted;
+    sorted.reserve(order.size());
+    for (int32_t i : order) {
+      WorkItem it = P->items[i];
+      it.row_begin = int32_t(P->item_rows.size());
+      const auto& rl = item_row_lists[i];
+      for (size_t k = 0; k < rl.size(); k += 2)
+        P->item_rows.push_back(ItemRow{rl[k], P->row_part_off[rl[k]] + rl[k + 1]});
+      sorted.push_back(it);
+    }
+    P->items.swap(sorted);
+    S.n_items = int64_t(P->items.size());
+    S.n_partials = P->row_part_off[n_rows];
+  }
+  // ---- prefill: heaviest query tiles first
+  if (prefill_ready) {
+    std::vector<int64_t> cost(P->q_tiles.size(), 0);
+    for (size_t i = 0; i < P->q_tiles.size(); ++i)
+      for (int k = 0; k < P->q_tiles[i].range_count; ++k) cost[i] += P->kv_ranges[P->q_tiles[i].range_begin + k].kv_len;
+    std::vector<int32_t> order(P->q_tiles.size());
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t c) { return cost[a] > cost[c]; });
+    std::vector<QTile> sorted;
+    sorted.reserve(order.size());
+    for (int32_t i : order) sorted.push_back(P->q_tiles[i]);
+    P->q_tiles.swap(sorted);
+    S.n_q_tiles = int64_t(P->q_tiles.size());
+    S.visible_pairs = visible_pairs;
+    S.tile_pairs = tile_pairs;
+  }
+
+  S.n_new_tokens = new_tok_count;
+  S.n_qnodes = int64_t(P->qnode.size());
+  S.n_segs = int64_t(P->seg_node.size());
+  S.decode_ready = decode_ready && new_tok_count > 0;
+  S.prefill_ready = prefill_ready && new_tok_count > 0;
+  S.unique_kv_tokens = unique_tokens;
+  S.per_row_kv_tokens = per_row_tokens;
+  P->stats = S;
+
+  // ---- device table layout
+  mv::DeviceLayout L;
+  size_t off = 0;
+  auto place = [&](size_t bytes) { size_t o = off; off = align256(off + bytes); return o; };
+  L.pos_id = place(P->pos_id.size() * sizeof(int32_t));
+  L.slot = place(P->slot.size() * sizeof(int64_t));
+  L.page_idx = place(P->page_idx.size() * sizeof(int32_t));
+  L.items = place(P->items.size() * sizeof(WorkItem));
+  L.item_rows = place(P->item_rows.size() * sizeof(ItemRow));
+  L.row_part_off = place(P->row_part_off.size() * sizeof(int32_t));
+  L.q_tiles = place(P->q_tiles.size() * sizeof(QTile));
+  L.kv_ranges = place(P->kv_ranges.size() * sizeof(KvRange));
+  L.total = std::max<size_t>(off, 256);
+  P->layout = L;
+  P->valid = true;
+  *out = P;
+  return MV_OK;
+}
+
+extern "C" mv_status mv_plan_table(const mv_plan* P, int which, const void** host_ptr, int64_t* count) {
+  if (!P || !P->valid || !host_ptr || !count) return MV_ERR_INVALID_ARG;
+  auto give32 = [&](const std::vector<int32_t>& v) { *host_ptr = v.data(); *count = int64_t(v.size()); return MV_OK; };
+  auto give64 = [&](const std::vector<int64_t>& v) { *host_ptr = v.data(); *count = int64_t(v.size()); return MV_OK; };
+  switch (which) {
+    case MV_TAB_LAYER: return give32(P->layer);
+    case MV_TAB_POS_START: return give32(P->pos_start);
+    case MV_TAB_POS_ID: return give32(P->pos_id);
+    case MV_TAB_SLOT: return give64(P->slot);
+    case MV_TAB_QNODE: return give32(P->qnode);
+    case MV_TAB_QNODE_TOK_OFF: return give32(P->qnode_tok_off);
+    case MV_TAB_SEG_OFF: return give32(P->seg_off);
+    case MV_TAB_SEG_NODE: return give32(P->seg_node);
+    case MV_TAB_SEG_LEN: return give32(P->seg_len);
+    case MV_TAB_KV_LEN: return give64(P->kv_len);
+    default: return MV_ERR_INVALID_ARG;
+  }
+}
+
+extern "C" mv_status mv_plan_get_stats(const mv_plan* P, mv_plan_stats* stats) {
+  if (!P || !P->valid || !stats) return MV_ERR_INVALID_ARG;
+  *stats = P->stats;
+  return MV_OK;
+}
+
+extern "C" size_t mv_plan_device_bytes(const mv_plan* P) { return (P && P->valid) ? P->layout.total : 0; }
+
+extern "C" const char* mv_status_string(mv_status s) {
+  switch (s) {
+    case MV_OK: return "MV_OK";
+    case MV_ERR_INVALID_ARG: return "MV_ERR_INVALID_ARG: null pointer, negative size, inconsistent offsets or bad enum";
+    case MV_ERR_NOT_TOPOLOGICAL: return "MV_ERR_NOT_TOPOLOGICAL: a parent index is not smaller than its child's index";
+    case MV_ERR_PAGE_CAPACITY: return "MV_ERR_PAGE_CAPACITY: a node's page list is too short for its tokens";
+    case MV_ERR_UNSUPPORTED: return "MV_ERR_UNSUPPORTED: geometry, dtype or batch shape not supported by this kernel";
+    case MV_ERR_WORKSPACE: return "MV_ERR_WORKSPACE: workspace or table buffer missing, too small or misaligned";
+    case MV_ERR_CUDA: return "MV_ERR_CUDA: a CUDA runtime call failed";
+    case MV_ERR_TIMEOUT: return "MV_ERR_TIMEOUT: a bounded device-side wait ran out";
+    default: return "unknown mv_status";
+  }
+}

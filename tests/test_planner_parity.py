@@ -1,0 +1,120 @@
+"""mv_plan_dag (host C++ planner, through the C ABI) against the oracle planner: bit-exact tables.
+Runs without a GPU: the planner is integer host code."""
+import re
+import os
+import ctypes
+
+import numpy as np
+import pytest
+
+from oracle import medverse_oracle as O
+from paper_2602_07529_b200 import synth, binding as B
+from helpers import batch_dict
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _compare(batch):
+    want = O.plan_tables(batch_dict(batch))
+    plan = B.Plan(batch)
+    for name in B.TABLES:
+        got = plan.table(name)
+        assert got.dtype == want[name].dtype, name
+        assert np.array_equal(got, want[name]), name
+    return plan, want
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "medverse_attn.h")).read()
+    declared = set(re.findall(r"\b(mv_[a-z_]+)\s*\(", hdr))
+    assert declared, "no declarations parsed"
+    assert declared == set(B.EXPORTS)
+    lib = ctypes.CDLL(B.LIB_PATH)
+    for name in sorted(declared):
+        assert hasattr(lib, name), name
+    assert B.mv_status_string(2).startswith("MV_ERR_NOT_TOPOLOGICAL")
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_configs_bit_exact(cfg):
+    wl = synth.CONFIGS[cfg]()
+    plan, want = _compare(wl.batch)
+    st = plan.stats()
+    assert st["n_new_tokens"] == len(want["pos_id"])
+    assert st["decode_ready"] == (1 if wl.kind == "decode" else 0)
+    assert st["prefill_ready"] == (1 if wl.kind == "prefill" else 0)
+    if wl.kind == "decode":
+        assert st["per_row_kv_tokens"] == int(want["kv_len"].sum())
+        vis_nodes = [want["seg_node"][want["seg_off"][i]:want["seg_off"][i + 1]] for i in range(len(want["qnode"]))]
+        assert st["unique_kv_tokens"] == synth.unique_visible_tokens(wl.batch, vis_nodes)
+
+
+def test_config3_other_frontiers():
+    for fl in (1, 2):
+        _compare(synth.config3(frontier_layer=fl).batch)
+
+
+@pytest.mark.parametrize("vis_mode", [0, 1])
+@pytest.mark.parametrize("pos_mode", [0, 1])
+def test_random_dags_bit_exact(vis_mode, pos_mode):
+    for seed in range(250):
+        for kind in ("decode", "prefill"):
+            wl = synth.random_dag_workload(seed, kind, n_req=3, max_nodes=12, max_len=70, vis_mode=vis_mode, pos_mode=pos_mode)
+            _compare(wl.batch)
+
+
+def test_replan_recycles_object():
+    plan = B.Plan(synth.config2().batch)
+    a = plan.table("slot")
+    plan.replan(synth.config1().batch)
+    want = O.plan_tables(batch_dict(synth.config1().batch))
+    assert np.array_equal(plan.table("pos_id"), want["pos_id"])
+    plan.replan(synth.config2().batch)
+    assert np.array_equal(plan.table("slot"), a)
+
+
+def test_prefill_visible_pairs_match_dense_mask():
+    """The planner's count of allowed (query, key) pairs equals the population of the oracle's dense mask."""
+    for seed in range(20):
+        for vis_mode in (0, 1):
+            wl = synth.random_dag_workload(seed, "prefill", n_req=2, max_nodes=8, max_len=40, vis_mode=vis_mode)
+            b = wl.batch
+            total = 0
+            for r in range(b.n_req):
+                lo, hi = int(b.node_off[r]), int(b.node_off[r + 1])
+                parents = [b.parents_of(g) for g in range(lo, hi)]
+                lay = O.node_layers(parents)
+                vis = O.visible_sets(parents, lay, vis_mode)
+                tok_node = [v for v in range(hi - lo) for _ in range(int(b.node_new[lo + v]))]
+                tok_index = [t for v in range(hi - lo) for t in range(int(b.node_new[lo + v]))]
+                if tok_node:
+                    total += int(O.allowed_mask(tok_node, tok_index, vis).sum())
+            assert B.Plan(b).stats()["visible_pairs"] == total
+
+
+def test_error_statuses():
+    def status_of(batch):
+        with pytest.raises(B.MvError) as e:
+            B.Plan(batch)
+        return e.value.status
+    good = synth.build_batch([[([], 20, 0), ([0], 5, 1), ([0, 1], 3, 1)]])
+    B.Plan(good)
+    import copy
+    bad = copy.deepcopy(good); bad.parent_idx = np.asarray([1, 0, 1], np.int32)      # node 1 lists itself
+    assert status_of(bad) == 2
+    bad = copy.deepcopy(good); bad.parent_idx = np.asarray([0, 0, 2], np.int32)      # node 2 lists itself
+    assert status_of(bad) == 2
+    bad = copy.deepcopy(good); bad.page_off = np.asarray([0, 1, 2, 3], np.int32)     # 20 tokens in one page
+    assert status_of(bad) == 3
+    bad = copy.deepcopy(good); bad.node_len = np.asarray([20, -1, 3], np.int32)
+    assert status_of(bad) == 1
+    bad = copy.deepcopy(good); bad.page_size = 32
+    assert status_of(bad) == 1
+    bad = copy.deepcopy(good); bad.vis_mode = 7
+    assert status_of(bad) == 1
+    bad = copy.deepcopy(good); bad.page_idx = -bad.page_idx - 1
+    assert status_of(bad) == 1
+    # empty batch and empty request are fine
+    empty = synth.build_batch([])
+    assert B.Plan(empty).stats()["n_new_tokens"] == 0
+    assert B.Plan(synth.build_batch([[], [([], 3, 1)]])).stats()["n_new_tokens"] == 1
