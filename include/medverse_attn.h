@@ -157,16 +157,20 @@ size_t mv_workspace_bytes(const mv_plan* plan, const mv_attn_geom* geom, int op)
 
 /* RoPE with adaptive positions fused into the KV-cache write (P(i) of Eq. 2 at the indices of Sec. 4.2).
  * For new token t (n = n_new_tokens of the plan):
- *   q_rot[t] = RoPE(q[t], pos_id[t]);  k_pages[slot[t]] = RoPE(k[t], pos_id[t]);  v_pages[slot[t]] = v[t].
+ *   q_rot[t] = RoPE(q[t], pos_id[t]);  k_pages[slot[t]] = k_rot[t] = RoPE(k[t], pos_id[t]);  v_pages[slot[t]] = v[t].
  * RoPE pairs element i with i + head_dim/2; the angle pos * rope_base^(-2i/head_dim) and its cos / sin are
  * evaluated in double precision and rounded to float; the rotation is float; results are stored in `dtype`.
  *   q       device [n][n_q_heads][head_dim]   raw queries, or NULL (then q_rot is not written)
  *   k, v    device [n][n_kv_heads][head_dim]  raw keys / values
- *   q_rot   device [n][n_q_heads][head_dim]   out (may alias q), or NULL with q
- *   k_pages, v_pages  device pools, updated in place at the new tokens' slots
- * Requires mv_plan_upload first.  Errors: MV_ERR_INVALID_ARG, MV_ERR_UNSUPPORTED, MV_ERR_CUDA. */
+ *   q_rot   device [n][n_q_heads][head_dim]   out (may alias q); NULL exactly when q is NULL
+ *   k_rot   device [n][n_kv_heads][head_dim]  out, optional (NULL to skip; may alias k): the rotated keys in
+ *           token order, which is what mv_dag_prefill_attn reads
+ *   k_pages, v_pages  device pools, updated in place at the new tokens' slots; both NULL skips the cache
+ *           write (then k_rot must be given)
+ * Requires mv_plan_upload first.  Errors: MV_ERR_INVALID_ARG, MV_ERR_UNSUPPORTED, MV_ERR_WORKSPACE, MV_ERR_CUDA. */
 mv_status mv_rope_write_kv(const mv_plan* plan, const mv_attn_geom* geom, const void* q, const void* k,
-                           const void* v, void* q_rot, void* k_pages, void* v_pages, void* cuda_stream);
+                           const void* v, void* q_rot, void* k_rot, void* k_pages, void* v_pages,
+                           void* cuda_stream);
 
 /* Multi-branch decode attention (Eq. 2 with the DAG mask of Eq. 3 over a shared paged cache, Sec. 4.3
  * Fork / Join): for every row r (the single new token of a frontier node v) and query head h,

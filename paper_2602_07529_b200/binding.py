@@ -70,7 +70,7 @@ def _load():
     lib.mv_plan_destroy.restype = None
     lib.mv_workspace_bytes.argtypes = [vp, C.POINTER(_Geom), C.c_int]
     lib.mv_workspace_bytes.restype = sz
-    lib.mv_rope_write_kv.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 7
+    lib.mv_rope_write_kv.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 8
     lib.mv_dag_decode_attn.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp, sz, vp]
     lib.mv_dag_prefill_attn.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp, sz, vp]
     lib.mv_decode_step_staging_bytes.argtypes = [vp, C.POINTER(_Geom)]
@@ -189,9 +189,9 @@ def mv_plan_dag(batch, chunk_tokens: int = 0) -> Plan:
     return Plan(batch, chunk_tokens)
 
 
-def mv_rope_write_kv(plan: Plan, geom: _Geom, q, k, v, q_rot, k_pages, v_pages, stream=None):
-    _check(lib.mv_rope_write_kv(plan.handle, C.byref(geom), _ptr(q), _ptr(k), _ptr(v), _ptr(q_rot), _ptr(k_pages),
-                                _ptr(v_pages), _stream_ptr(stream)), "mv_rope_write_kv")
+def mv_rope_write_kv(plan: Plan, geom: _Geom, q, k, v, q_rot, k_rot, k_pages, v_pages, stream=None):
+    _check(lib.mv_rope_write_kv(plan.handle, C.byref(geom), _ptr(q), _ptr(k), _ptr(v), _ptr(q_rot), _ptr(k_rot),
+                                _ptr(k_pages), _ptr(v_pages), _stream_ptr(stream)), "mv_rope_write_kv")
 
 
 def mv_dag_decode_attn(plan: Plan, geom: _Geom, q_rot, k_pages, v_pages, out, workspace, stream=None):

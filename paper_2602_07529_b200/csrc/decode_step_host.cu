@@ -50,7 +50,7 @@ extern "C" mv_status mv_decode_step_host(mv_plan* P, const mv_attn_geom* g, cons
     (void)cudaGetLastError();
     return MV_ERR_CUDA;
   }
-  st = mv_rope_write_kv(P, g, base + L.q, base + L.k, base + L.v, base + L.q, k_pages, v_pages, cuda_stream);
+  st = mv_rope_write_kv(P, g, base + L.q, base + L.k, base + L.v, base + L.q, nullptr, k_pages, v_pages, cuda_stream);
   if (st != MV_OK) return st;
   st = mv_dag_decode_attn(P, g, base + L.q, k_pages, v_pages, base + L.out, base + L.ws,
                           mv_workspace_bytes(P, g, MV_OP_DECODE_ATTN), cuda_stream);

@@ -49,11 +49,12 @@ struct Vec16<__nv_bfloat16> {
 };
 
 template <typename T, int D>
-__global__ void __launch_bounds__(128) rope_write_kv_kernel(const T* __restrict__ q, const T* __restrict__ k,
-                                                            const T* __restrict__ v, T* __restrict__ q_rot,
-                                                            T* __restrict__ k_pages, T* __restrict__ v_pages,
-                                                            const int32_t* __restrict__ pos_id,
-                                                            const int64_t* __restrict__ slot, int n_tok, int Hq,
+__global__ void __launch_bounds__(128) rope_write_kv_kernel(const T* q, const T* k,
+                                                            const T* v, T* q_rot,
+                                                            T* k_rot, T* k_pages,
+                                                            T* v_pages,
+                                                            const int32_t* pos_id,
+                                                            const int64_t* slot, int n_tok, int Hq,
                                                             int Hkv, double neg_log2_base_2_over_d) {
   constexpr int HALF = D / 2;
   constexpr int N = Vec16<T>::N;
@@ -82,6 +83,8 @@ __global__ void __launch_bounds__(128) rope_write_kv_kernel(const T* __restrict_
     const int h = uu / CH, c = uu % CH;
     const T* src = is_q ? q + (int64_t(t) * Hq + h) * D : k + (int64_t(t) * Hkv + h) * D;
     T* dst = is_q ? q_rot + (int64_t(t) * Hq + h) * D : k_pages + (((page * Hkv + h) << 4) + off) * D;
+    T* dst2 = is_q ? nullptr : k_rot + (int64_t(t) * Hkv + h) * D;
+    const bool w1 = is_q || k_pages != nullptr, w2 = !is_q && k_rot != nullptr;
     float lo[N], hi[N], olo[N], ohi[N];
     Vec16<T>::load(src + c * N, lo);
     Vec16<T>::load(src + HALF + c * N, hi);
@@ -91,9 +94,16 @@ __global__ void __launch_bounds__(128) rope_write_kv_kernel(const T* __restrict_
       olo[i] = lo[i] * cc - hi[i] * ss;
       ohi[i] = hi[i] * cc + lo[i] * ss;
     }
-    Vec16<T>::store(dst + c * N, olo);
-    Vec16<T>::store(dst + HALF + c * N, ohi);
+    if (w1) {
+      Vec16<T>::store(dst + c * N, olo);
+      Vec16<T>::store(dst + HALF + c * N, ohi);
+    }
+    if (w2) {
+      Vec16<T>::store(dst2 + c * N, olo);
+      Vec16<T>::store(dst2 + HALF + c * N, ohi);
+    }
   }
+  if (v_pages == nullptr) return;
   // v is stored unrotated
   constexpr int VCH = D / N;
   for (int u = threadIdx.x; u < Hkv * VCH; u += blockDim.x) {
@@ -105,17 +115,19 @@ __global__ void __launch_bounds__(128) rope_write_kv_kernel(const T* __restrict_
 
 template <typename T>
 mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* q_rot,
-                 void* k_pages, void* v_pages, cudaStream_t st) {
+                 void* k_rot, void* k_pages, void* v_pages, cudaStream_t st) {
   const int n = int(P->stats.n_new_tokens);
   const int32_t* pos = mv::table<int32_t>(P, P->layout.pos_id);
   const int64_t* slot = mv::table<int64_t>(P, P->layout.slot);
   const double c = -2.0 * log2(g->rope_base) / double(g->head_dim);
   if (g->head_dim == 128)
-    rope_write_kv_kernel<T, 128><<<n, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_pages,
-                                                    (T*)v_pages, pos, slot, n, g->n_q_heads, g->n_kv_heads, c);
+    rope_write_kv_kernel<T, 128><<<n, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_rot,
+                                                    (T*)k_pages, (T*)v_pages, pos, slot, n, g->n_q_heads,
+                                                    g->n_kv_heads, c);
   else
-    rope_write_kv_kernel<T, 64><<<n, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_pages,
-                                                   (T*)v_pages, pos, slot, n, g->n_q_heads, g->n_kv_heads, c);
+    rope_write_kv_kernel<T, 64><<<n, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_rot,
+                                                   (T*)k_pages, (T*)v_pages, pos, slot, n, g->n_q_heads,
+                                                   g->n_kv_heads, c);
   mv::g_launches++;
   if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
   return MV_OK;
@@ -124,17 +136,20 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
 }  // namespace
 
 extern "C" mv_status mv_rope_write_kv(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k,
-                                      const void* v, void* q_rot, void* k_pages, void* v_pages, void* cuda_stream) {
+                                      const void* v, void* q_rot, void* k_rot, void* k_pages, void* v_pages,
+                                      void* cuda_stream) {
   if (!P || !P->valid) return MV_ERR_INVALID_ARG;
   mv_status st = mv::check_geom(g);
   if (st != MV_OK) return st;
   if (!P->device_buf) return MV_ERR_WORKSPACE;
   if (P->stats.n_new_tokens == 0) return MV_OK;
-  if (!k || !v || !k_pages || !v_pages) return MV_ERR_INVALID_ARG;
+  if (!k || !v) return MV_ERR_INVALID_ARG;
+  if ((k_pages == nullptr) != (v_pages == nullptr)) return MV_ERR_INVALID_ARG;
+  if (!k_pages && !k_rot) return MV_ERR_INVALID_ARG;
   if ((q == nullptr) != (q_rot == nullptr)) return MV_ERR_INVALID_ARG;
-  if (P->stats.max_page_id >= g->num_pages) return MV_ERR_INVALID_ARG;
+  if (k_pages && P->stats.max_page_id >= g->num_pages) return MV_ERR_INVALID_ARG;
   if (g->rope_base <= 0.0) return MV_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  return g->dtype == MV_BF16 ? launch<__nv_bfloat16>(P, g, q, k, v, q_rot, k_pages, v_pages, s)
-                             : launch<float>(P, g, q, k, v, q_rot, k_pages, v_pages, s);
+  return g->dtype == MV_BF16 ? launch<__nv_bfloat16>(P, g, q, k, v, q_rot, k_rot, k_pages, v_pages, s)
+                             : launch<float>(P, g, q, k, v, q_rot, k_rot, k_pages, v_pages, s);
 }
