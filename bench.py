@@ -186,12 +186,10 @@ def run_ours(args):
 
     # ---- ring of plans / table buffers so that re-planning never races an upload in flight
     RING = 4
-    plans = [B.Plan(b, args.chunk) for _ in range(RING)]
+    plans = [B.Plan(b, args.chunk, g.n_kv_heads, g.group) for _ in range(RING)]
     tables = [torch.empty(max(256, plans[0].device_bytes() * 2), dtype=torch.uint8, device=dev) for _ in range(RING)]
     ring_ev = [torch.cuda.Event() for _ in range(RING)]
-    arrs = plans[0]._keep
-    cb = B._DagBatch(int(b.n_req), *[a.ctypes.data for a in arrs], int(b.page_size), int(b.vis_mode), int(b.pos_mode),
-                     int(args.chunk))
+    cb = plans[0].c_batch
     stream = torch.cuda.current_stream()
     sp = C.c_void_p(stream.cuda_stream)
     geom = st.geom

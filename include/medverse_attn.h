@@ -80,6 +80,10 @@ typedef struct {
   int32_t vis_mode;          /* mv_vis_mode */
   int32_t pos_mode;          /* mv_pos_mode */
   int32_t chunk_tokens;      /* decode split-KV chunk length in tokens (multiple of page_size); 0 = automatic */
+  int32_t n_kv_heads;        /* scheduling hint: KV heads of the geometry the plan will run with (0 = 8)       */
+  int32_t group_size;        /* scheduling hint: n_q_heads / n_kv_heads (0 = 8).  A chunk's row set is split so
+                                that rows * group_size <= 64; mv_dag_decode_attn returns MV_ERR_UNSUPPORTED if
+                                the geometry's real group size breaks that bound                               */
 } mv_dag_batch;
 
 typedef struct {
@@ -121,6 +125,8 @@ typedef struct {
   int64_t tile_pairs;          /* prefill: (query, key) pairs inside the KV ranges the kernel walks,
                                   rounded up to whole 128x64 tiles                                         */
   int64_t max_page_id;         /* largest page id referenced                                                */
+  int64_t max_item_rows;       /* decode: largest row set of a work item                                    */
+  int64_t sched_kv_heads, sched_group; /* the scheduling hints in effect                                    */
 } mv_plan_stats;
 
 enum { MV_OP_ROPE_WRITE_KV = 0, MV_OP_DECODE_ATTN = 1, MV_OP_PREFILL_ATTN = 2 };

@@ -5,10 +5,15 @@
 // the set of rows (frontier tokens) that see that node.  The chunk is streamed from HBM exactly once and
 // serves every sibling row and the whole GQA group: the q-vectors (rows x group) are the M dimension of
 // bf16 tensor-core tiles (m16n8k16, fp32 accumulate), so that the arithmetic (16-64 flop per KV byte)
-// does not throttle the HBM stream.  Each CTA keeps a multi-stage cp.async pipeline of 64-token stages
-// (16-byte coalesced copies of whole 4 KB page blocks, XOR-swizzled in shared memory for conflict-free
-// ldmatrix) and an online softmax; partial (max, sum, output) triples go to the split-KV workspace and a
-// second kernel merges the partials of every (row, head).
+// does not throttle the HBM stream.
+//
+// Persistent CTAs (two per SM) pull units from an atomic work counter, longest first, and keep ONE
+// cp.async pipeline of 64-token stages running across unit boundaries: the loads for the next unit are
+// already in flight while the current unit is finished, so the HBM stream never drains.  Every thread
+// copies 16-byte pieces of a single 4 KB page block per stage (coalesced), into XOR-swizzled shared memory
+// (conflict-free ldmatrix).  Softmax is online, in log2 units; each unit leaves one partial (max, sum,
+// unnormalised output) per q-vector in the split-KV workspace and a second kernel merges the partials
+// of every (row, head).
 #include "common.cuh"
 
 namespace {
@@ -17,7 +22,6 @@ using bf16 = __nv_bfloat16;
 constexpr int NTHREADS = 128;  // 4 warps
 constexpr int ST = 64;         // tokens per pipeline stage (4 pages)
 constexpr int NSTAGES = 3;
-constexpr int MAX_CHUNK_PAGES = 256;
 
 struct DecodeArgs {
   const bf16* q;
@@ -28,92 +32,198 @@ struct DecodeArgs {
   const mv::ItemRow* item_rows;
   float* part_o;   // [n_partials][Hq][D]
   float* part_ml;  // [n_partials][Hq][2]  (max in log2 units, sum)
-  int Hq, Hkv, G;
+  int32_t* sched;  // [0] next unit, [1] CTAs finished; both zero between launches
+  int Hq, Hkv, G, n_units;
   float scale_log2;  // softmax scale * log2(e)
 };
 
+struct Unit {  // uniform across the CTA
+  int page_begin, n_tokens, row_begin, n_rows, kvh, n_stages;
+};
+
 template <int D>
-__device__ __forceinline__ uint32_t swz(int row, int chunk) {  // byte offset of 16-byte chunk `chunk` of row `row`
+struct Cfg {
+  static constexpr int CPR = D / 8;                 // 16-byte chunks per token row
+  static constexpr int KV_BYTES = ST * D * 2;       // K (or V) bytes of a stage
+  static constexpr int STAGE_BYTES = 2 * KV_BYTES;  // K then V
+  static constexpr int NCP = CPR / 2;               // cp.async per thread per stage for K (same for V)
+  static constexpr int SMEM = NSTAGES * STAGE_BYTES;
+};
+
+template <int D>
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {  // byte offset of 16-byte chunk `chunk` of token row `row`
   return uint32_t(row) * (D * 2) + (uint32_t(chunk ^ (row & 7)) << 4);
 }
 
+__device__ __forceinline__ Unit load_unit(const DecodeArgs& a, int u) {
+  Unit x;
+  if (u < a.n_units) {
+    const int4 it = *reinterpret_cast<const int4*>(a.items + u / a.Hkv);
+    x.page_begin = it.x; x.n_tokens = it.y; x.row_begin = it.z; x.n_rows = it.w;
+    x.kvh = u % a.Hkv;
+    x.n_stages = (it.y + ST - 1) / ST;
+  } else {
+    x.page_begin = 0; x.n_tokens = 0; x.row_begin = 0; x.n_rows = 0; x.kvh = 0; x.n_stages = 0;
+  }
+  return x;
+}
+
+// The producer side of the pipeline: walks the stages of the current unit, then of the next one.
 template <int D>
-struct Smem {
-  static constexpr int STAGE_BYTES = ST * D * 2;  // one of K or V
-  static constexpr int Q_BYTES = 64 * D * 2;
-  static constexpr int TOTAL = NSTAGES * 2 * STAGE_BYTES + Q_BYTES + MAX_CHUNK_PAGES * 4;
+struct Loader {
+  int which = 0;   // 0: current unit, 1: next unit, 2: beyond (nothing to issue)
+  int stage = 0;   // next stage of that unit to issue
+  int issued = 0;  // stages issued so far (buffer = issued % NSTAGES)
+  int page = 0;    // prefetched page id of this thread's page slot for the stage about to be issued
+  uint32_t dst[Cfg<D>::NCP];  // swizzled shared-memory offsets of this thread's pieces (stage relative)
+  int row0;                   // first token row (inside the page) this thread copies
+  int pslot, j;
+
+  __device__ __forceinline__ void init(int tid) {
+    pslot = tid >> 5;
+    j = tid & 31;
+    row0 = j / Cfg<D>::CPR;
+#pragma unroll
+    for (int k = 0; k < Cfg<D>::NCP; ++k) {
+      const int idx = j + 32 * k;
+      dst[k] = swz<D>(pslot * 16 + idx / Cfg<D>::CPR, idx % Cfg<D>::CPR);
+    }
+  }
+  __device__ __forceinline__ void prefetch_page(const DecodeArgs& a, const Unit& cu, const Unit& nu) {
+    const Unit& u = which == 0 ? cu : nu;
+    const bool ok = which <= 1 && stage < u.n_stages && (stage * ST + pslot * 16) < u.n_tokens;
+    page = ok ? __ldg(a.page_idx + u.page_begin + stage * 4 + pslot) : -1;
+  }
+  // Issues the copies of the next stage as one cp.async group; returns false (and commits nothing) when every
+  // stage of the current and the next unit has been issued already.
+  __device__ __forceinline__ bool issue(const DecodeArgs& a, const Unit& cu, const Unit& nu, uint32_t smem_base) {
+    const Unit& u = which == 0 ? cu : nu;
+    if (!(which <= 1 && stage < u.n_stages)) return false;
+    {
+      const uint32_t kd = smem_base + (issued % NSTAGES) * Cfg<D>::STAGE_BYTES;
+      const uint32_t vd = kd + Cfg<D>::KV_BYTES;
+      const int n_valid = u.n_tokens - (stage * ST + pslot * 16);  // valid token rows of this thread's page
+      const int64_t blk = page >= 0 ? ((int64_t(page) * a.Hkv + u.kvh) << 4) * D + j * 8 : 0;
+      const bf16* ks = a.k_pages + blk;
+      const bf16* vs = a.v_pages + blk;
+      constexpr int ROW_STEP = 32 / Cfg<D>::CPR;  // token rows between successive pieces of a thread
+      if (n_valid >= 16) {
+#pragma unroll
+        for (int k = 0; k < Cfg<D>::NCP; ++k) {
+          mv::cp_async_16(kd + dst[k], ks + k * 256, 16);
+          mv::cp_async_16(vd + dst[k], vs + k * 256, 16);
+        }
+      } else {
+#pragma unroll
+        for (int k = 0; k < Cfg<D>::NCP; ++k) {
+          const bool ok = (row0 + k * ROW_STEP) < n_valid;  // beyond the node's last token: zero-fill
+          mv::cp_async_16(kd + dst[k], ok ? ks + k * 256 : a.k_pages, ok ? 16 : 0);
+          mv::cp_async_16(vd + dst[k], ok ? vs + k * 256 : a.v_pages, ok ? 16 : 0);
+        }
+      }
+      ++stage;
+      if (stage == u.n_stages) {
+        ++which;
+        stage = 0;
+      }
+      prefetch_page(a, cu, nu);
+    }
+    mv::cp_async_commit();
+    ++issued;
+    return true;
+  }
+  // Brings the pipeline back to NSTAGES-1 stages in flight (as far as stages exist).
+  __device__ __forceinline__ void top_up(const DecodeArgs& a, const Unit& cu, const Unit& nu, uint32_t smem_base, int consumed) {
+    while (issued - consumed < NSTAGES - 1 && issue(a, cu, nu, smem_base)) {
+    }
+  }
 };
 
-// One pass: up to MT*16 q-vectors against the whole chunk.  Warp w: m-tile (w % MT), kv split (w / MT).
+// Waits until the group of the stage about to be consumed has landed: `lead` = issued - consumed groups are
+// outstanding at most, of which all but the oldest may stay pending.
+__device__ __forceinline__ void wait_stage(int lead) {
+  static_assert(NSTAGES == 3, "wait_stage enumerates the pending counts of a 3-stage pipeline");
+  if (lead >= 2) mv::cp_async_wait<1>();
+  else mv::cp_async_wait<0>();
+}
+
+// merge (m, l, o) of another kv-split into mine; both in this thread's fragment layout
+template <int DT>
+__device__ __forceinline__ void merge_frag(float& m0, float& m1, float& l0, float& l1, float (&o)[DT][4], const float4 oml,
+                                           const float4* other_o, int lane) {
+  const float n0 = fmaxf(m0, oml.x), n1 = fmaxf(m1, oml.y);
+  const float ws0 = (m0 == -INFINITY) ? 0.f : mv::fast_exp2(m0 - n0), wo0 = (oml.x == -INFINITY) ? 0.f : mv::fast_exp2(oml.x - n0);
+  const float ws1 = (m1 == -INFINITY) ? 0.f : mv::fast_exp2(m1 - n1), wo1 = (oml.y == -INFINITY) ? 0.f : mv::fast_exp2(oml.y - n1);
+  m0 = n0; m1 = n1;
+  l0 = l0 * ws0 + oml.z * wo0;
+  l1 = l1 * ws1 + oml.w * wo1;
+#pragma unroll
+  for (int i = 0; i < DT; ++i) {
+    const float4 t = other_o[i * 32 + lane];
+    o[i][0] = o[i][0] * ws0 + t.x * wo0;
+    o[i][1] = o[i][1] * ws0 + t.y * wo0;
+    o[i][2] = o[i][2] * ws1 + t.z * wo1;
+    o[i][3] = o[i][3] * ws1 + t.w * wo1;
+  }
+}
+
+// Consumes all stages of unit `cu` with MT m-tiles of 16 q-vectors; warp w: m-tile (w % MT), kv split (w / MT).
 template <int D, int MT>
-__device__ __forceinline__ void decode_pass(const DecodeArgs& a, const mv::WorkItem& it, int kvh, int qv0, int nqv,
-                                            unsigned char* smem) {
+__device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu, const Unit& nu, Loader<D>& ld,
+                                             int& consumed, unsigned char* smem, uint32_t smem_base, int32_t pending,
+                                             int32_t* s_next) {
   constexpr int KS = 4 / MT;      // kv splits inside a stage
   constexpr int WT = ST / KS;     // tokens per warp per stage
   constexpr int NT = WT / 8;      // S n-tiles per warp
   constexpr int KSTEPS = D / 16;  // k-steps of QK^T
   constexpr int DT = D / 8;       // O n-tiles
-  constexpr int CPR = D / 8;      // 16-byte chunks per row
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int mt = warp % MT, ks = warp / MT;
-  unsigned char* k_s = smem;
-  unsigned char* v_s = smem + NSTAGES * Smem<D>::STAGE_BYTES;
-  unsigned char* q_s = smem + 2 * NSTAGES * Smem<D>::STAGE_BYTES;
-  const int32_t* pages = reinterpret_cast<const int32_t*>(q_s + Smem<D>::Q_BYTES);
-  const uint32_t k_u = mv::smem_u32(k_s), v_u = mv::smem_u32(v_s), q_u = mv::smem_u32(q_s);
+  const int nqv = cu.n_rows * a.G;
 
-  // ---- stage the pass's q-vectors (zero rows beyond nqv); q-vector x = (row x / G, head kvh*G + x % G)
-  for (int i = tid; i < MT * 16 * CPR; i += NTHREADS) {
-    const int x = i / CPR, c = i % CPR;
-    uint4 val = make_uint4(0, 0, 0, 0);
-    if (x < nqv) {
-      const int xr = (qv0 + x) / a.G, xg = (qv0 + x) % a.G;
-      const int row = a.item_rows[it.row_begin + xr].row;
-      val = *reinterpret_cast<const uint4*>(a.q + (int64_t(row) * a.Hq + kvh * a.G + xg) * D + c * 8);
-    }
-    *reinterpret_cast<uint4*>(q_s + swz<D>(x, c)) = val;
-  }
-
-  const int n_stages = (it.n_tokens + ST - 1) / ST;
-  auto load_stage = [&](int s) {
-    if (s < n_stages) {
-      const int buf = s % NSTAGES;
-      const uint32_t kd = k_u + buf * Smem<D>::STAGE_BYTES, vd = v_u + buf * Smem<D>::STAGE_BYTES;
-#pragma unroll
-      for (int i = tid; i < ST * CPR; i += NTHREADS) {
-        const int r = i / CPR, c = i % CPR;
-        const int tok = s * ST + r;
-        const bool ok = tok < it.n_tokens;
-        const int64_t page = ok ? pages[tok >> 4] : 0;
-        const int64_t off = (((page * a.Hkv + kvh) << 4) + (tok & 15)) * D + c * 8;
-        mv::cp_async_16(kd + swz<D>(r, c), a.k_pages + (ok ? off : 0), ok ? 16 : 0);
-        mv::cp_async_16(vd + swz<D>(r, c), a.v_pages + (ok ? off : 0), ok ? 16 : 0);
-      }
-    }
-    mv::cp_async_commit();
-  };
-#pragma unroll
-  for (int s = 0; s < NSTAGES - 1; ++s) load_stage(s);
-  __syncthreads();  // q_s (and the page list) visible
-
+  // ---- this thread's two q rows, straight from global memory into the A-fragment layout
   uint32_t qf[KSTEPS][4];
+  int part0 = -1, part1 = -1;  // partial slot (x Hq + head) of the two rows, -1 = padding row
+  {
+    const int x0 = mt * 16 + (lane >> 2), x1 = x0 + 8;
+    const uint32_t* p0 = nullptr;
+    const uint32_t* p1 = nullptr;
+    if (x0 < nqv) {
+      const mv::ItemRow ir = a.item_rows[cu.row_begin + x0 / a.G];
+      const int head = cu.kvh * a.G + x0 % a.G;
+      p0 = reinterpret_cast<const uint32_t*>(a.q + (int64_t(ir.row) * a.Hq + head) * D) + (lane & 3);
+      part0 = ir.part * a.Hq + head;
+    }
+    if (x1 < nqv) {
+      const mv::ItemRow ir = a.item_rows[cu.row_begin + x1 / a.G];
+      const int head = cu.kvh * a.G + x1 % a.G;
+      p1 = reinterpret_cast<const uint32_t*>(a.q + (int64_t(ir.row) * a.Hq + head) * D) + (lane & 3);
+      part1 = ir.part * a.Hq + head;
+    }
 #pragma unroll
-  for (int kk = 0; kk < KSTEPS; ++kk)
-    mv::ldmatrix_x4(qf[kk], q_u + swz<D>(mt * 16 + (lane & 15), kk * 2 + (lane >> 4)));
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+      qf[kk][0] = p0 ? __ldg(p0 + kk * 8) : 0u;
+      qf[kk][1] = p1 ? __ldg(p1 + kk * 8) : 0u;
+      qf[kk][2] = p0 ? __ldg(p0 + kk * 8 + 4) : 0u;
+      qf[kk][3] = p1 ? __ldg(p1 + kk * 8 + 4) : 0u;
+    }
+  }
 
   float oacc[DT][4];
 #pragma unroll
   for (int i = 0; i < DT; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // rows lane/4 and lane/4 + 8 of the m-tile
+  const int tok_w = ks * WT;                                  // first token of this warp inside a stage
 
-  for (int s = 0; s < n_stages; ++s) {
-    mv::cp_async_wait<NSTAGES - 2>();
+  for (int s = 0; s < cu.n_stages; ++s) {
+    wait_stage(ld.issued - consumed);
     __syncthreads();
-    load_stage(s + NSTAGES - 1);
-    const int buf = s % NSTAGES;
-    const uint32_t kb = k_u + buf * Smem<D>::STAGE_BYTES, vb = v_u + buf * Smem<D>::STAGE_BYTES;
-    const int tok_w = ks * WT;  // first token of this warp inside the stage
-    if (s * ST + tok_w >= it.n_tokens) continue;  // warp-uniform: nothing valid for this warp
+    ld.issue(a, cu, nu, smem_base);  // refills the buffer consumed one iteration ago
+    if (s == 0 && tid == 0) *s_next = pending;  // unit after `nu`; read by everyone after this unit's epilogue
+    const uint32_t kb = smem_base + (consumed % NSTAGES) * Cfg<D>::STAGE_BYTES, vb = kb + Cfg<D>::KV_BYTES;
+    ++consumed;
+    const int tok_lim = cu.n_tokens - (s * ST + tok_w);  // valid tokens of this warp's slice
+    if (tok_lim <= 0) continue;                          // warp-uniform
 
     float sacc[NT][4];
 #pragma unroll
@@ -130,17 +240,25 @@ __device__ __forceinline__ void decode_pass(const DecodeArgs& a, const mv::WorkI
       }
     }
     // scale to log2 units, mask the ragged tail, online softmax
-    const int tok_lim = it.n_tokens - (s * ST + tok_w);  // tokens of this warp slice that are valid
     float mx0 = -INFINITY, mx1 = -INFINITY;
+    if (tok_lim >= WT) {
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
+      for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
-        const float sv = (col < tok_lim) ? sacc[nt][e] * a.scale_log2 : -INFINITY;
-        sacc[nt][e] = sv;
-        if (e < 2) mx0 = fmaxf(mx0, sv);
-        else mx1 = fmaxf(mx1, sv);
+        for (int e = 0; e < 4; ++e) sacc[nt][e] *= a.scale_log2;
+        mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
+        mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
+      }
+    } else {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
+          sacc[nt][e] = (col < tok_lim) ? sacc[nt][e] * a.scale_log2 : -INFINITY;
+        }
+        mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
+        mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
       }
     }
     mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
@@ -148,25 +266,27 @@ __device__ __forceinline__ void decode_pass(const DecodeArgs& a, const mv::WorkI
     mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
     mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
     const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);  // finite: column 0 of the slice is valid
-    const float al0 = mv::fast_exp2(m0 - mn0), al1 = mv::fast_exp2(m1 - mn1);
-    m0 = mn0;
-    m1 = mn1;
-    float ps0 = 0.f, ps1 = 0.f;
+    const bool grow = (mn0 > m0) || (mn1 > m1);
+    if (__any_sync(0xffffffffu, grow)) {  // rescale only when some row's maximum moved
+      const float al0 = mv::fast_exp2(m0 - mn0), al1 = mv::fast_exp2(m1 - mn1);
+      l0 *= al0;
+      l1 *= al1;
+#pragma unroll
+      for (int i = 0; i < DT; ++i) {
+        oacc[i][0] *= al0; oacc[i][1] *= al0;
+        oacc[i][2] *= al1; oacc[i][3] *= al1;
+      }
+      m0 = mn0;
+      m1 = mn1;
+    }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      sacc[nt][0] = mv::fast_exp2(sacc[nt][0] - mn0);
-      sacc[nt][1] = mv::fast_exp2(sacc[nt][1] - mn0);
-      sacc[nt][2] = mv::fast_exp2(sacc[nt][2] - mn1);
-      sacc[nt][3] = mv::fast_exp2(sacc[nt][3] - mn1);
-      ps0 += sacc[nt][0] + sacc[nt][1];
-      ps1 += sacc[nt][2] + sacc[nt][3];
-    }
-    l0 = l0 * al0 + ps0;  // per-thread partial sums; reduced over the quad at the end
-    l1 = l1 * al1 + ps1;
-#pragma unroll
-    for (int i = 0; i < DT; ++i) {
-      oacc[i][0] *= al0; oacc[i][1] *= al0;
-      oacc[i][2] *= al1; oacc[i][3] *= al1;
+      sacc[nt][0] = mv::fast_exp2(sacc[nt][0] - m0);
+      sacc[nt][1] = mv::fast_exp2(sacc[nt][1] - m0);
+      sacc[nt][2] = mv::fast_exp2(sacc[nt][2] - m1);
+      sacc[nt][3] = mv::fast_exp2(sacc[nt][3] - m1);
+      l0 += sacc[nt][0] + sacc[nt][1];  // per-thread partial sums; reduced over the quad at the end
+      l1 += sacc[nt][2] + sacc[nt][3];
     }
     // O += P V
 #pragma unroll
@@ -186,78 +306,105 @@ __device__ __forceinline__ void decode_pass(const DecodeArgs& a, const mv::WorkI
       }
     }
   }
-  mv::cp_async_wait<0>();
-  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-  __syncthreads();  // every warp is done with the stage buffers: reuse them for the cross-warp combine
 
-  float* red_o = reinterpret_cast<float*>(smem);                 // [4 warps][16][D]
-  float* red_ml = red_o + 4 * 16 * D;                             // [4 warps][16][2]
-  {
-    const int r0 = lane >> 2, c0 = (lane & 3) * 2;
-    float* wo = red_o + warp * 16 * D;
+  // ---- epilogue: combine the KS kv-splits through the stage buffer that was consumed last (it is refilled
+  // only after the next top-of-loop barrier), then write one partial per q-vector
+  if (KS > 1) {
+    float4* sc_o = reinterpret_cast<float4*>(smem + ((consumed - 1) % NSTAGES) * Cfg<D>::STAGE_BYTES);  // [2][DT][32]
+    float4* sc_ml = sc_o + 2 * DT * 32;                                                               // [2][32]
+    __syncthreads();  // everyone has finished reading the last stage
+    if (KS == 4) {
+      if (warp >= 2) {
+        float4* so = sc_o + (warp - 2) * DT * 32;
 #pragma unroll
-    for (int i = 0; i < DT; ++i) {
-      *reinterpret_cast<float2*>(wo + r0 * D + i * 8 + c0) = make_float2(oacc[i][0], oacc[i][1]);
-      *reinterpret_cast<float2*>(wo + (r0 + 8) * D + i * 8 + c0) = make_float2(oacc[i][2], oacc[i][3]);
-    }
-    if ((lane & 3) == 0) {
-      red_ml[(warp * 16 + r0) * 2] = m0;
-      red_ml[(warp * 16 + r0) * 2 + 1] = l0;
-      red_ml[(warp * 16 + r0 + 8) * 2] = m1;
-      red_ml[(warp * 16 + r0 + 8) * 2 + 1] = l1;
+        for (int i = 0; i < DT; ++i) so[i * 32 + lane] = make_float4(oacc[i][0], oacc[i][1], oacc[i][2], oacc[i][3]);
+        sc_ml[(warp - 2) * 32 + lane] = make_float4(m0, m1, l0, l1);
+      }
+      __syncthreads();
+      if (warp < 2) merge_frag<DT>(m0, m1, l0, l1, oacc, sc_ml[warp * 32 + lane], sc_o + warp * DT * 32, lane);
+      __syncthreads();
+      if (warp == 1) {
+#pragma unroll
+        for (int i = 0; i < DT; ++i) sc_o[i * 32 + lane] = make_float4(oacc[i][0], oacc[i][1], oacc[i][2], oacc[i][3]);
+        sc_ml[lane] = make_float4(m0, m1, l0, l1);
+      }
+      __syncthreads();
+      if (warp == 0) merge_frag<DT>(m0, m1, l0, l1, oacc, sc_ml[lane], sc_o, lane);
+    } else {  // KS == 2: warps 2,3 hand their state to warps 0,1 (same m-tile)
+      if (ks == 1) {
+        float4* so = sc_o + mt * DT * 32;
+#pragma unroll
+        for (int i = 0; i < DT; ++i) so[i * 32 + lane] = make_float4(oacc[i][0], oacc[i][1], oacc[i][2], oacc[i][3]);
+        sc_ml[mt * 32 + lane] = make_float4(m0, m1, l0, l1);
+      }
+      __syncthreads();
+      if (ks == 0) merge_frag<DT>(m0, m1, l0, l1, oacc, sc_ml[mt * 32 + lane], sc_o + mt * DT * 32, lane);
     }
   }
-  __syncthreads();
-  // combine the KS kv-splits of every q-vector and write the partial (unnormalised o, max, sum)
-  for (int x = 0; x < nqv; ++x) {
-    const int xm = x / 16, xr = x % 16;
-    float mt_ = -INFINITY;
+  if (ks == 0) {
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    const int c0 = (lane & 3) * 2;
+    if (part0 >= 0) {
+      float* po = a.part_o + int64_t(part0) * D + c0;
 #pragma unroll
-    for (int k2 = 0; k2 < KS; ++k2) mt_ = fmaxf(mt_, red_ml[((xm + MT * k2) * 16 + xr) * 2]);
-    float lsum = 0.f;
-    float w[KS];
-#pragma unroll
-    for (int k2 = 0; k2 < KS; ++k2) {
-      const float mk = red_ml[((xm + MT * k2) * 16 + xr) * 2];
-      w[k2] = (mk == -INFINITY) ? 0.f : mv::fast_exp2(mk - mt_);
-      lsum += w[k2] * red_ml[((xm + MT * k2) * 16 + xr) * 2 + 1];
+      for (int i = 0; i < DT; ++i) *reinterpret_cast<float2*>(po + i * 8) = make_float2(oacc[i][0], oacc[i][1]);
+      if ((lane & 3) == 0) *reinterpret_cast<float2*>(a.part_ml + int64_t(part0) * 2) = make_float2(m0, l0);
     }
-    const int xrow = (qv0 + x) / a.G, xg = (qv0 + x) % a.G;
-    const mv::ItemRow ir = a.item_rows[it.row_begin + xrow];
-    const int64_t pslot = int64_t(ir.part) * a.Hq + kvh * a.G + xg;
-    for (int c = tid; c < D; c += NTHREADS) {
-      float acc = 0.f;
+    if (part1 >= 0) {
+      float* po = a.part_o + int64_t(part1) * D + c0;
 #pragma unroll
-      for (int k2 = 0; k2 < KS; ++k2) acc += w[k2] * red_o[((xm + MT * k2) * 16 + xr) * D + c];
-      a.part_o[pslot * D + c] = acc;
-    }
-    if (tid == 0) {
-      a.part_ml[pslot * 2] = mt_;
-      a.part_ml[pslot * 2 + 1] = lsum;
+      for (int i = 0; i < DT; ++i) *reinterpret_cast<float2*>(po + i * 8) = make_float2(oacc[i][2], oacc[i][3]);
+      if ((lane & 3) == 0) *reinterpret_cast<float2*>(a.part_ml + int64_t(part1) * 2) = make_float2(m1, l1);
     }
   }
-  __syncthreads();  // the combine buffers alias the stage buffers of the next pass
 }
 
 template <int D>
-__global__ void __launch_bounds__(NTHREADS) decode_attn_kernel(const DecodeArgs a) {
+__global__ void __launch_bounds__(NTHREADS, 2) decode_attn_kernel(const DecodeArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
-  const int unit = blockIdx.x;
-  const mv::WorkItem it = a.items[unit / a.Hkv];
-  const int kvh = unit % a.Hkv;
-  int32_t* pages = reinterpret_cast<int32_t*>(smem + 2 * NSTAGES * Smem<D>::STAGE_BYTES + Smem<D>::Q_BYTES);
-  const int n_pages = (it.n_tokens + 15) >> 4;
-  for (int i = threadIdx.x; i < n_pages; i += NTHREADS) pages[i] = a.page_idx[it.page_begin + i];
+  __shared__ int32_t s_ids[3];
+  const int tid = threadIdx.x;
+  const uint32_t smem_base = mv::smem_u32(smem);
+  if (tid == 0) {
+    s_ids[0] = atomicAdd(a.sched, 1);
+    s_ids[1] = atomicAdd(a.sched, 1);
+  }
   __syncthreads();
-  const int nq_total = it.n_rows * a.G;
-  for (int qv0 = 0; qv0 < nq_total; qv0 += 64) {
-    const int nqv = min(64, nq_total - qv0);
-    if (nqv <= 16) decode_pass<D, 1>(a, it, kvh, qv0, nqv, smem);
-    else if (nqv <= 32) decode_pass<D, 2>(a, it, kvh, qv0, nqv, smem);
-    else decode_pass<D, 4>(a, it, kvh, qv0, nqv, smem);
+  Unit cu = load_unit(a, s_ids[0]);
+  Unit nu = load_unit(a, s_ids[1]);
+  Loader<D> ld;
+  ld.init(tid);
+  ld.prefetch_page(a, cu, nu);
+  int consumed = 0;
+  ld.top_up(a, cu, nu, smem_base, consumed);
+  while (cu.n_stages > 0) {
+    int32_t pending = 0;
+    if (tid == 0) pending = atomicAdd(a.sched, 1);  // the unit after `nu`; consumed one barrier later
+    const int nqv = cu.n_rows * a.G;
+    if (nqv <= 16) process_unit<D, 1>(a, cu, nu, ld, consumed, smem, smem_base, pending, &s_ids[2]);
+    else if (nqv <= 32) process_unit<D, 2>(a, cu, nu, ld, consumed, smem, smem_base, pending, &s_ids[2]);
+    else process_unit<D, 4>(a, cu, nu, ld, consumed, smem, smem_base, pending, &s_ids[2]);
+    __syncthreads();  // s_ids[2] is visible; the epilogue's scratch reads are done
+    cu = nu;
+    nu = load_unit(a, s_ids[2]);
+    // the loader had finished `cu` (it was consumed), so it stands in the old `nu` or beyond it
+    ld.which -= 1;
+    if (ld.which == 1) ld.prefetch_page(a, cu, nu);  // it was beyond: it now stands at the first stage of the new `nu`
+    ld.top_up(a, cu, nu, smem_base, consumed);
+  }
+  mv::cp_async_wait<0>();
+  // the last CTA to finish re-arms the scheduler words for the next launch
+  if (tid == 0) {
+    __threadfence();
+    const int done = atomicAdd(a.sched + 1, 1);
+    if (done == int(gridDim.x) - 1) {
+      a.sched[0] = 0;
+      a.sched[1] = 0;
+      __threadfence();
+    }
   }
 }
 
@@ -281,12 +428,17 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const float* __restri
   float l = 0.f;
   for (int p = p0; p < p1; ++p) {
     const int64_t ps = int64_t(p) * Hq + h;
-    const float mp = part_ml[ps * 2];
-    const float wgt = (mp == -INFINITY) ? 0.f : exp2f(mp - m);
-    l += wgt * part_ml[ps * 2 + 1];
+    const float2 ml = *reinterpret_cast<const float2*>(part_ml + ps * 2);
+    const float wgt = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m);
+    l += wgt * ml.y;
     const float* po = part_o + ps * D + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] += wgt * po[e];
+    if (E == 4) {
+      const float4 t = *reinterpret_cast<const float4*>(po);
+      acc[0] += wgt * t.x; acc[1] += wgt * t.y; acc[2] += wgt * t.z; acc[3 % E] += wgt * t.w;
+    } else {
+      const float2 t = *reinterpret_cast<const float2*>(po);
+      acc[0] += wgt * t.x; acc[1] += wgt * t.y;
+    }
   }
   const float inv = 1.f / l;
   bf16* o = out + (int64_t(row) * Hq + h) * D + lane * E;
@@ -294,12 +446,24 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const float* __restri
   for (int e = 0; e < E; e += 2) *reinterpret_cast<__nv_bfloat162*>(o + e) = __floats2bfloat162_rn(acc[e] * inv, acc[e + 1] * inv);
 }
 
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      (void)cudaGetLastError();
+      n = 148;
+    }
+  }
+  return n;
+}
+
 template <int D>
 mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* kp, const void* vp, void* out,
                  void* ws, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(decode_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::TOTAL) != cudaSuccess) {
+    if (cudaFuncSetAttribute(decode_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::SMEM) != cudaSuccess) {
       (void)cudaGetLastError();
       return MV_ERR_CUDA;
     }
@@ -316,12 +480,14 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
   a.item_rows = mv::table<mv::ItemRow>(P, P->layout.item_rows);
   a.part_o = static_cast<float*>(ws);
   a.part_ml = reinterpret_cast<float*>(static_cast<char*>(ws) + o_bytes);
+  a.sched = const_cast<int32_t*>(mv::table<int32_t>(P, P->layout.sched));
   a.Hq = g->n_q_heads;
   a.Hkv = g->n_kv_heads;
   a.G = g->n_q_heads / g->n_kv_heads;
+  a.n_units = int(P->stats.n_items) * g->n_kv_heads;
   a.scale_log2 = mv::softmax_scale(g) * 1.4426950408889634f;
-  const int n_units = int(P->stats.n_items) * g->n_kv_heads;
-  decode_attn_kernel<D><<<n_units, NTHREADS, Smem<D>::TOTAL, st>>>(a);
+  const int grid = std::min(a.n_units, 2 * sm_count());
+  decode_attn_kernel<D><<<grid, NTHREADS, Cfg<D>::SMEM, st>>>(a);
   mv::g_launches++;
   if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
   const int n_rows = int(P->stats.n_new_tokens);
@@ -340,8 +506,9 @@ extern "C" mv_status mv_dag_decode_attn(const mv_plan* P, const mv_attn_geom* g,
   if (!P || !P->valid) return MV_ERR_INVALID_ARG;
   mv_status st = mv::check_geom(g);
   if (st != MV_OK) return st;
+  if (P->stats.n_new_tokens == 0) return MV_OK;
   if (g->dtype != MV_BF16 || !P->stats.decode_ready) return MV_ERR_UNSUPPORTED;
-  if (P->stats.chunk_tokens > MAX_CHUNK_PAGES * 16) return MV_ERR_UNSUPPORTED;
+  if (P->stats.max_item_rows * (g->n_q_heads / g->n_kv_heads) > 64) return MV_ERR_UNSUPPORTED;
   if (!q_rot || !k_pages || !v_pages || !out) return MV_ERR_INVALID_ARG;
   if (!P->device_buf) return MV_ERR_WORKSPACE;
   if (P->stats.max_page_id >= g->num_pages) return MV_ERR_INVALID_ARG;

@@ -34,8 +34,8 @@ struct KvRange {
 };
 
 struct DeviceLayout {  // byte offsets into the device table buffer (all multiples of 256)
-  size_t pos_id = 0, slot = 0, page_idx = 0, items = 0, item_rows = 0, row_part_off = 0, q_tiles = 0,
-         kv_ranges = 0, total = 0;
+  size_t pos_id = 0, slot = 0, page_idx = 0, items = 0, item_rows = 0, row_part_off = 0, sched = 0,
+         q_tiles = 0, kv_ranges = 0, total = 0;
 };
 
 }  // namespace mv
@@ -49,6 +49,7 @@ struct mv_plan {
   std::vector<mv::WorkItem> items;
   std::vector<mv::ItemRow> item_rows;
   std::vector<int32_t> row_part_off;
+  int32_t sched_zero[64] = {};  // device-side scheduler words (work counter, finished-CTA counter), uploaded as zeros
   std::vector<mv::QTile> q_tiles;
   std::vector<mv::KvRange> kv_ranges;
   mv_plan_stats stats{};

@@ -51,6 +51,7 @@ extern "C" mv_status mv_plan_upload(mv_plan* P, void* device_buf, size_t device_
   put(h, L.items, P->items);
   put(h, L.item_rows, P->item_rows);
   put(h, L.row_part_off, P->row_part_off);
+  std::memcpy(h + L.sched, P->sched_zero, sizeof(P->sched_zero));
   put(h, L.q_tiles, P->q_tiles);
   put(h, L.kv_ranges, P->kv_ranges);
   // only the bytes in use travel (the tail of the last table)

@@ -42,6 +42,7 @@ mv_status check_batch(const mv_dag_batch* b) {
   if (b->vis_mode != MV_VIS_ANCESTORS && b->vis_mode != MV_VIS_LAYERWISE) return MV_ERR_INVALID_ARG;
   if (b->pos_mode != MV_POS_MAX_PARENT_END && b->pos_mode != MV_POS_FRONTIER_ALIGNED) return MV_ERR_INVALID_ARG;
   if (b->chunk_tokens < 0 || (b->chunk_tokens % b->page_size) != 0) return MV_ERR_INVALID_ARG;
+  if (b->n_kv_heads < 0 || b->group_size < 0) return MV_ERR_INVALID_ARG;
   if (b->node_off[0] != 0) return MV_ERR_INVALID_ARG;
   for (int r = 0; r < b->n_req; ++r)
     if (b->node_off[r + 1] < b->node_off[r]) return MV_ERR_INVALID_ARG;
@@ -120,10 +121,12 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   std::vector<int32_t> pos_end, layer_end;
   std::vector<int64_t> node_tok_start(n_nodes, 0);  // flattened index of a node's first NEW token
   std::vector<std::vector<int32_t>> rows_of_node;    // decode: rows that see each node (request local)
-  struct PendingItem { int32_t page_begin, n_tokens, row_begin, n_rows; };
   int64_t unique_tokens = 0, per_row_tokens = 0, visible_pairs = 0, tile_pairs = 0;
   std::vector<int32_t> row_parts;  // per row: number of partials
-  std::vector<std::vector<int32_t>> item_row_lists;  // parallel to P->items before sorting
+  std::vector<int32_t> flat_rows;  // (row, local partial index) pairs of every item, in item creation order
+  const int sched_kv_heads = b->n_kv_heads > 0 ? b->n_kv_heads : 8;
+  const int sched_group = b->group_size > 0 ? b->group_size : 8;
+  const int max_rows_per_item = std::max(1, 64 / sched_group);
 
   // automatic chunk length: aim for a few work items per CTA slot, assuming 8 KV heads
   int chunk = b->chunk_tokens;
@@ -137,7 +140,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       if (!has_new) continue;
       for (int g = lo; g < hi; ++g) total_unique += b->node_len[g] + b->node_new[g];
     }
-    int64_t c = (total_unique * 8) / (148 * 2 * 6);
+    int64_t c = (total_unique * sched_kv_heads) / (148 * 2 * 6);
     c = ((c + 63) / 64) * 64;
     chunk = int(std::min<int64_t>(1024, std::max<int64_t>(256, c)));
   }
@@ -249,19 +252,20 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
         for (int c = 0; c * pages_per_chunk < n_pages; ++c) {
           const int pb = c * pages_per_chunk;
           const int pe = std::min(n_pages, pb + pages_per_chunk);
-          WorkItem it;
-          it.page_begin = b->page_off[lo + u] + pb;
-          it.n_tokens = std::min(L, pe * ps) - pb * ps;
-          it.row_begin = 0;
-          it.n_rows = int32_t(rows.size());
-          P->items.push_back(it);
-          std::vector<int32_t> rl;
-          rl.reserve(rows.size() * 2);
-          for (int32_t row : rows) {
-            rl.push_back(row);
-            rl.push_back(row_parts[row]++);  // partial index local to the row, made global below
+          // a row set larger than one tensor-core pass (64 q-vectors) is split; each part re-reads the chunk
+          for (size_t r0 = 0; r0 < rows.size(); r0 += size_t(max_rows_per_item)) {
+            const size_t r1 = std::min(rows.size(), r0 + size_t(max_rows_per_item));
+            WorkItem it;
+            it.page_begin = b->page_off[lo + u] + pb;
+            it.n_tokens = std::min(L, pe * ps) - pb * ps;
+            it.row_begin = int32_t(flat_rows.size() / 2);
+            it.n_rows = int32_t(r1 - r0);
+            P->items.push_back(it);
+            for (size_t k = r0; k < r1; ++k) {
+              flat_rows.push_back(rows[k]);
+              flat_rows.push_back(row_parts[rows[k]]++);  // partial index local to the row, made global below
+            }
           }
-          item_row_lists.push_back(std::move(rl));
         }
       }
     }
@@ -333,10 +337,13 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     sorted.reserve(order.size());
     for (int32_t i : order) {
       WorkItem it = P->items[i];
+      const int32_t src = it.row_begin;
       it.row_begin = int32_t(P->item_rows.size());
-      const auto& rl = item_row_lists[i];
-      for (size_t k = 0; k < rl.size(); k += 2)
-        P->item_rows.push_back(ItemRow{rl[k], P->row_part_off[rl[k]] + rl[k + 1]});
+      for (int32_t k = 0; k < it.n_rows; ++k) {
+        const int32_t row = flat_rows[2 * size_t(src + k)], local = flat_rows[2 * size_t(src + k) + 1];
+        P->item_rows.push_back(ItemRow{row, P->row_part_off[row] + local});
+      }
+      S.max_item_rows = std::max<int64_t>(S.max_item_rows, it.n_rows);
       sorted.push_back(it);
     }
     P->items.swap(sorted);
@@ -365,6 +372,8 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   S.n_segs = int64_t(P->seg_node.size());
   S.decode_ready = decode_ready && new_tok_count > 0;
   S.prefill_ready = prefill_ready && new_tok_count > 0;
+  S.sched_kv_heads = sched_kv_heads;
+  S.sched_group = sched_group;
   S.unique_kv_tokens = unique_tokens;
   S.per_row_kv_tokens = per_row_tokens;
   P->stats = S;
@@ -379,6 +388,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   L.items = place(P->items.size() * sizeof(WorkItem));
   L.item_rows = place(P->item_rows.size() * sizeof(ItemRow));
   L.row_part_off = place(P->row_part_off.size() * sizeof(int32_t));
+  L.sched = place(sizeof(P->sched_zero));
   L.q_tiles = place(P->q_tiles.size() * sizeof(QTile));
   L.kv_ranges = place(P->kv_ranges.size() * sizeof(KvRange));
   L.total = std::max<size_t>(off, 256);

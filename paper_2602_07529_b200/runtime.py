@@ -23,8 +23,9 @@ def _dev_bytes(n: int, device):
 class PlanOnDevice:
     """A plan plus the caller-owned device buffer its kernel tables were uploaded to."""
 
-    def __init__(self, batch, device="cuda", chunk_tokens: int = 0, stream=None):
-        self.plan = B.Plan(batch, chunk_tokens)
+    def __init__(self, batch, device="cuda", chunk_tokens: int = 0, stream=None, geom: synth.Geometry | None = None):
+        hints = (geom.n_kv_heads, geom.group) if geom is not None else (0, 0)
+        self.plan = B.Plan(batch, chunk_tokens, *hints)
         self.tables = _dev_bytes(self.plan.device_bytes(), device)
         self.plan.upload(self.tables, stream)
 
@@ -81,13 +82,13 @@ class DecodeState:
         hist = synth.DagBatch(b.n_req, b.node_off, np.zeros_like(b.node_len), b.node_len, b.parent_off, b.parent_idx,
                               b.page_off, b.page_idx, b.page_size, b.num_pages, b.vis_mode, b.pos_mode)
         _, kh, vh = _stack_values(wl, "history", device)
-        hp = PlanOnDevice(hist, device)
+        hp = PlanOnDevice(hist, device, geom=g)
         for kp, vp in self.pools:
             B.mv_rope_write_kv(hp.plan, self.geom, None, kh, vh, None, None, kp, vp)
         torch.cuda.synchronize()
         del kh, vh, hp
         self.q, self.k, self.v = _stack_values(wl, "new", device)
-        self.pod = PlanOnDevice(b, device, chunk_tokens)
+        self.pod = PlanOnDevice(b, device, chunk_tokens, geom=g)
         self.plan = self.pod.plan
         self.q_rot = torch.empty_like(self.q)
         self.out = torch.empty_like(self.q)
@@ -108,7 +109,7 @@ class PrefillState:
         self.geom = B.geom_of(wl)
         dt = torch_dtype(g)
         self.q, self.k, self.v = _stack_values(wl, "all", device)
-        self.pod = PlanOnDevice(b, device)
+        self.pod = PlanOnDevice(b, device, geom=g)
         self.plan = self.pod.plan
         shape = (b.num_pages, g.n_kv_heads, g.page_size, g.head_dim)
         self.k_pages = torch.zeros(shape, dtype=dt, device=device)
