@@ -222,6 +222,12 @@ mv_status mv_decode_step_host(mv_plan* plan, const mv_attn_geom* geom, const voi
                               const void* v_host, void* out_host, void* k_pages, void* v_pages, void* staging,
                               size_t staging_bytes, void* cuda_stream);
 
+/* Reads the device-side status word of the kernels that last ran with this plan's uploaded tables: MV_OK, or
+ * MV_ERR_TIMEOUT if a bounded wait inside a kernel ran out (the kernel then still terminated, with an
+ * undefined result).  Copies 4 bytes device->host on `cuda_stream` and synchronises that stream.
+ *   status  host, out */
+mv_status mv_plan_read_status(const mv_plan* plan, void* cuda_stream, int32_t* status);
+
 const char* mv_status_string(mv_status s);
 
 /* Number of kernel launches the library has issued in this process since load (diagnostic counter). */

@@ -26,7 +26,7 @@ TABLES = {"layer": (0, np.int32), "pos_start": (1, np.int32), "pos_id": (2, np.i
 EXPORTS = ["mv_plan_dag", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_bytes", "mv_plan_upload",
            "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
            "mv_dag_prefill_attn", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_status_string",
-           "mv_launch_count"]
+           "mv_launch_count", "mv_plan_read_status"]
 
 
 class MvError(RuntimeError):
@@ -78,6 +78,7 @@ def _load():
     lib.mv_decode_step_host.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 7 + [sz, vp]
     lib.mv_status_string.argtypes = [C.c_int]
     lib.mv_status_string.restype = C.c_char_p
+    lib.mv_plan_read_status.argtypes = [vp, vp, C.POINTER(i32)]
     lib.mv_launch_count.argtypes = []
     lib.mv_launch_count.restype = i64
     for name in EXPORTS:
@@ -170,6 +171,12 @@ class Plan:
     def upload(self, device_buf, stream=None):
         _check(lib.mv_plan_upload(self._h, _ptr(device_buf), device_buf.numel() * device_buf.element_size(),
                                   _stream_ptr(stream)), "mv_plan_upload")
+
+    def read_status(self, stream=None) -> int:
+        """Device status word of the last kernels run with this plan (0 = fine); synchronises the stream."""
+        out = C.c_int32(-1)
+        _check(lib.mv_plan_read_status(self._h, _stream_ptr(stream), C.byref(out)), "mv_plan_read_status")
+        return int(out.value)
 
     def workspace_bytes(self, geom: _Geom, op: int) -> int:
         return int(lib.mv_workspace_bytes(self._h, C.byref(geom), op))

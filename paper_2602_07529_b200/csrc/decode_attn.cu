@@ -8,12 +8,16 @@
 // does not throttle the HBM stream.
 //
 // Persistent CTAs (two per SM) pull units from an atomic work counter, longest first, and keep ONE
-// cp.async pipeline of 64-token stages running across unit boundaries: the loads for the next unit are
-// already in flight while the current unit is finished, so the HBM stream never drains.  Every thread
-// copies 16-byte pieces of a single 4 KB page block per stage (coalesced), into XOR-swizzled shared memory
-// (conflict-free ldmatrix).  Softmax is online, in log2 units; each unit leaves one partial (max, sum,
-// unnormalised output) per q-vector in the split-KV workspace and a second kernel merges the partials
-// of every (row, head).
+// pipeline of 64-token stages running across unit boundaries.  A stage is filled by TMA: one elected
+// thread issues a [16 tokens][64 elements] box per half page block (cp.async.bulk.tensor, 128-byte
+// shared-memory swizzle, completion counted on an mbarrier), so no thread spends issue slots or
+// load-store-unit entries on the copy, and ldmatrix reads the tiles without bank conflicts.  Warps hand
+// a consumed stage back through a second mbarrier; there is no CTA-wide barrier inside a unit.  Softmax
+// is online, in log2 units; each unit leaves one partial (max, sum, unnormalised output) per q-vector in
+// the split-KV workspace and a second kernel merges the partials of every (row, head).
+//
+// Every wait on an mbarrier is bounded: if it runs out, the CTA records MV_ERR_TIMEOUT in the plan's
+// status word, stops waiting and still reaches every barrier, so the kernel always terminates.
 #include "common.cuh"
 
 namespace {
@@ -25,14 +29,12 @@ constexpr int NSTAGES = 3;
 
 struct DecodeArgs {
   const bf16* q;
-  const bf16* k_pages;
-  const bf16* v_pages;
   const int32_t* page_idx;
   const mv::WorkItem* items;
   const mv::ItemRow* item_rows;
   float* part_o;   // [n_partials][Hq][D]
   float* part_ml;  // [n_partials][Hq][2]  (max in log2 units, sum)
-  int32_t* sched;  // [0] next unit, [1] CTAs finished; both zero between launches
+  int32_t* sched;  // [0] next unit, [1] CTAs finished (both zero between launches), [2] status word
   int Hq, Hkv, G, n_units;
   float scale_log2;  // softmax scale * log2(e)
 };
@@ -44,15 +46,18 @@ struct Unit {  // uniform across the CTA
 template <int D>
 struct Cfg {
   static constexpr int CPR = D / 8;                 // 16-byte chunks per token row
+  static constexpr int HALVES = D / 64;             // 128-byte column blocks per row (one TMA box each)
+  static constexpr int HALF_BYTES = ST * 128;       // one column block of a stage: [64 tokens][128 B]
   static constexpr int KV_BYTES = ST * D * 2;       // K (or V) bytes of a stage
   static constexpr int STAGE_BYTES = 2 * KV_BYTES;  // K then V
-  static constexpr int NCP = CPR / 2;               // cp.async per thread per stage for K (same for V)
-  static constexpr int SMEM = NSTAGES * STAGE_BYTES;
+  static constexpr int SMEM = NSTAGES * STAGE_BYTES + 1024;  // + slack to align the base to 1024 B
 };
 
+// Byte offset of 16-byte chunk `chunk` of token row `row` inside a K (or V) stage tile as TMA lays it out:
+// column block h = chunk / 8 holds [64 tokens][128 B]; inside it the hardware XORs the chunk index with row % 8.
 template <int D>
-__device__ __forceinline__ uint32_t swz(int row, int chunk) {  // byte offset of 16-byte chunk `chunk` of token row `row`
-  return uint32_t(row) * (D * 2) + (uint32_t(chunk ^ (row & 7)) << 4);
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+  return uint32_t(chunk >> 3) * Cfg<D>::HALF_BYTES + uint32_t(row) * 128 + (uint32_t((chunk & 7) ^ (row & 7)) << 4);
 }
 
 __device__ __forceinline__ Unit load_unit(const DecodeArgs& a, int u) {
@@ -68,84 +73,73 @@ __device__ __forceinline__ Unit load_unit(const DecodeArgs& a, int u) {
   return x;
 }
 
-// The producer side of the pipeline: walks the stages of the current unit, then of the next one.
+struct Sync {  // shared-memory addresses of the pipeline barriers and flags
+  uint32_t full, empty;  // arrays of NSTAGES mbarriers (8 bytes each)
+  volatile int* abort;   // set once a bounded wait ran out
+  int32_t* status;       // global status word
+};
+
+__device__ __forceinline__ void wait_or_flag(const Sync& sy, uint32_t bar, uint32_t parity) {
+  if (*sy.abort) return;
+  if (!mv::mbar_wait_bounded(bar, parity)) {
+    *sy.abort = 1;
+    atomicExch(sy.status, int(MV_ERR_TIMEOUT));
+  }
+}
+
+// The producer side of the pipeline, run by thread 0: walks the stages of the current unit, then of the next.
 template <int D>
 struct Loader {
   int which = 0;   // 0: current unit, 1: next unit, 2: beyond (nothing to issue)
   int stage = 0;   // next stage of that unit to issue
   int issued = 0;  // stages issued so far (buffer = issued % NSTAGES)
-  int page = 0;    // prefetched page id of this thread's page slot for the stage about to be issued
-  uint32_t dst[Cfg<D>::NCP];  // swizzled shared-memory offsets of this thread's pieces (stage relative)
-  int row0;                   // first token row (inside the page) this thread copies
-  int pslot, j;
+  int pg[4] = {0, 0, 0, 0};  // prefetched page ids of the stage about to be issued
 
-  __device__ __forceinline__ void init(int tid) {
-    pslot = tid >> 5;
-    j = tid & 31;
-    row0 = j / Cfg<D>::CPR;
+  __device__ __forceinline__ void prefetch_pages(const DecodeArgs& a, const Unit& cu, const Unit& nu) {
+    const Unit& u = which == 0 ? cu : nu;
+    if (which <= 1 && stage < u.n_stages) {
+      const int n_pages = (u.n_tokens - stage * ST + 15) >> 4;
 #pragma unroll
-    for (int k = 0; k < Cfg<D>::NCP; ++k) {
-      const int idx = j + 32 * k;
-      dst[k] = swz<D>(pslot * 16 + idx / Cfg<D>::CPR, idx % Cfg<D>::CPR);
+      for (int p = 0; p < 4; ++p) pg[p] = p < n_pages ? __ldg(a.page_idx + u.page_begin + stage * 4 + p) : 0;
     }
   }
-  __device__ __forceinline__ void prefetch_page(const DecodeArgs& a, const Unit& cu, const Unit& nu) {
-    const Unit& u = which == 0 ? cu : nu;
-    const bool ok = which <= 1 && stage < u.n_stages && (stage * ST + pslot * 16) < u.n_tokens;
-    page = ok ? __ldg(a.page_idx + u.page_begin + stage * 4 + pslot) : -1;
-  }
-  // Issues the copies of the next stage as one cp.async group; returns false (and commits nothing) when every
-  // stage of the current and the next unit has been issued already.
-  __device__ __forceinline__ bool issue(const DecodeArgs& a, const Unit& cu, const Unit& nu, uint32_t smem_base) {
+  __device__ __forceinline__ bool issue(const DecodeArgs& a, const Unit& cu, const Unit& nu, uint32_t smem_base, const Sync& sy,
+                                        const CUtensorMap* tm_k, const CUtensorMap* tm_v) {
     const Unit& u = which == 0 ? cu : nu;
     if (!(which <= 1 && stage < u.n_stages)) return false;
-    {
-      const uint32_t kd = smem_base + (issued % NSTAGES) * Cfg<D>::STAGE_BYTES;
-      const uint32_t vd = kd + Cfg<D>::KV_BYTES;
-      const int n_valid = u.n_tokens - (stage * ST + pslot * 16);  // valid token rows of this thread's page
-      const int64_t blk = page >= 0 ? ((int64_t(page) * a.Hkv + u.kvh) << 4) * D + j * 8 : 0;
-      const bf16* ks = a.k_pages + blk;
-      const bf16* vs = a.v_pages + blk;
-      constexpr int ROW_STEP = 32 / Cfg<D>::CPR;  // token rows between successive pieces of a thread
-      if (n_valid >= 16) {
+    const int b = issued % NSTAGES;
+    wait_or_flag(sy, sy.empty + 8 * b, ((issued / NSTAGES) & 1) ^ 1);  // every warp has released the buffer
+    const int n_pages = min(4, (u.n_tokens - stage * ST + 15) >> 4);
+    const uint32_t bar = sy.full + 8 * b;
+    mv::mbar_arrive_expect_tx(bar, uint32_t(n_pages) * 16 * D * 2 * 2);
+    const uint32_t kd = smem_base + b * Cfg<D>::STAGE_BYTES, vd = kd + Cfg<D>::KV_BYTES;
 #pragma unroll
-        for (int k = 0; k < Cfg<D>::NCP; ++k) {
-          mv::cp_async_16(kd + dst[k], ks + k * 256, 16);
-          mv::cp_async_16(vd + dst[k], vs + k * 256, 16);
-        }
-      } else {
+    for (int p = 0; p < 4; ++p) {
+      if (p < n_pages) {
+        const int row = (pg[p] * a.Hkv + u.kvh) << 4;
 #pragma unroll
-        for (int k = 0; k < Cfg<D>::NCP; ++k) {
-          const bool ok = (row0 + k * ROW_STEP) < n_valid;  // beyond the node's last token: zero-fill
-          mv::cp_async_16(kd + dst[k], ok ? ks + k * 256 : a.k_pages, ok ? 16 : 0);
-          mv::cp_async_16(vd + dst[k], ok ? vs + k * 256 : a.v_pages, ok ? 16 : 0);
+        for (int h = 0; h < Cfg<D>::HALVES; ++h) {
+          mv::tma_load_2d(kd + h * Cfg<D>::HALF_BYTES + p * 2048, tm_k, h * 64, row, bar);
+          mv::tma_load_2d(vd + h * Cfg<D>::HALF_BYTES + p * 2048, tm_v, h * 64, row, bar);
         }
       }
-      ++stage;
-      if (stage == u.n_stages) {
-        ++which;
-        stage = 0;
-      }
-      prefetch_page(a, cu, nu);
     }
-    mv::cp_async_commit();
+    ++stage;
+    if (stage == u.n_stages) {
+      ++which;
+      stage = 0;
+    }
+    prefetch_pages(a, cu, nu);
     ++issued;
     return true;
   }
-  // Brings the pipeline back to NSTAGES-1 stages in flight (as far as stages exist).
-  __device__ __forceinline__ void top_up(const DecodeArgs& a, const Unit& cu, const Unit& nu, uint32_t smem_base, int consumed) {
-    while (issued - consumed < NSTAGES - 1 && issue(a, cu, nu, smem_base)) {
+  // Keeps up to NSTAGES stages issued ahead of the consumers (as far as stages exist).
+  __device__ __forceinline__ void top_up(const DecodeArgs& a, const Unit& cu, const Unit& nu, uint32_t smem_base, const Sync& sy,
+                                         const CUtensorMap* tm_k, const CUtensorMap* tm_v, int consumed) {
+    while (issued - consumed < NSTAGES && issue(a, cu, nu, smem_base, sy, tm_k, tm_v)) {
     }
   }
 };
-
-// Waits until the group of the stage about to be consumed has landed: `lead` = issued - consumed groups are
-// outstanding at most, of which all but the oldest may stay pending.
-__device__ __forceinline__ void wait_stage(int lead) {
-  static_assert(NSTAGES == 3, "wait_stage enumerates the pending counts of a 3-stage pipeline");
-  if (lead >= 2) mv::cp_async_wait<1>();
-  else mv::cp_async_wait<0>();
-}
 
 // merge (m, l, o) of another kv-split into mine; both in this thread's fragment layout
 template <int DT>
@@ -169,9 +163,9 @@ __device__ __forceinline__ void merge_frag(float& m0, float& m1, float& l0, floa
 
 // Consumes all stages of unit `cu` with MT m-tiles of 16 q-vectors; warp w: m-tile (w % MT), kv split (w / MT).
 template <int D, int MT>
-__device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu, const Unit& nu, Loader<D>& ld,
-                                             int& consumed, unsigned char* smem, uint32_t smem_base, int32_t pending,
-                                             int32_t* s_next) {
+__device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu, const Unit& nu, Loader<D>& ld, int& consumed,
+                                             unsigned char* smem, uint32_t smem_base, const Sync& sy, const CUtensorMap* tm_k,
+                                             const CUtensorMap* tm_v, int32_t pending, int32_t* s_next) {
   constexpr int KS = 4 / MT;      // kv splits inside a stage
   constexpr int WT = ST / KS;     // tokens per warp per stage
   constexpr int NT = WT / 8;      // S n-tiles per warp
@@ -216,102 +210,120 @@ __device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu
   const int tok_w = ks * WT;                                  // first token of this warp inside a stage
 
   for (int s = 0; s < cu.n_stages; ++s) {
-    wait_stage(ld.issued - consumed);
-    __syncthreads();
-    ld.issue(a, cu, nu, smem_base);  // refills the buffer consumed one iteration ago
-    if (s == 0 && tid == 0) *s_next = pending;  // unit after `nu`; read by everyone after this unit's epilogue
-    const uint32_t kb = smem_base + (consumed % NSTAGES) * Cfg<D>::STAGE_BYTES, vb = kb + Cfg<D>::KV_BYTES;
+    if (tid == 0) {
+      ld.top_up(a, cu, nu, smem_base, sy, tm_k, tm_v, consumed);
+      if (s == 0) *s_next = pending;  // unit after `nu`; read by everyone after this unit's epilogue
+    }
+    const int b = consumed % NSTAGES;
+    wait_or_flag(sy, sy.full + 8 * b, (consumed / NSTAGES) & 1);
+    const uint32_t kb = smem_base + b * Cfg<D>::STAGE_BYTES, vb = kb + Cfg<D>::KV_BYTES;
     ++consumed;
+    const bool last = (s == cu.n_stages - 1);
     const int tok_lim = cu.n_tokens - (s * ST + tok_w);  // valid tokens of this warp's slice
-    if (tok_lim <= 0) continue;                          // warp-uniform
-
-    float sacc[NT][4];
-#pragma unroll
-    for (int i = 0; i < NT; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
-#pragma unroll
-    for (int kk = 0; kk < KSTEPS; ++kk) {
-#pragma unroll
-      for (int np = 0; np < NT / 2; ++np) {
-        uint32_t b[4];
-        const int tok = tok_w + np * 16 + (lane & 7) + ((lane >> 4) << 3);
-        mv::ldmatrix_x4(b, kb + swz<D>(tok, kk * 2 + ((lane >> 3) & 1)));
-        mv::mma_bf16_16816(sacc[2 * np], qf[kk], b[0], b[1]);
-        mv::mma_bf16_16816(sacc[2 * np + 1], qf[kk], b[2], b[3]);
-      }
-    }
-    // scale to log2 units, mask the ragged tail, online softmax
-    float mx0 = -INFINITY, mx1 = -INFINITY;
-    if (tok_lim >= WT) {
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) sacc[nt][e] *= a.scale_log2;
-        mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
-        mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
-      }
-    } else {
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
-          sacc[nt][e] = (col < tok_lim) ? sacc[nt][e] * a.scale_log2 : -INFINITY;
+    if (tok_lim > 0) {                                   // warp-uniform
+      if (tok_lim < WT) {
+        // ragged end of the node: rows past the last token hold whatever the page (or an older stage) left
+        // there; V must be zero where P is zero, or 0 * NaN would poison the output
+        const int r0 = tok_w + tok_lim, nz = (WT - tok_lim) * Cfg<D>::CPR;
+        for (int i = lane; i < nz; i += 32) {
+          const int r = r0 + i / Cfg<D>::CPR, c = i % Cfg<D>::CPR;
+          *reinterpret_cast<uint4*>(smem + (vb - smem_base) + tile_off<D>(r, c)) = make_uint4(0, 0, 0, 0);
         }
-        mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
-        mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
+        __syncwarp();
+      }
+      float sacc[NT][4];
+#pragma unroll
+      for (int i = 0; i < NT; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
+#pragma unroll
+      for (int kk = 0; kk < KSTEPS; ++kk) {
+#pragma unroll
+        for (int np = 0; np < NT / 2; ++np) {
+          uint32_t bq[4];
+          const int tok = tok_w + np * 16 + (lane & 7) + ((lane >> 4) << 3);
+          mv::ldmatrix_x4(bq, kb + tile_off<D>(tok, kk * 2 + ((lane >> 3) & 1)));
+          mv::mma_bf16_16816(sacc[2 * np], qf[kk], bq[0], bq[1]);
+          mv::mma_bf16_16816(sacc[2 * np + 1], qf[kk], bq[2], bq[3]);
+        }
+      }
+      // scale to log2 units, mask the ragged tail, online softmax
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+      if (tok_lim >= WT) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) sacc[nt][e] *= a.scale_log2;
+          mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
+          mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
+        }
+      } else {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
+            sacc[nt][e] = (col < tok_lim) ? sacc[nt][e] * a.scale_log2 : -INFINITY;
+          }
+          mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
+          mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
+        }
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);  // finite: column 0 of the slice is valid
+      const bool grow = (mn0 > m0) || (mn1 > m1);
+      if (__any_sync(0xffffffffu, grow)) {  // rescale only when some row's maximum moved
+        const float al0 = mv::fast_exp2(m0 - mn0), al1 = mv::fast_exp2(m1 - mn1);
+        l0 *= al0;
+        l1 *= al1;
+#pragma unroll
+        for (int i = 0; i < DT; ++i) {
+          oacc[i][0] *= al0; oacc[i][1] *= al0;
+          oacc[i][2] *= al1; oacc[i][3] *= al1;
+        }
+        m0 = mn0;
+        m1 = mn1;
+      }
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        sacc[nt][0] = mv::fast_exp2(sacc[nt][0] - m0);
+        sacc[nt][1] = mv::fast_exp2(sacc[nt][1] - m0);
+        sacc[nt][2] = mv::fast_exp2(sacc[nt][2] - m1);
+        sacc[nt][3] = mv::fast_exp2(sacc[nt][3] - m1);
+        l0 += sacc[nt][0] + sacc[nt][1];  // per-thread partial sums; reduced over the quad at the end
+        l1 += sacc[nt][2] + sacc[nt][3];
+      }
+      // O += P V
+#pragma unroll
+      for (int kt = 0; kt < WT / 16; ++kt) {
+        uint32_t pa[4];
+        pa[0] = mv::pack_bf16(sacc[2 * kt][0], sacc[2 * kt][1]);
+        pa[1] = mv::pack_bf16(sacc[2 * kt][2], sacc[2 * kt][3]);
+        pa[2] = mv::pack_bf16(sacc[2 * kt + 1][0], sacc[2 * kt + 1][1]);
+        pa[3] = mv::pack_bf16(sacc[2 * kt + 1][2], sacc[2 * kt + 1][3]);
+#pragma unroll
+        for (int dp = 0; dp < DT / 2; ++dp) {
+          uint32_t bv[4];
+          const int tok = tok_w + kt * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+          mv::ldmatrix_x4_trans(bv, vb + tile_off<D>(tok, dp * 2 + (lane >> 4)));
+          mv::mma_bf16_16816(oacc[2 * dp], pa, bv[0], bv[1]);
+          mv::mma_bf16_16816(oacc[2 * dp + 1], pa, bv[2], bv[3]);
+        }
       }
     }
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);  // finite: column 0 of the slice is valid
-    const bool grow = (mn0 > m0) || (mn1 > m1);
-    if (__any_sync(0xffffffffu, grow)) {  // rescale only when some row's maximum moved
-      const float al0 = mv::fast_exp2(m0 - mn0), al1 = mv::fast_exp2(m1 - mn1);
-      l0 *= al0;
-      l1 *= al1;
-#pragma unroll
-      for (int i = 0; i < DT; ++i) {
-        oacc[i][0] *= al0; oacc[i][1] *= al0;
-        oacc[i][2] *= al1; oacc[i][3] *= al1;
-      }
-      m0 = mn0;
-      m1 = mn1;
-    }
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      sacc[nt][0] = mv::fast_exp2(sacc[nt][0] - m0);
-      sacc[nt][1] = mv::fast_exp2(sacc[nt][1] - m0);
-      sacc[nt][2] = mv::fast_exp2(sacc[nt][2] - m1);
-      sacc[nt][3] = mv::fast_exp2(sacc[nt][3] - m1);
-      l0 += sacc[nt][0] + sacc[nt][1];  // per-thread partial sums; reduced over the quad at the end
-      l1 += sacc[nt][2] + sacc[nt][3];
-    }
-    // O += P V
-#pragma unroll
-    for (int kt = 0; kt < WT / 16; ++kt) {
-      uint32_t pa[4];
-      pa[0] = mv::pack_bf16(sacc[2 * kt][0], sacc[2 * kt][1]);
-      pa[1] = mv::pack_bf16(sacc[2 * kt][2], sacc[2 * kt][3]);
-      pa[2] = mv::pack_bf16(sacc[2 * kt + 1][0], sacc[2 * kt + 1][1]);
-      pa[3] = mv::pack_bf16(sacc[2 * kt + 1][2], sacc[2 * kt + 1][3]);
-#pragma unroll
-      for (int dp = 0; dp < DT / 2; ++dp) {
-        uint32_t b[4];
-        const int tok = tok_w + kt * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
-        mv::ldmatrix_x4_trans(b, vb + swz<D>(tok, dp * 2 + (lane >> 4)));
-        mv::mma_bf16_16816(oacc[2 * dp], pa, b[0], b[1]);
-        mv::mma_bf16_16816(oacc[2 * dp + 1], pa, b[2], b[3]);
-      }
+    if (!last) {  // hand the stage back; the unit's last stage is kept as scratch for the epilogue
+      __syncwarp();
+      if (lane == 0) mv::mbar_arrive(sy.empty + 8 * b);
     }
   }
 
-  // ---- epilogue: combine the KS kv-splits through the stage buffer that was consumed last (it is refilled
-  // only after the next top-of-loop barrier), then write one partial per q-vector
+  // ---- epilogue: combine the KS kv-splits through the stage buffer that was consumed last, then write one
+  // partial per q-vector
+  const int b_last = (consumed - 1) % NSTAGES;
   if (KS > 1) {
-    float4* sc_o = reinterpret_cast<float4*>(smem + ((consumed - 1) % NSTAGES) * Cfg<D>::STAGE_BYTES);  // [2][DT][32]
-    float4* sc_ml = sc_o + 2 * DT * 32;                                                               // [2][32]
+    float4* sc_o = reinterpret_cast<float4*>(smem + b_last * Cfg<D>::STAGE_BYTES);  // [2][DT][32]
+    float4* sc_ml = sc_o + 2 * DT * 32;                                             // [2][32]
     __syncthreads();  // everyone has finished reading the last stage
     if (KS == 4) {
       if (warp >= 2) {
@@ -340,7 +352,10 @@ __device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu
       __syncthreads();
       if (ks == 0) merge_frag<DT>(m0, m1, l0, l1, oacc, sc_ml[mt * 32 + lane], sc_o + mt * DT * 32, lane);
     }
+    mv::fence_proxy_async();  // the scratch writes precede the TMA refill of this buffer
   }
+  __syncwarp();
+  if (lane == 0) mv::mbar_arrive(sy.empty + 8 * b_last);
   if (ks == 0) {
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
     l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
@@ -363,12 +378,29 @@ __device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu
 }
 
 template <int D>
-__global__ void __launch_bounds__(NTHREADS, 2) decode_attn_kernel(const DecodeArgs a) {
-  extern __shared__ __align__(128) unsigned char smem[];
+__global__ void __launch_bounds__(NTHREADS, 2) decode_attn_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tm_k,
+                                                                  const __grid_constant__ CUtensorMap tm_v) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) uint64_t s_bar[2 * NSTAGES];
   __shared__ int32_t s_ids[3];
+  __shared__ int s_abort;
   const int tid = threadIdx.x;
-  const uint32_t smem_base = mv::smem_u32(smem);
+  const uint32_t raw = mv::smem_u32(smem_raw);
+  const uint32_t smem_base = (raw + 1023u) & ~1023u;  // the swizzle pattern is anchored at 1024-byte boundaries
+  unsigned char* smem = smem_raw + (smem_base - raw);
+  Sync sy;
+  sy.full = mv::smem_u32(&s_bar[0]);
+  sy.empty = mv::smem_u32(&s_bar[NSTAGES]);
+  sy.abort = &s_abort;
+  sy.status = a.sched + 2;
   if (tid == 0) {
+    s_abort = 0;
+    for (int i = 0; i < NSTAGES; ++i) {
+      mv::mbar_init(sy.full + 8 * i, 1);   // the producer's arrive (+ the bytes TMA reports)
+      mv::mbar_init(sy.empty + 8 * i, 4);  // one arrive per consumer warp
+    }
+    mv::mbar_fence_init();
+    mv::fence_proxy_async();
     s_ids[0] = atomicAdd(a.sched, 1);
     s_ids[1] = atomicAdd(a.sched, 1);
   }
@@ -376,31 +408,34 @@ __global__ void __launch_bounds__(NTHREADS, 2) decode_attn_kernel(const DecodeAr
   Unit cu = load_unit(a, s_ids[0]);
   Unit nu = load_unit(a, s_ids[1]);
   Loader<D> ld;
-  ld.init(tid);
-  ld.prefetch_page(a, cu, nu);
   int consumed = 0;
-  ld.top_up(a, cu, nu, smem_base, consumed);
+  if (tid == 0) {
+    ld.prefetch_pages(a, cu, nu);
+    ld.top_up(a, cu, nu, smem_base, sy, &tm_k, &tm_v, consumed);
+  }
   while (cu.n_stages > 0) {
     int32_t pending = 0;
-    if (tid == 0) pending = atomicAdd(a.sched, 1);  // the unit after `nu`; consumed one barrier later
+    if (tid == 0) pending = atomicAdd(a.sched, 1);  // the unit after `nu`; published one stage later
     const int nqv = cu.n_rows * a.G;
-    if (nqv <= 16) process_unit<D, 1>(a, cu, nu, ld, consumed, smem, smem_base, pending, &s_ids[2]);
-    else if (nqv <= 32) process_unit<D, 2>(a, cu, nu, ld, consumed, smem, smem_base, pending, &s_ids[2]);
-    else process_unit<D, 4>(a, cu, nu, ld, consumed, smem, smem_base, pending, &s_ids[2]);
-    __syncthreads();  // s_ids[2] is visible; the epilogue's scratch reads are done
+    if (nqv <= 16) process_unit<D, 1>(a, cu, nu, ld, consumed, smem, smem_base, sy, &tm_k, &tm_v, pending, &s_ids[2]);
+    else if (nqv <= 32) process_unit<D, 2>(a, cu, nu, ld, consumed, smem, smem_base, sy, &tm_k, &tm_v, pending, &s_ids[2]);
+    else process_unit<D, 4>(a, cu, nu, ld, consumed, smem, smem_base, sy, &tm_k, &tm_v, pending, &s_ids[2]);
+    __syncthreads();  // s_ids[2] is visible to everyone
     cu = nu;
     nu = load_unit(a, s_ids[2]);
-    // the loader had finished `cu` (it was consumed), so it stands in the old `nu` or beyond it
-    ld.which -= 1;
-    if (ld.which == 1) ld.prefetch_page(a, cu, nu);  // it was beyond: it now stands at the first stage of the new `nu`
-    ld.top_up(a, cu, nu, smem_base, consumed);
+    __syncthreads();  // s_ids[2] may be overwritten from here on
+    if (tid == 0) {
+      // the loader had finished the old `cu` (it was consumed), so it stands in the old `nu` or beyond it
+      ld.which -= 1;
+      if (ld.which == 1) ld.prefetch_pages(a, cu, nu);  // it was beyond: it now stands at the first stage of the new `nu`
+      ld.top_up(a, cu, nu, smem_base, sy, &tm_k, &tm_v, consumed);
+    }
   }
-  mv::cp_async_wait<0>();
-  // the last CTA to finish re-arms the scheduler words for the next launch
+  // every stage that was issued has been consumed (the loader never runs past `nu`, and `nu` is empty here)
   if (tid == 0) {
     __threadfence();
     const int done = atomicAdd(a.sched + 1, 1);
-    if (done == int(gridDim.x) - 1) {
+    if (done == int(gridDim.x) - 1) {  // the last CTA to finish re-arms the scheduler words for the next launch
       a.sched[0] = 0;
       a.sched[1] = 0;
       __threadfence();
@@ -458,6 +493,14 @@ int sm_count() {
   return n;
 }
 
+struct TmapCache {  // the pools rarely change between calls: keep the last pair of tensor maps
+  const void* k = nullptr;
+  const void* v = nullptr;
+  int64_t rows = 0;
+  int d = 0;
+  CUtensorMap tm_k, tm_v;
+};
+
 template <int D>
 mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* kp, const void* vp, void* out,
                  void* ws, cudaStream_t st) {
@@ -469,12 +512,24 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
     }
     attr_set = true;
   }
+  static thread_local TmapCache tc[4];
+  static thread_local int tc_next = 0;
+  const int64_t rows = g->num_pages * g->n_kv_heads * 16;
+  TmapCache* hit = nullptr;
+  for (auto& c : tc)
+    if (c.k == kp && c.v == vp && c.rows == rows && c.d == D) hit = &c;
+  if (!hit) {
+    hit = &tc[tc_next];
+    tc_next = (tc_next + 1) % 4;
+    hit->k = nullptr;
+    if (!mv::make_tmap_bf16_2d(&hit->tm_k, kp, uint64_t(rows), D, 16) || !mv::make_tmap_bf16_2d(&hit->tm_v, vp, uint64_t(rows), D, 16))
+      return MV_ERR_CUDA;
+    hit->k = kp; hit->v = vp; hit->rows = rows; hit->d = D;
+  }
   const size_t parts = size_t(P->stats.n_partials);
   const size_t o_bytes = (parts * g->n_q_heads * D * sizeof(float) + 255) & ~size_t(255);
   DecodeArgs a;
   a.q = static_cast<const bf16*>(q);
-  a.k_pages = static_cast<const bf16*>(kp);
-  a.v_pages = static_cast<const bf16*>(vp);
   a.page_idx = mv::table<int32_t>(P, P->layout.page_idx);
   a.items = mv::table<mv::WorkItem>(P, P->layout.items);
   a.item_rows = mv::table<mv::ItemRow>(P, P->layout.item_rows);
@@ -487,7 +542,7 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
   a.n_units = int(P->stats.n_items) * g->n_kv_heads;
   a.scale_log2 = mv::softmax_scale(g) * 1.4426950408889634f;
   const int grid = std::min(a.n_units, 2 * sm_count());
-  decode_attn_kernel<D><<<grid, NTHREADS, Cfg<D>::SMEM, st>>>(a);
+  decode_attn_kernel<D><<<grid, NTHREADS, Cfg<D>::SMEM, st>>>(a, hit->tm_k, hit->tm_v);
   mv::g_launches++;
   if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
   const int n_rows = int(P->stats.n_new_tokens);
@@ -512,9 +567,23 @@ extern "C" mv_status mv_dag_decode_attn(const mv_plan* P, const mv_attn_geom* g,
   if (!q_rot || !k_pages || !v_pages || !out) return MV_ERR_INVALID_ARG;
   if (!P->device_buf) return MV_ERR_WORKSPACE;
   if (P->stats.max_page_id >= g->num_pages) return MV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k_pages) & 15) || (reinterpret_cast<uintptr_t>(v_pages) & 15)) return MV_ERR_INVALID_ARG;
   const size_t need = mv_workspace_bytes(P, g, MV_OP_DECODE_ATTN);
   if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return MV_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   return g->head_dim == 128 ? launch<128>(P, g, q_rot, k_pages, v_pages, out, workspace, s)
                             : launch<64>(P, g, q_rot, k_pages, v_pages, out, workspace, s);
+}
+
+extern "C" mv_status mv_plan_read_status(const mv_plan* P, void* cuda_stream, int32_t* status) {
+  if (!P || !P->valid || !status) return MV_ERR_INVALID_ARG;
+  if (!P->device_buf) return MV_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const char* src = static_cast<const char*>(P->device_buf) + P->layout.sched + 2 * sizeof(int32_t);
+  if (cudaMemcpyAsync(status, src, sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return MV_ERR_CUDA;
+  }
+  return MV_OK;
 }

@@ -229,6 +229,7 @@ def test_decode_random_dags(chunk, hq, hkv, d):
             st = rt.DecodeState(wl, chunk_tokens=chunk, canary=True)
             got = _np(st.step())
             torch.cuda.synchronize()
+            assert st.plan.read_status() == 0
             check_decode(wl, got)
 
 
@@ -237,7 +238,13 @@ def test_decode_config2_small_all_rows():
     wl = synth.config2(n_req=3, prefix=700, branches=4, branch_len=90)
     st = rt.DecodeState(wl, canary=True)
     got = _np(st.step())
+    assert st.plan.read_status() == 0
     check_decode(wl, got)
+    # the same plan and tables serve repeated launches (scheduler words re-arm themselves)
+    for _ in range(3):
+        again = _np(st.step())
+        assert np.array_equal(again, got)
+    assert st.plan.read_status() == 0
 
 
 def test_decode_many_siblings_more_than_64_qvectors():
