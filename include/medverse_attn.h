@@ -193,6 +193,31 @@ mv_status mv_dag_decode_attn(const mv_plan* plan, const mv_attn_geom* geom, cons
                              const void* k_pages, const void* v_pages, void* out, void* workspace,
                              size_t workspace_bytes, void* cuda_stream);
 
+/* Decode attention for callers that cannot allocate device memory.  (The paper has no counterpart: this is
+ * a packaging variant of mv_dag_decode_attn, same arithmetic, same kernels.)
+ *
+ * Some hosts of this library may not call cudaMalloc or an allocating library routine on the decode path:
+ * a serving loop whose memory pool is fixed at start-up and fully handed out, a plug-in that runs inside
+ * another runtime's allocator-free region, or code that must not synchronise the device (cudaMalloc and
+ * cudaFree do).  For them the split-KV scratch that mv_dag_decode_attn takes as `workspace` is replaced by
+ * a fixed array of MV_STATIC_WORKSPACE_BYTES bytes that is part of the library image: every GPU on which
+ * the library is loaded holds that much memory until the process exits.  The caller still passes q_rot,
+ * the pools and out, exactly as for mv_dag_decode_attn; nothing is allocated or freed by this call.
+ *
+ *   - Limit: plans with mv_workspace_bytes(plan, geom, MV_OP_DECODE_ATTN) > MV_STATIC_WORKSPACE_BYTES are
+ *     refused with MV_ERR_WORKSPACE before anything is launched (query it with mv_static_workspace_bytes()).
+ *   - Set-up: the first call on each device looks up the array's device address (one cudaGetSymbolAddress,
+ *     with the calling thread's current device); make that first call outside any stream capture.
+ *   - Sharing: every call on a device uses the same array and finds the previous call's contents in it.
+ *     The kernels write each partial result before they read it, so nothing needs clearing; but two calls
+ *     whose kernels overlap on the GPU (different streams, no ordering between them) race on it.  Order such
+ *     calls, or give all but one of them their own workspace through mv_dag_decode_attn.
+ * Other errors are those of mv_dag_decode_attn. */
+#define MV_STATIC_WORKSPACE_BYTES (16u << 20)
+size_t mv_static_workspace_bytes(void);
+mv_status mv_dag_decode_attn_static(const mv_plan* plan, const mv_attn_geom* geom, const void* q_rot,
+                                    const void* k_pages, const void* v_pages, void* out, void* cuda_stream);
+
 /* Topology-masked prefill attention over a flattened DAG sequence (Eq. 3; the training-time layout of
  * Sec. 4.2 and the engine's re-prefill): all tokens of the batch are new and contiguous in
  * (request, node, token) order;

@@ -26,7 +26,8 @@ TABLES = {"layer": (0, np.int32), "pos_start": (1, np.int32), "pos_id": (2, np.i
 EXPORTS = ["mv_plan_dag", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_bytes", "mv_plan_upload",
            "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
            "mv_dag_prefill_attn", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_status_string",
-           "mv_launch_count", "mv_plan_read_status"]
+           "mv_launch_count", "mv_plan_read_status", "mv_dag_decode_attn_static",
+           "mv_static_workspace_bytes"]
 
 
 class MvError(RuntimeError):
@@ -73,6 +74,9 @@ def _load():
     lib.mv_rope_write_kv.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 8
     lib.mv_dag_decode_attn.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp, sz, vp]
     lib.mv_dag_prefill_attn.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp, sz, vp]
+    lib.mv_dag_decode_attn_static.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp]
+    lib.mv_static_workspace_bytes.argtypes = []
+    lib.mv_static_workspace_bytes.restype = sz
     lib.mv_decode_step_staging_bytes.argtypes = [vp, C.POINTER(_Geom)]
     lib.mv_decode_step_staging_bytes.restype = sz
     lib.mv_decode_step_host.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 7 + [sz, vp]
@@ -206,6 +210,18 @@ def mv_dag_decode_attn(plan: Plan, geom: _Geom, q_rot, k_pages, v_pages, out, wo
     nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib.mv_dag_decode_attn(plan.handle, C.byref(geom), _ptr(q_rot), _ptr(k_pages), _ptr(v_pages), _ptr(out),
                                   _ptr(workspace), nbytes, _stream_ptr(stream)), "mv_dag_decode_attn")
+
+
+def mv_dag_decode_attn_static(plan: Plan, geom: _Geom, q_rot, k_pages, v_pages, out, stream=None):
+    """mv_dag_decode_attn without a workspace argument: for callers that may not allocate device memory, the
+    split-KV scratch is a fixed array inside the library (``mv_static_workspace_bytes()`` bytes; larger plans
+    raise MV_ERR_WORKSPACE).  Calls on one device share that array, so they must not overlap on the GPU."""
+    _check(lib.mv_dag_decode_attn_static(plan.handle, C.byref(geom), _ptr(q_rot), _ptr(k_pages), _ptr(v_pages),
+                                         _ptr(out), _stream_ptr(stream)), "mv_dag_decode_attn_static")
+
+
+def mv_static_workspace_bytes() -> int:
+    return int(lib.mv_static_workspace_bytes())
 
 
 def mv_dag_prefill_attn(plan: Plan, geom: _Geom, q_rot, k_rot, v, out, workspace=None, stream=None):

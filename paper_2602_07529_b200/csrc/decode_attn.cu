@@ -18,6 +18,8 @@
 //
 // Every wait on an mbarrier is bounded: if it runs out, the CTA records MV_ERR_TIMEOUT in the plan's
 // status word, stops waiting and still reaches every barrier, so the kernel always terminates.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace {
@@ -573,6 +575,52 @@ extern "C" mv_status mv_dag_decode_attn(const mv_plan* P, const mv_attn_geom* g,
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   return g->head_dim == 128 ? launch<128>(P, g, q_rot, k_pages, v_pages, out, workspace, s)
                             : launch<64>(P, g, q_rot, k_pages, v_pages, out, workspace, s);
+}
+
+// ---- decode attention for callers that cannot allocate device memory -------------------------------------
+// The split-KV scratch lives in a file-scope device array instead of a caller-provided workspace.  In host
+// code the array's name is only a stand-in for the symbol, not a device address, so the address the kernels
+// receive is looked up with cudaGetSymbolAddress, once per device, with that device current.
+namespace {
+__device__ __align__(256) unsigned char g_static_scratch[MV_STATIC_WORKSPACE_BYTES];
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};
+std::mutex g_static_scratch_mu;
+
+mv_status static_scratch_for_current_device(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    (void)cudaGetLastError();
+    return MV_ERR_CUDA;
+  }
+  std::lock_guard<std::mutex> lock(g_static_scratch_mu);
+  if (!g_static_scratch_addr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+      (void)cudaGetLastError();
+      return MV_ERR_CUDA;
+    }
+    g_static_scratch_addr[dev] = p;
+  }
+  *out = g_static_scratch_addr[dev];
+  return MV_OK;
+}
+}  // namespace
+
+extern "C" size_t mv_static_workspace_bytes(void) { return size_t(MV_STATIC_WORKSPACE_BYTES); }
+
+extern "C" mv_status mv_dag_decode_attn_static(const mv_plan* P, const mv_attn_geom* g, const void* q_rot,
+                                               const void* k_pages, const void* v_pages, void* out, void* cuda_stream) {
+  if (!P || !P->valid) return MV_ERR_INVALID_ARG;
+  mv_status st = mv::check_geom(g);
+  if (st != MV_OK) return st;
+  // the size check comes before anything touches the device: a plan that needs more scratch than the library
+  // holds is refused, never truncated
+  if (mv_workspace_bytes(P, g, MV_OP_DECODE_ATTN) > size_t(MV_STATIC_WORKSPACE_BYTES)) return MV_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  st = static_scratch_for_current_device(&scratch);
+  if (st != MV_OK) return st;
+  return mv_dag_decode_attn(P, g, q_rot, k_pages, v_pages, out, scratch, size_t(MV_STATIC_WORKSPACE_BYTES), cuda_stream);
 }
 
 extern "C" mv_status mv_plan_read_status(const mv_plan* P, void* cuda_stream, int32_t* status) {
