@@ -18,8 +18,12 @@
  *   - Errors: an mv_status is returned; argument errors are found on the host before any launch.
  *     Kernels never trap.  mv_status_string() names a status.
  *   - Layouts: q, k, v, q_rot, out are [tokens][heads][head_dim], row-major, element type
- *     mv_attn_geom.dtype.  The K and V page pools are separate buffers, each
- *     [num_pages][n_kv_heads][page_size][head_dim] of the same element type.
+ *     mv_attn_geom.dtype.  The K and V page pools are separate buffers of the same element type, each
+ *     [num_pages][n_kv_heads][head_dim / 64][page_size][64]: the block of one (page, KV head) is contiguous
+ *     (4 KB for bf16, head_dim 128) and holds the head vectors of its 16 tokens split into 64-element column
+ *     blocks, so that one bulk tensor copy with the 128-byte shared-memory swizzle moves the whole block.
+ *     Element c of token t of (page p, head h) is at ((p * n_kv_heads + h) * (head_dim / 64) + c / 64) * 1024
+ *     + t * 64 + c % 64.  Only mv_rope_write_kv writes the pools and only mv_dag_decode_attn reads them.
  *   - Order: "new tokens" (rows) are ordered (request, node index, token index) ascending.
  *   - Supported geometry: head_dim 64 or 128; n_q_heads a multiple of n_kv_heads; page_size 16.
  *     Anything else returns MV_ERR_UNSUPPORTED.  There is no CPU fallback.
@@ -79,16 +83,20 @@ typedef struct {
   int32_t page_size;         /* 16 */
   int32_t vis_mode;          /* mv_vis_mode */
   int32_t pos_mode;          /* mv_pos_mode */
-  int32_t chunk_tokens;      /* decode split-KV chunk length in tokens (multiple of page_size); 0 = automatic */
-  int32_t n_kv_heads;        /* scheduling hint: KV heads of the geometry the plan will run with (0 = 8)       */
-  int32_t group_size;        /* scheduling hint: n_q_heads / n_kv_heads (0 = 8).  A chunk's row set is split so
+  int32_t chunk_tokens;      /* decode: longest KV slice of one work unit in tokens (multiple of page_size);
+                                0 = no limit (slices are cut only where a CTA's equal share of the step ends)  */
+  int32_t n_kv_heads;        /* scheduling: KV heads of the geometry the plan will run with (0 = 8);
+                                mv_dag_decode_attn returns MV_ERR_UNSUPPORTED for any other head count         */
+  int32_t group_size;        /* scheduling: n_q_heads / n_kv_heads (0 = 8).  A node's row set is split so
                                 that rows * group_size <= 64; mv_dag_decode_attn returns MV_ERR_UNSUPPORTED if
                                 the geometry's real group size breaks that bound                               */
+  int32_t sched_ctas;        /* scheduling: CTAs the decode kernel runs with (0 = 296, two per SM of a 148-SM
+                                part); the step's KV stream is cut into that many equal shares                 */
 } mv_dag_batch;
 
 typedef struct {
   int32_t n_q_heads, n_kv_heads, head_dim, page_size;
-  int64_t num_pages;   /* pages in each of the K and V pools */
+  int64_t num_pages;   /* pages in each of the K and V pools (see "Layouts" above for the block layout) */
   int32_t dtype;       /* mv_dtype of q/k/v/out and of the pools */
   float sm_scale;      /* softmax scale; 0 means 1/sqrt(head_dim) */
   double rope_base;    /* theta_i = rope_base^(-2i/head_dim) */
@@ -115,9 +123,9 @@ typedef struct {
   int64_t n_nodes, n_new_tokens, n_qnodes, n_segs;
   int64_t decode_ready;        /* 1 if every q-node has exactly one new token (mv_dag_decode_attn applies) */
   int64_t prefill_ready;       /* 1 if no node holds older tokens (mv_dag_prefill_attn applies)            */
-  int64_t n_items;             /* decode: (KV chunk, row set) work items per KV head                        */
-  int64_t n_partials;          /* decode: split-KV partial results per query head                          */
-  int64_t chunk_tokens;        /* decode: chunk length used                                                 */
+  int64_t n_items;             /* decode: work units = (KV slice of a node, KV head, row set)                */
+  int64_t n_partials;          /* decode: split-KV partial results, each holding group_size head vectors    */
+  int64_t chunk_tokens;        /* decode: the slice limit in effect, or a CTA's share in tokens if none    */
   int64_t unique_kv_tokens;    /* tokens of every node at least one row sees, each once                    */
   int64_t per_row_kv_tokens;   /* sum over rows of visible tokens                                          */
   int64_t n_q_tiles;           /* prefill: query tiles                                                      */
@@ -127,6 +135,9 @@ typedef struct {
   int64_t max_page_id;         /* largest page id referenced                                                */
   int64_t max_item_rows;       /* decode: largest row set of a work item                                    */
   int64_t sched_kv_heads, sched_group; /* the scheduling hints in effect                                    */
+  int64_t n_ctas;              /* decode: CTAs the step was cut for                                         */
+  int64_t max_cta_cost;        /* decode: largest share handed to one CTA, in tokens of one KV head (a unit
+                                  counts as its tokens + 48)                                                */
 } mv_plan_stats;
 
 enum { MV_OP_ROPE_WRITE_KV = 0, MV_OP_DECODE_ATTN = 1, MV_OP_PREFILL_ATTN = 2 };

@@ -40,7 +40,8 @@ class _DagBatch(C.Structure):
     _fields_ = [("n_req", C.c_int32), ("node_off", C.c_void_p), ("node_len", C.c_void_p), ("node_new", C.c_void_p),
                 ("parent_off", C.c_void_p), ("parent_idx", C.c_void_p), ("page_off", C.c_void_p),
                 ("page_idx", C.c_void_p), ("page_size", C.c_int32), ("vis_mode", C.c_int32), ("pos_mode", C.c_int32),
-                ("chunk_tokens", C.c_int32), ("n_kv_heads", C.c_int32), ("group_size", C.c_int32)]
+                ("chunk_tokens", C.c_int32), ("n_kv_heads", C.c_int32), ("group_size", C.c_int32),
+                ("sched_ctas", C.c_int32)]
 
 
 class _Geom(C.Structure):
@@ -52,7 +53,7 @@ class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_nodes", "n_new_tokens", "n_qnodes", "n_segs", "decode_ready", "prefill_ready", "n_items", "n_partials",
         "chunk_tokens", "unique_kv_tokens", "per_row_kv_tokens", "n_q_tiles", "visible_pairs", "tile_pairs",
-        "max_page_id", "max_item_rows", "sched_kv_heads", "sched_group")]
+        "max_page_id", "max_item_rows", "sched_kv_heads", "sched_group", "n_ctas", "max_cta_cost")]
 
 
 def _load():
@@ -135,18 +136,18 @@ def geom_of(workload) -> _Geom:
 class Plan:
     """Owner of an ``mv_plan*``.  ``Plan(batch)`` plans; ``plan.replan(batch)`` recycles the same object."""
 
-    def __init__(self, batch=None, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0):
+    def __init__(self, batch=None, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0, sched_ctas: int = 0):
         self._h = C.c_void_p(None)
         self._keep = None
         if batch is not None:
-            self.replan(batch, chunk_tokens, n_kv_heads, group_size)
+            self.replan(batch, chunk_tokens, n_kv_heads, group_size, sched_ctas)
 
-    def replan(self, batch, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0):
+    def replan(self, batch, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0, sched_ctas: int = 0):
         arrs = [_i32(getattr(batch, n)) for n in ("node_off", "node_len", "node_new", "parent_off", "parent_idx",
                                                    "page_off", "page_idx")]
         self._keep = arrs
         b = _DagBatch(int(batch.n_req), *[a.ctypes.data for a in arrs], int(batch.page_size), int(batch.vis_mode),
-                      int(batch.pos_mode), int(chunk_tokens), int(n_kv_heads), int(group_size))
+                      int(batch.pos_mode), int(chunk_tokens), int(n_kv_heads), int(group_size), int(sched_ctas))
         self.c_batch = b
         _check(lib.mv_plan_dag(C.byref(b), C.byref(self._h)), "mv_plan_dag")
         return self
@@ -197,8 +198,8 @@ class Plan:
             pass
 
 
-def mv_plan_dag(batch, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0) -> Plan:
-    return Plan(batch, chunk_tokens, n_kv_heads, group_size)
+def mv_plan_dag(batch, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0, sched_ctas: int = 0) -> Plan:
+    return Plan(batch, chunk_tokens, n_kv_heads, group_size, sched_ctas)
 
 
 def mv_rope_write_kv(plan: Plan, geom: _Geom, q, k, v, q_rot, k_rot, k_pages, v_pages, stream=None):

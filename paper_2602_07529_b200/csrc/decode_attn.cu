@@ -1,20 +1,24 @@
 // Multi-branch decode attention over a shared paged KV cache (Eq. 2 with the DAG mask of Eq. 3; Fork =
 // shared prefix pages referenced by many rows, Join = union of the predecessors' segment lists, Sec. 4.3).
 //
-// Segment-major: the unit of work is (a page-aligned chunk of ONE node's KV, one KV head) together with
-// the set of rows (frontier tokens) that see that node.  The chunk is streamed from HBM exactly once and
-// serves every sibling row and the whole GQA group: the q-vectors (rows x group) are the M dimension of
-// bf16 tensor-core tiles (m16n8k16, fp32 accumulate), so that the arithmetic (16-64 flop per KV byte)
-// does not throttle the HBM stream.
+// Segment-major: a request's frontier rows and all the KV they see form one stream of 64-token stages, node
+// after node; a stage belongs to one node and carries the set of rows that see that node (the DAG mask at
+// stage granularity).  The unit of work is a run of such stages for one KV head.  Every stage is streamed
+// from HBM exactly once and serves every sibling row and the whole GQA group: the q-vectors (rows x group)
+// are the M dimension of bf16 tensor-core tiles (m16n8k16, fp32 accumulate), so that the arithmetic (16-64
+// flop per KV byte) does not throttle the HBM stream; rows that do not see a stage's node are masked out of
+// its softmax, and a warp none of whose rows see it skips it.
 //
-// Persistent CTAs (two per SM) pull units from an atomic work counter, longest first, and keep ONE
-// pipeline of 64-token stages running across unit boundaries.  A stage is filled by TMA: one elected
-// thread issues a [16 tokens][64 elements] box per half page block (cp.async.bulk.tensor, 128-byte
-// shared-memory swizzle, completion counted on an mbarrier), so no thread spends issue slots or
-// load-store-unit entries on the copy, and ldmatrix reads the tiles without bank conflicts.  Warps hand
-// a consumed stage back through a second mbarrier; there is no CTA-wide barrier inside a unit.  Softmax
-// is online, in log2 units; each unit leaves one partial (max, sum, unnormalised output) per q-vector in
-// the split-KV workspace and a second kernel merges the partials of every (row, head).
+// The planner cuts the step's whole KV stream into one equal share per CTA (two CTAs per SM), so there is
+// no run-time scheduler.  A CTA is one producer warp and four consumer warps around ONE ring of 64-token
+// stages that keeps running across unit boundaries.  The producer fills a stage with TMA: one box per
+// contiguous (page, KV head) block of K and of V (cp.async.bulk.tensor, 128-byte shared-memory swizzle,
+// completion counted on an mbarrier), eight lanes issuing one box each; it also stages the next unit's
+// q-vectors and partial-slot ids in shared memory (cp.async, completion on an mbarrier) while the current
+// unit is still being consumed.  Consumers hand a stage back through a second mbarrier.  Softmax is
+// online, in log2 units; each unit leaves one partial (max, sum, unnormalised output) per q-vector in the
+// split-KV workspace and a second kernel, launched with programmatic stream serialisation so that its
+// launch overlaps this kernel's tail, merges the partials of every (row, head).
 //
 // Every wait on an mbarrier is bounded: if it runs out, the CTA records MV_ERR_TIMEOUT in the plan's
 // status word, stops waiting and still reaches every barrier, so the kernel always terminates.
@@ -25,60 +29,68 @@
 namespace {
 
 using bf16 = __nv_bfloat16;
-constexpr int NTHREADS = 128;  // 4 warps
-constexpr int ST = 64;         // tokens per pipeline stage (4 pages)
+constexpr int NCONS = 128;           // consumer threads (4 warps)
+constexpr int NTHREADS = NCONS + 32; // + the producer warp (warp 4)
+constexpr int ST = 64;               // tokens per pipeline stage (4 pages)
 constexpr int NSTAGES = 3;
+constexpr int MAXQV = 64;            // q-vectors (rows x group) of one unit
 
 struct DecodeArgs {
   const bf16* q;
-  const int32_t* page_idx;
-  const mv::WorkItem* items;
+  const mv::StageDesc* stages;
+  const mv::WorkUnit* units;
+  const int32_t* cta_unit_off;
   const mv::ItemRow* item_rows;
-  float* part_o;   // [n_partials][Hq][D]
-  float* part_ml;  // [n_partials][Hq][2]  (max in log2 units, sum)
-  int32_t* sched;  // [0] next unit, [1] CTAs finished (both zero between launches), [2] status word
-  int Hq, Hkv, G, n_units;
+  float* part_o;    // [n_partials * G][D]
+  float* part_ml;   // [n_partials * G][2]  (max in log2 units, sum)
+  int32_t* status;  // device status word
+  int Hq, Hkv, G;
   float scale_log2;  // softmax scale * log2(e)
-};
-
-struct Unit {  // uniform across the CTA
-  int page_begin, n_tokens, row_begin, n_rows, kvh, n_stages;
 };
 
 template <int D>
 struct Cfg {
   static constexpr int CPR = D / 8;                 // 16-byte chunks per token row
   static constexpr int HALVES = D / 64;             // 128-byte column blocks per row (one TMA box each)
-  static constexpr int HALF_BYTES = ST * 128;       // one column block of a stage: [64 tokens][128 B]
+  static constexpr int PAGE_BYTES = 16 * D * 2;     // K (or V) block of one (page, KV head): one TMA box
   static constexpr int KV_BYTES = ST * D * 2;       // K (or V) bytes of a stage
   static constexpr int STAGE_BYTES = 2 * KV_BYTES;  // K then V
-  static constexpr int SMEM = NSTAGES * STAGE_BYTES + 1024;  // + slack to align the base to 1024 B
+  static constexpr int Q_BYTES = MAXQV * D * 2;     // q-vectors of one unit, [64][D] bf16, chunk-swizzled
+  // dynamic shared memory: stages | q | meta (see Smem)
+  static constexpr int OFF_Q = NSTAGES * STAGE_BYTES;
+  static constexpr int OFF_META = OFF_Q + Q_BYTES;
+  static constexpr int SMEM = OFF_META + 896;  // D = 128: 115,584 B, so that two CTAs share an SM
 };
 
-// Byte offset of 16-byte chunk `chunk` of token row `row` inside a K (or V) stage tile as TMA lays it out:
-// column block h = chunk / 8 holds [64 tokens][128 B]; inside it the hardware XORs the chunk index with row % 8.
+struct Meta {                       // tail of the dynamic shared memory
+  float2 ml[4][16];                 // epilogue: (max, sum) of every row of every consumer warp    512 B
+  int32_t pv[MAXQV];                // partial vector index (partial * G + head in group) or -1    256 B
+  int32_t n_stages, n_qv;
+  int32_t st_tokens[NSTAGES];       // per stage buffer: valid tokens
+  uint32_t st_mask_lo[NSTAGES], st_mask_hi[NSTAGES];  // per stage buffer: rows that see the stage
+  uint64_t full[NSTAGES], empty[NSTAGES], q_full, q_empty;
+  int abort;
+};
+static_assert(sizeof(Meta) <= 896, "meta area");
+
+// Byte offset of 16-byte chunk `chunk` of token row `row` inside a K (or V) stage tile as TMA lays it out: a
+// stage is four page blocks; a page block is [column block chunk / 8][16 tokens][128 B], and inside a
+// 128-byte row the hardware XORs the chunk index with row % 8.
 template <int D>
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
-  return uint32_t(chunk >> 3) * Cfg<D>::HALF_BYTES + uint32_t(row) * 128 + (uint32_t((chunk & 7) ^ (row & 7)) << 4);
+  return uint32_t(row >> 4) * Cfg<D>::PAGE_BYTES + uint32_t(chunk >> 3) * 2048 + uint32_t(row & 15) * 128 +
+         (uint32_t((chunk & 7) ^ (row & 7)) << 4);
+}
+// q buffer: row x, 16-byte chunk c at x * (D*2) + ((c ^ (x & 7)) << 4)
+template <int D>
+__device__ __forceinline__ uint32_t q_off(int x, int c) {
+  return uint32_t(x) * (D * 2) + (uint32_t(c ^ (x & 7)) << 4);
 }
 
-__device__ __forceinline__ Unit load_unit(const DecodeArgs& a, int u) {
-  Unit x;
-  if (u < a.n_units) {
-    const int4 it = *reinterpret_cast<const int4*>(a.items + u / a.Hkv);
-    x.page_begin = it.x; x.n_tokens = it.y; x.row_begin = it.z; x.n_rows = it.w;
-    x.kvh = u % a.Hkv;
-    x.n_stages = (it.y + ST - 1) / ST;
-  } else {
-    x.page_begin = 0; x.n_tokens = 0; x.row_begin = 0; x.n_rows = 0; x.kvh = 0; x.n_stages = 0;
-  }
-  return x;
-}
-
-struct Sync {  // shared-memory addresses of the pipeline barriers and flags
-  uint32_t full, empty;  // arrays of NSTAGES mbarriers (8 bytes each)
-  volatile int* abort;   // set once a bounded wait ran out
-  int32_t* status;       // global status word
+struct Sync {
+  uint32_t full, empty, q_full, q_empty;  // shared-memory addresses
+  volatile int* abort;                    // set once a bounded wait ran out
+  int32_t* status;                        // global status word
 };
 
 __device__ __forceinline__ void wait_or_flag(const Sync& sy, uint32_t bar, uint32_t parity) {
@@ -89,85 +101,125 @@ __device__ __forceinline__ void wait_or_flag(const Sync& sy, uint32_t bar, uint3
   }
 }
 
-// The producer side of the pipeline, run by thread 0: walks the stages of the current unit, then of the next.
-template <int D>
-struct Loader {
-  int which = 0;   // 0: current unit, 1: next unit, 2: beyond (nothing to issue)
-  int stage = 0;   // next stage of that unit to issue
-  int issued = 0;  // stages issued so far (buffer = issued % NSTAGES)
-  int pg[4] = {0, 0, 0, 0};  // prefetched page ids of the stage about to be issued
-
-  __device__ __forceinline__ void prefetch_pages(const DecodeArgs& a, const Unit& cu, const Unit& nu) {
-    const Unit& u = which == 0 ? cu : nu;
-    if (which <= 1 && stage < u.n_stages) {
-      const int n_pages = (u.n_tokens - stage * ST + 15) >> 4;
-#pragma unroll
-      for (int p = 0; p < 4; ++p) pg[p] = p < n_pages ? __ldg(a.page_idx + u.page_begin + stage * 4 + p) : 0;
-    }
-  }
-  __device__ __forceinline__ bool issue(const DecodeArgs& a, const Unit& cu, const Unit& nu, uint32_t smem_base, const Sync& sy,
-                                        const CUtensorMap* tm_k, const CUtensorMap* tm_v) {
-    const Unit& u = which == 0 ? cu : nu;
-    if (!(which <= 1 && stage < u.n_stages)) return false;
-    const int b = issued % NSTAGES;
-    wait_or_flag(sy, sy.empty + 8 * b, ((issued / NSTAGES) & 1) ^ 1);  // every warp has released the buffer
-    const int n_pages = min(4, (u.n_tokens - stage * ST + 15) >> 4);
-    const uint32_t bar = sy.full + 8 * b;
-    mv::mbar_arrive_expect_tx(bar, uint32_t(n_pages) * 16 * D * 2 * 2);
-    const uint32_t kd = smem_base + b * Cfg<D>::STAGE_BYTES, vd = kd + Cfg<D>::KV_BYTES;
-#pragma unroll
-    for (int p = 0; p < 4; ++p) {
-      if (p < n_pages) {
-        const int row = (pg[p] * a.Hkv + u.kvh) << 4;
-#pragma unroll
-        for (int h = 0; h < Cfg<D>::HALVES; ++h) {
-          mv::tma_load_2d(kd + h * Cfg<D>::HALF_BYTES + p * 2048, tm_k, h * 64, row, bar);
-          mv::tma_load_2d(vd + h * Cfg<D>::HALF_BYTES + p * 2048, tm_v, h * 64, row, bar);
-        }
-      }
-    }
-    ++stage;
-    if (stage == u.n_stages) {
-      ++which;
-      stage = 0;
-    }
-    prefetch_pages(a, cu, nu);
-    ++issued;
-    return true;
-  }
-  // Keeps up to NSTAGES stages issued ahead of the consumers (as far as stages exist).
-  __device__ __forceinline__ void top_up(const DecodeArgs& a, const Unit& cu, const Unit& nu, uint32_t smem_base, const Sync& sy,
-                                         const CUtensorMap* tm_k, const CUtensorMap* tm_v, int consumed) {
-    while (issued - consumed < NSTAGES && issue(a, cu, nu, smem_base, sy, tm_k, tm_v)) {
-    }
-  }
+// ---- producer warp: walks the CTA's units; per unit the q-vectors + slot ids, then the KV stages -----------------
+struct UnitRegs {  // a unit's descriptor, loaded ahead of use
+  int stage_begin = 0, n_stages = 0, row_begin = 0, n_rows = 0, kvh = 0;
+};
+struct StageRegs {  // one stage descriptor per lane (a window of 32 stages)
+  int4 a = make_int4(0, 0, 0, 0), b = make_int4(0, 0, 0, 0);
 };
 
-// merge (m, l, o) of another kv-split into mine; both in this thread's fragment layout
-template <int DT>
-__device__ __forceinline__ void merge_frag(float& m0, float& m1, float& l0, float& l1, float (&o)[DT][4], const float4 oml,
-                                           const float4* other_o, int lane) {
-  const float n0 = fmaxf(m0, oml.x), n1 = fmaxf(m1, oml.y);
-  const float ws0 = (m0 == -INFINITY) ? 0.f : mv::fast_exp2(m0 - n0), wo0 = (oml.x == -INFINITY) ? 0.f : mv::fast_exp2(oml.x - n0);
-  const float ws1 = (m1 == -INFINITY) ? 0.f : mv::fast_exp2(m1 - n1), wo1 = (oml.y == -INFINITY) ? 0.f : mv::fast_exp2(oml.y - n1);
-  m0 = n0; m1 = n1;
-  l0 = l0 * ws0 + oml.z * wo0;
-  l1 = l1 * ws1 + oml.w * wo1;
-#pragma unroll
-  for (int i = 0; i < DT; ++i) {
-    const float4 t = other_o[i * 32 + lane];
-    o[i][0] = o[i][0] * ws0 + t.x * wo0;
-    o[i][1] = o[i][1] * ws0 + t.y * wo0;
-    o[i][2] = o[i][2] * ws1 + t.z * wo1;
-    o[i][3] = o[i][3] * ws1 + t.w * wo1;
+template <int D>
+__device__ __forceinline__ void producer(const DecodeArgs& a, int u_begin, int u_end, uint32_t smem_base, Meta* meta, const Sync& sy,
+                                         const CUtensorMap* tm_k, const CUtensorMap* tm_v) {
+  const int lane = threadIdx.x & 31;
+  int issued = 0;  // stages issued so far (buffer = issued % NSTAGES)
+  // Table reads run ahead of their use so that no load sits on the issue path: the descriptor of unit u + 2,
+  // and the row list and first stage window of unit u + 1, are requested while unit u is being issued.
+  auto load_unit = [&](int u) {
+    UnitRegs w;
+    if (u < u_end) {
+      const int4* p = reinterpret_cast<const int4*>(a.units + u);
+      const int4 x = __ldg(p), y = __ldg(p + 1);
+      w.stage_begin = x.x; w.n_stages = x.y; w.row_begin = x.z; w.n_rows = x.w; w.kvh = y.x;
+    }
+    return w;
+  };
+  auto load_rows = [&](const UnitRegs& w, int base) {
+    return base + lane < w.n_rows ? a.item_rows[w.row_begin + base + lane] : mv::ItemRow{-1, -1};
+  };
+  auto load_window = [&](const UnitRegs& w, int first) {  // stages first + lane of the unit
+    StageRegs r;
+    if (first + lane < w.n_stages) {
+      const int4* p = reinterpret_cast<const int4*>(a.stages + w.stage_begin + first + lane);
+      r.a = __ldg(p);
+      r.b = __ldg(p + 1);
+    }
+    return r;
+  };
+  UnitRegs wu = load_unit(u_begin), wu1 = load_unit(u_begin + 1);
+  mv::ItemRow ir0 = load_rows(wu, 0), ir1 = load_rows(wu, 32);
+  StageRegs win = load_window(wu, 0);
+  for (int u = u_begin; u < u_end; ++u) {
+    const int ui = u - u_begin;
+    const UnitRegs wu2 = load_unit(u + 2);
+    const mv::ItemRow nir0 = load_rows(wu1, 0), nir1 = load_rows(wu1, 32);
+    const StageRegs nwin = load_window(wu1, 0);
+    // ---- q-vectors and partial-slot ids of this unit
+    const int n_qv = wu.n_rows * a.G;
+    const int n_pad = min(MAXQV, (n_qv + 15) & ~15);
+    if (lane == 0) wait_or_flag(sy, sy.q_empty, (ui & 1) ^ 1);
+    __syncwarp();
+    for (int x = lane; x < MAXQV; x += 32) {  // every lane takes part in the shuffles
+      const int r = min(x / a.G, MAXQV - 1);
+      const int p_lo = __shfl_sync(0xffffffffu, ir0.part, r & 31), p_hi = __shfl_sync(0xffffffffu, ir1.part, r & 31);
+      const int part = r < 32 ? p_lo : p_hi;
+      meta->pv[x] = (x < n_qv && part >= 0) ? part * a.G + x % a.G : -1;
+    }
+    if (lane == 0) {
+      meta->n_stages = wu.n_stages;
+      meta->n_qv = n_qv;
+    }
+    for (int i0 = 0; i0 < n_pad * Cfg<D>::CPR; i0 += 32) {  // n_pad * CPR is a multiple of 32
+      const int i = i0 + lane;
+      const int x = i / Cfg<D>::CPR, c = i % Cfg<D>::CPR;
+      const int r = min(x / a.G, MAXQV - 1);
+      const int r_lo = __shfl_sync(0xffffffffu, ir0.row, r & 31), r_hi = __shfl_sync(0xffffffffu, ir1.row, r & 31);
+      const int row = r < 32 ? r_lo : r_hi;
+      const bool ok = x < n_qv;
+      const bf16* src = a.q + (ok ? (int64_t(row) * a.Hq + wu.kvh * a.G + x % a.G) * D + c * 8 : 0);
+      mv::cp_async_16(smem_base + Cfg<D>::OFF_Q + q_off<D>(x, c), src, ok ? 16 : 0);  // padding rows are zero-filled
+    }
+    mv::cp_async_mbar_arrive_noinc(sy.q_full);  // 32 arrivals, each when the lane's copies have landed
+    __syncwarp();                               // the lanes' meta stores precede lane 0's releasing arrive
+    if (lane == 0) mv::mbar_arrive(sy.q_full);
+    // ---- KV stages, 32 descriptors per window
+    StageRegs nxt;
+    for (int s = 0; s < wu.n_stages; ++s) {
+      if ((s & 31) == 0) {
+        if (s > 0) win = nxt;
+        nxt = load_window(wu, s + 32);
+      }
+      const int src = s & 31;
+      const int4 da = make_int4(__shfl_sync(0xffffffffu, win.a.x, src), __shfl_sync(0xffffffffu, win.a.y, src),
+                                __shfl_sync(0xffffffffu, win.a.z, src), __shfl_sync(0xffffffffu, win.a.w, src));
+      const int n_tok = __shfl_sync(0xffffffffu, win.b.x, src);
+      const int m_lo = __shfl_sync(0xffffffffu, win.b.y, src), m_hi = __shfl_sync(0xffffffffu, win.b.z, src);
+      const int b = issued % NSTAGES;
+      const int n_pages = (n_tok + 15) >> 4;
+      const uint32_t bar = sy.full + 8 * b;
+      if (lane == 0) {
+        wait_or_flag(sy, sy.empty + 8 * b, ((issued / NSTAGES) & 1) ^ 1);  // every consumer warp has released the buffer
+        meta->st_tokens[b] = n_tok;
+        meta->st_mask_lo[b] = uint32_t(m_lo);
+        meta->st_mask_hi[b] = uint32_t(m_hi);
+        mv::mbar_arrive_expect_tx(bar, uint32_t(n_pages) * 16 * D * 2 * 2);  // releases the stores above
+      }
+      __syncwarp();
+      // lane j < 8: page j / 2 of the stage, K or V; one box = the whole contiguous (page, head) block
+      const int p = (lane >> 1) & 3, kv = lane & 1;
+      const int page = p == 0 ? da.x : p == 1 ? da.y : p == 2 ? da.z : da.w;
+      if (lane < 8 && p < n_pages) {
+        const int row = (page * a.Hkv + wu.kvh) * (16 * Cfg<D>::HALVES);
+        const uint32_t dst = smem_base + b * Cfg<D>::STAGE_BYTES + kv * Cfg<D>::KV_BYTES + p * Cfg<D>::PAGE_BYTES;
+        mv::tma_load_2d(dst, kv ? tm_v : tm_k, 0, row, bar);
+      }
+      ++issued;
+    }
+    wu = wu1;
+    wu1 = wu2;
+    ir0 = nir0;
+    ir1 = nir1;
+    win = nwin;
   }
 }
 
-// Consumes all stages of unit `cu` with MT m-tiles of 16 q-vectors; warp w: m-tile (w % MT), kv split (w / MT).
+// ---- consumer side ---------------------------------------------------------------------------------------
+// Consumes all stages of one unit with MT m-tiles of 16 q-vectors; warp w: m-tile (w % MT), kv split (w / MT).
 template <int D, int MT>
-__device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu, const Unit& nu, Loader<D>& ld, int& consumed,
-                                             unsigned char* smem, uint32_t smem_base, const Sync& sy, const CUtensorMap* tm_k,
-                                             const CUtensorMap* tm_v, int32_t pending, int32_t* s_next) {
+__device__ __forceinline__ void consume_unit(const DecodeArgs& a, int n_stages, int pv0, int pv1, int row0, int row1, uint64_t tile_rows,
+                                             const uint32_t (&qf)[D / 16][4], int& consumed, unsigned char* smem, uint32_t smem_base,
+                                             Meta* meta, const Sync& sy) {
   constexpr int KS = 4 / MT;      // kv splits inside a stage
   constexpr int WT = ST / KS;     // tokens per warp per stage
   constexpr int NT = WT / 8;      // S n-tiles per warp
@@ -175,54 +227,24 @@ __device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu
   constexpr int DT = D / 8;       // O n-tiles
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int mt = warp % MT, ks = warp / MT;
-  const int nqv = cu.n_rows * a.G;
-
-  // ---- this thread's two q rows, straight from global memory into the A-fragment layout
-  uint32_t qf[KSTEPS][4];
-  int part0 = -1, part1 = -1;  // partial slot (x Hq + head) of the two rows, -1 = padding row
-  {
-    const int x0 = mt * 16 + (lane >> 2), x1 = x0 + 8;
-    const uint32_t* p0 = nullptr;
-    const uint32_t* p1 = nullptr;
-    if (x0 < nqv) {
-      const mv::ItemRow ir = a.item_rows[cu.row_begin + x0 / a.G];
-      const int head = cu.kvh * a.G + x0 % a.G;
-      p0 = reinterpret_cast<const uint32_t*>(a.q + (int64_t(ir.row) * a.Hq + head) * D) + (lane & 3);
-      part0 = ir.part * a.Hq + head;
-    }
-    if (x1 < nqv) {
-      const mv::ItemRow ir = a.item_rows[cu.row_begin + x1 / a.G];
-      const int head = cu.kvh * a.G + x1 % a.G;
-      p1 = reinterpret_cast<const uint32_t*>(a.q + (int64_t(ir.row) * a.Hq + head) * D) + (lane & 3);
-      part1 = ir.part * a.Hq + head;
-    }
-#pragma unroll
-    for (int kk = 0; kk < KSTEPS; ++kk) {
-      qf[kk][0] = p0 ? __ldg(p0 + kk * 8) : 0u;
-      qf[kk][1] = p1 ? __ldg(p1 + kk * 8) : 0u;
-      qf[kk][2] = p0 ? __ldg(p0 + kk * 8 + 4) : 0u;
-      qf[kk][3] = p1 ? __ldg(p1 + kk * 8 + 4) : 0u;
-    }
-  }
+  (void)mt;
 
   float oacc[DT][4];
 #pragma unroll
   for (int i = 0; i < DT; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // rows lane/4 and lane/4 + 8 of the m-tile
   const int tok_w = ks * WT;                                  // first token of this warp inside a stage
+  int b = 0;
 
-  for (int s = 0; s < cu.n_stages; ++s) {
-    if (tid == 0) {
-      ld.top_up(a, cu, nu, smem_base, sy, tm_k, tm_v, consumed);
-      if (s == 0) *s_next = pending;  // unit after `nu`; read by everyone after this unit's epilogue
-    }
-    const int b = consumed % NSTAGES;
+  for (int s = 0; s < n_stages; ++s) {
+    b = consumed % NSTAGES;
     wait_or_flag(sy, sy.full + 8 * b, (consumed / NSTAGES) & 1);
     const uint32_t kb = smem_base + b * Cfg<D>::STAGE_BYTES, vb = kb + Cfg<D>::KV_BYTES;
     ++consumed;
-    const bool last = (s == cu.n_stages - 1);
-    const int tok_lim = cu.n_tokens - (s * ST + tok_w);  // valid tokens of this warp's slice
-    if (tok_lim > 0) {                                   // warp-uniform
+    const bool last = (s == n_stages - 1);
+    const int tok_lim = meta->st_tokens[b] - tok_w;  // valid tokens of this warp's slice
+    const uint64_t seen_by = (uint64_t(meta->st_mask_hi[b]) << 32) | meta->st_mask_lo[b];  // rows that see the stage's node
+    if (tok_lim > 0 && (seen_by & tile_rows) != 0) {  // warp-uniform: some row of this m-tile sees the stage
       if (tok_lim < WT) {
         // ragged end of the node: rows past the last token hold whatever the page (or an older stage) left
         // there; V must be zero where P is zero, or 0 * NaN would poison the output
@@ -249,7 +271,7 @@ __device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu
       }
       // scale to log2 units, mask the ragged tail, online softmax
       float mx0 = -INFINITY, mx1 = -INFINITY;
-      if (tok_lim >= WT) {
+      if (tok_lim >= WT && (seen_by & tile_rows) == tile_rows) {  // every row of the m-tile sees every token
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
@@ -257,13 +279,14 @@ __device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu
           mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
           mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
         }
-      } else {
+      } else {  // the DAG mask (a row that does not see the node) and the ragged end of the node
+        const bool vis0 = row0 >= 0 && ((seen_by >> row0) & 1), vis1 = row1 >= 0 && ((seen_by >> row1) & 1);
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
-            sacc[nt][e] = (col < tok_lim) ? sacc[nt][e] * a.scale_log2 : -INFINITY;
+            sacc[nt][e] = (col < tok_lim && (e < 2 ? vis0 : vis1)) ? sacc[nt][e] * a.scale_log2 : -INFINITY;
           }
           mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
           mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
@@ -273,10 +296,10 @@ __device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu
       mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
       mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
       mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-      const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);  // finite: column 0 of the slice is valid
+      const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);  // still -inf for a row that has seen nothing yet
       const bool grow = (mn0 > m0) || (mn1 > m1);
       if (__any_sync(0xffffffffu, grow)) {  // rescale only when some row's maximum moved
-        const float al0 = mv::fast_exp2(m0 - mn0), al1 = mv::fast_exp2(m1 - mn1);
+        const float al0 = mv::fast_exp2(m0 - (mn0 == -INFINITY ? 0.f : mn0)), al1 = mv::fast_exp2(m1 - (mn1 == -INFINITY ? 0.f : mn1));
         l0 *= al0;
         l1 *= al1;
 #pragma unroll
@@ -287,12 +310,13 @@ __device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu
         m0 = mn0;
         m1 = mn1;
       }
+      const float e0 = (m0 == -INFINITY) ? 0.f : m0, e1 = (m1 == -INFINITY) ? 0.f : m1;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        sacc[nt][0] = mv::fast_exp2(sacc[nt][0] - m0);
-        sacc[nt][1] = mv::fast_exp2(sacc[nt][1] - m0);
-        sacc[nt][2] = mv::fast_exp2(sacc[nt][2] - m1);
-        sacc[nt][3] = mv::fast_exp2(sacc[nt][3] - m1);
+        sacc[nt][0] = mv::fast_exp2(sacc[nt][0] - e0);
+        sacc[nt][1] = mv::fast_exp2(sacc[nt][1] - e0);
+        sacc[nt][2] = mv::fast_exp2(sacc[nt][2] - e1);
+        sacc[nt][3] = mv::fast_exp2(sacc[nt][3] - e1);
         l0 += sacc[nt][0] + sacc[nt][1];  // per-thread partial sums; reduced over the quad at the end
         l1 += sacc[nt][2] + sacc[nt][3];
       }
@@ -314,148 +338,175 @@ __device__ __forceinline__ void process_unit(const DecodeArgs& a, const Unit& cu
         }
       }
     }
-    if (!last) {  // hand the stage back; the unit's last stage is kept as scratch for the epilogue
+    if (!last || KS == 1) {  // hand the stage back; with kv splits the unit's last stage is kept as epilogue scratch
+      if (last) mv::fence_proxy_async();  // a ragged stage was patched with ordinary stores; TMA refills it next
       __syncwarp();
       if (lane == 0) mv::mbar_arrive(sy.empty + 8 * b);
     }
   }
 
-  // ---- epilogue: combine the KS kv-splits through the stage buffer that was consumed last, then write one
-  // partial per q-vector
-  const int b_last = (consumed - 1) % NSTAGES;
-  if (KS > 1) {
-    float4* sc_o = reinterpret_cast<float4*>(smem + b_last * Cfg<D>::STAGE_BYTES);  // [2][DT][32]
-    float4* sc_ml = sc_o + 2 * DT * 32;                                             // [2][32]
-    __syncthreads();  // everyone has finished reading the last stage
-    if (KS == 4) {
-      if (warp >= 2) {
-        float4* so = sc_o + (warp - 2) * DT * 32;
-#pragma unroll
-        for (int i = 0; i < DT; ++i) so[i * 32 + lane] = make_float4(oacc[i][0], oacc[i][1], oacc[i][2], oacc[i][3]);
-        sc_ml[(warp - 2) * 32 + lane] = make_float4(m0, m1, l0, l1);
-      }
-      __syncthreads();
-      if (warp < 2) merge_frag<DT>(m0, m1, l0, l1, oacc, sc_ml[warp * 32 + lane], sc_o + warp * DT * 32, lane);
-      __syncthreads();
-      if (warp == 1) {
-#pragma unroll
-        for (int i = 0; i < DT; ++i) sc_o[i * 32 + lane] = make_float4(oacc[i][0], oacc[i][1], oacc[i][2], oacc[i][3]);
-        sc_ml[lane] = make_float4(m0, m1, l0, l1);
-      }
-      __syncthreads();
-      if (warp == 0) merge_frag<DT>(m0, m1, l0, l1, oacc, sc_ml[lane], sc_o, lane);
-    } else {  // KS == 2: warps 2,3 hand their state to warps 0,1 (same m-tile)
-      if (ks == 1) {
-        float4* so = sc_o + mt * DT * 32;
-#pragma unroll
-        for (int i = 0; i < DT; ++i) so[i * 32 + lane] = make_float4(oacc[i][0], oacc[i][1], oacc[i][2], oacc[i][3]);
-        sc_ml[mt * 32 + lane] = make_float4(m0, m1, l0, l1);
-      }
-      __syncthreads();
-      if (ks == 0) merge_frag<DT>(m0, m1, l0, l1, oacc, sc_ml[mt * 32 + lane], sc_o + mt * DT * 32, lane);
-    }
-    mv::fence_proxy_async();  // the scratch writes precede the TMA refill of this buffer
-  }
-  __syncwarp();
-  if (lane == 0) mv::mbar_arrive(sy.empty + 8 * b_last);
-  if (ks == 0) {
+  // ---- epilogue: one partial (m, l, unnormalised o) per q-vector
+  const int c0 = (lane & 3) * 2;
+  if (KS == 1) {
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
     l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-    const int c0 = (lane & 3) * 2;
-    if (part0 >= 0) {
-      float* po = a.part_o + int64_t(part0) * D + c0;
+    if (pv0 >= 0) {
+      float* po = a.part_o + int64_t(pv0) * D + c0;
 #pragma unroll
       for (int i = 0; i < DT; ++i) *reinterpret_cast<float2*>(po + i * 8) = make_float2(oacc[i][0], oacc[i][1]);
-      if ((lane & 3) == 0) *reinterpret_cast<float2*>(a.part_ml + int64_t(part0) * 2) = make_float2(m0, l0);
+      if ((lane & 3) == 0) *reinterpret_cast<float2*>(a.part_ml + int64_t(pv0) * 2) = make_float2(m0, l0);
     }
-    if (part1 >= 0) {
-      float* po = a.part_o + int64_t(part1) * D + c0;
+    if (pv1 >= 0) {
+      float* po = a.part_o + int64_t(pv1) * D + c0;
 #pragma unroll
       for (int i = 0; i < DT; ++i) *reinterpret_cast<float2*>(po + i * 8) = make_float2(oacc[i][2], oacc[i][3]);
-      if ((lane & 3) == 0) *reinterpret_cast<float2*>(a.part_ml + int64_t(part1) * 2) = make_float2(m1, l1);
+      if ((lane & 3) == 0) *reinterpret_cast<float2*>(a.part_ml + int64_t(pv1) * 2) = make_float2(m1, l1);
+    }
+    return;
+  }
+  // The KS warps of an m-tile combine their states through the stage buffer that was consumed last
+  // ([warp][n-tile][lane] float4, exactly one stage); each of them then finishes and stores DT / KS n-tiles.
+  float4* sc_o = reinterpret_cast<float4*>(smem + b * Cfg<D>::STAGE_BYTES);
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  mv::named_bar_sync(1, NCONS);  // every consumer has finished reading the last stage
+#pragma unroll
+  for (int i = 0; i < DT; ++i) sc_o[(warp * DT + i) * 32 + lane] = make_float4(oacc[i][0], oacc[i][1], oacc[i][2], oacc[i][3]);
+  if ((lane & 3) == 0) {
+    meta->ml[warp][lane >> 2] = make_float2(m0, l0);
+    meta->ml[warp][(lane >> 2) + 8] = make_float2(m1, l1);
+  }
+  mv::named_bar_sync(1, NCONS);
+  float w0[KS], w1[KS];
+  float mm0 = -INFINITY, mm1 = -INFINITY;
+#pragma unroll
+  for (int k = 0; k < KS; ++k) {
+    mm0 = fmaxf(mm0, meta->ml[mt + MT * k][lane >> 2].x);
+    mm1 = fmaxf(mm1, meta->ml[mt + MT * k][(lane >> 2) + 8].x);
+  }
+  float ll0 = 0.f, ll1 = 0.f;
+#pragma unroll
+  for (int k = 0; k < KS; ++k) {
+    const float2 t0 = meta->ml[mt + MT * k][lane >> 2], t1 = meta->ml[mt + MT * k][(lane >> 2) + 8];
+    w0[k] = (t0.x == -INFINITY) ? 0.f : mv::fast_exp2(t0.x - mm0);
+    w1[k] = (t1.x == -INFINITY) ? 0.f : mv::fast_exp2(t1.x - mm1);
+    ll0 += w0[k] * t0.y;
+    ll1 += w1[k] * t1.y;
+  }
+  constexpr int IPW = DT / KS;  // n-tiles this warp finishes
+#pragma unroll
+  for (int ii = 0; ii < IPW; ++ii) {
+    const int i = ks * IPW + ii;
+    float r0 = 0.f, r1 = 0.f, r2 = 0.f, r3 = 0.f;
+#pragma unroll
+    for (int k = 0; k < KS; ++k) {
+      const float4 t = sc_o[((mt + MT * k) * DT + i) * 32 + lane];
+      r0 += w0[k] * t.x; r1 += w0[k] * t.y;
+      r2 += w1[k] * t.z; r3 += w1[k] * t.w;
+    }
+    if (pv0 >= 0) *reinterpret_cast<float2*>(a.part_o + int64_t(pv0) * D + i * 8 + c0) = make_float2(r0, r1);
+    if (pv1 >= 0) *reinterpret_cast<float2*>(a.part_o + int64_t(pv1) * D + i * 8 + c0) = make_float2(r2, r3);
+  }
+  if (ks == 0) {
+    if ((lane & 3) == 0) {
+      if (pv0 >= 0) *reinterpret_cast<float2*>(a.part_ml + int64_t(pv0) * 2) = make_float2(mm0, ll0);
+      if (pv1 >= 0) *reinterpret_cast<float2*>(a.part_ml + int64_t(pv1) * 2) = make_float2(mm1, ll1);
     }
   }
+  mv::fence_proxy_async();  // the scratch accesses precede the TMA refill of this buffer
+  __syncwarp();
+  if (lane == 0) mv::mbar_arrive(sy.empty + 8 * b);
+}
+
+template <int D, int MT>
+__device__ __forceinline__ void consumer_unit(const DecodeArgs& a, int n_stages, int n_qv, int& consumed, unsigned char* smem,
+                                              uint32_t smem_base, Meta* meta, const Sync& sy) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int mt = warp % MT;
+  // this thread's two q rows of the m-tile, their partial slots and their rows of the row group
+  const int x0 = mt * 16 + (lane >> 2), x1 = x0 + 8;
+  const int pv0 = meta->pv[x0], pv1 = meta->pv[x1];
+  const int row0 = x0 < n_qv ? x0 / a.G : -1, row1 = x1 < n_qv ? x1 / a.G : -1;
+  uint64_t tile_rows = 0;  // rows of the row group that own a q-vector of this m-tile
+  if (mt * 16 < n_qv) {
+    const int r_lo = (mt * 16) / a.G, r_hi = (min(mt * 16 + 15, n_qv - 1)) / a.G;
+    tile_rows = (r_hi - r_lo == 63 ? ~uint64_t(0) : ((uint64_t(1) << (r_hi - r_lo + 1)) - 1)) << r_lo;
+  }
+  uint32_t qf[D / 16][4];
+#pragma unroll
+  for (int kk = 0; kk < D / 16; ++kk)
+    mv::ldmatrix_x4(qf[kk], smem_base + Cfg<D>::OFF_Q + q_off<D>(mt * 16 + (lane & 15), kk * 2 + (lane >> 4)));
+  __syncwarp();
+  if (lane == 0) mv::mbar_arrive(sy.q_empty);  // the unit's q buffer and header are free again
+  consume_unit<D, MT>(a, n_stages, pv0, pv1, row0, row1, tile_rows, qf, consumed, smem, smem_base, meta, sy);
 }
 
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, 2) decode_attn_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tm_k,
                                                                   const __grid_constant__ CUtensorMap tm_v) {
-  extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t s_bar[2 * NSTAGES];
-  __shared__ int32_t s_ids[3];
-  __shared__ int s_abort;
-  const int tid = threadIdx.x;
-  const uint32_t raw = mv::smem_u32(smem_raw);
-  const uint32_t smem_base = (raw + 1023u) & ~1023u;  // the swizzle pattern is anchored at 1024-byte boundaries
-  unsigned char* smem = smem_raw + (smem_base - raw);
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const uint32_t smem_base = mv::smem_u32(smem);
+  Meta* meta = reinterpret_cast<Meta*>(smem + Cfg<D>::OFF_META);
   Sync sy;
-  sy.full = mv::smem_u32(&s_bar[0]);
-  sy.empty = mv::smem_u32(&s_bar[NSTAGES]);
-  sy.abort = &s_abort;
-  sy.status = a.sched + 2;
+  sy.full = mv::smem_u32(&meta->full[0]);
+  sy.empty = mv::smem_u32(&meta->empty[0]);
+  sy.q_full = mv::smem_u32(&meta->q_full);
+  sy.q_empty = mv::smem_u32(&meta->q_empty);
+  sy.abort = &meta->abort;
+  sy.status = a.status;
+  if ((smem_base & 1023u) != 0) {  // the swizzle pattern is anchored at 1024-byte boundaries
+    if (tid == 0) atomicExch(a.status, int(MV_ERR_UNSUPPORTED));
+    return;
+  }
   if (tid == 0) {
-    s_abort = 0;
+    meta->abort = 0;
     for (int i = 0; i < NSTAGES; ++i) {
       mv::mbar_init(sy.full + 8 * i, 1);   // the producer's arrive (+ the bytes TMA reports)
       mv::mbar_init(sy.empty + 8 * i, 4);  // one arrive per consumer warp
     }
+    mv::mbar_init(sy.q_full, 33);   // 32 copy-completion arrivals + the producer's releasing arrive
+    mv::mbar_init(sy.q_empty, 4);   // one arrive per consumer warp
     mv::mbar_fence_init();
     mv::fence_proxy_async();
-    s_ids[0] = atomicAdd(a.sched, 1);
-    s_ids[1] = atomicAdd(a.sched, 1);
   }
   __syncthreads();
-  Unit cu = load_unit(a, s_ids[0]);
-  Unit nu = load_unit(a, s_ids[1]);
-  Loader<D> ld;
+  const int u_begin = a.cta_unit_off[blockIdx.x], u_end = a.cta_unit_off[blockIdx.x + 1];
+  if (warp == 4) {
+    producer<D>(a, u_begin, u_end, smem_base, meta, sy, &tm_k, &tm_v);
+    mv::grid_dependency_launch_dependents();
+    return;
+  }
   int consumed = 0;
-  if (tid == 0) {
-    ld.prefetch_pages(a, cu, nu);
-    ld.top_up(a, cu, nu, smem_base, sy, &tm_k, &tm_v, consumed);
+  for (int u = u_begin; u < u_end; ++u) {
+    wait_or_flag(sy, sy.q_full, (u - u_begin) & 1);
+    const int n_stages = meta->n_stages, n_qv = meta->n_qv;
+    if (n_qv <= 16) consumer_unit<D, 1>(a, n_stages, n_qv, consumed, smem, smem_base, meta, sy);
+    else if (n_qv <= 32) consumer_unit<D, 2>(a, n_stages, n_qv, consumed, smem, smem_base, meta, sy);
+    else consumer_unit<D, 4>(a, n_stages, n_qv, consumed, smem, smem_base, meta, sy);
   }
-  while (cu.n_stages > 0) {
-    int32_t pending = 0;
-    if (tid == 0) pending = atomicAdd(a.sched, 1);  // the unit after `nu`; published one stage later
-    const int nqv = cu.n_rows * a.G;
-    if (nqv <= 16) process_unit<D, 1>(a, cu, nu, ld, consumed, smem, smem_base, sy, &tm_k, &tm_v, pending, &s_ids[2]);
-    else if (nqv <= 32) process_unit<D, 2>(a, cu, nu, ld, consumed, smem, smem_base, sy, &tm_k, &tm_v, pending, &s_ids[2]);
-    else process_unit<D, 4>(a, cu, nu, ld, consumed, smem, smem_base, sy, &tm_k, &tm_v, pending, &s_ids[2]);
-    __syncthreads();  // s_ids[2] is visible to everyone
-    cu = nu;
-    nu = load_unit(a, s_ids[2]);
-    __syncthreads();  // s_ids[2] may be overwritten from here on
-    if (tid == 0) {
-      // the loader had finished the old `cu` (it was consumed), so it stands in the old `nu` or beyond it
-      ld.which -= 1;
-      if (ld.which == 1) ld.prefetch_pages(a, cu, nu);  // it was beyond: it now stands at the first stage of the new `nu`
-      ld.top_up(a, cu, nu, smem_base, sy, &tm_k, &tm_v, consumed);
-    }
-  }
-  // every stage that was issued has been consumed (the loader never runs past `nu`, and `nu` is empty here)
-  if (tid == 0) {
-    __threadfence();
-    const int done = atomicAdd(a.sched + 1, 1);
-    if (done == int(gridDim.x) - 1) {  // the last CTA to finish re-arms the scheduler words for the next launch
-      a.sched[0] = 0;
-      a.sched[1] = 0;
-      __threadfence();
-    }
-  }
+  // this CTA's share is done: once every CTA got here (or exited) the merge kernel may become resident, so its
+  // launch overlaps the tail of this grid; it still waits for the grid's completion before it reads a partial
+  mv::grid_dependency_launch_dependents();
 }
 
 // Merge of the split-KV partials of one (row, head): one warp each.
 template <int D>
 __global__ void __launch_bounds__(128) decode_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                                           const int32_t* __restrict__ row_part_off, bf16* __restrict__ out,
-                                                           int n_rows, int Hq) {
+                                                           const int32_t* __restrict__ rowkv_part_off, bf16* __restrict__ out,
+                                                           int n_rows, int Hq, int G) {
   const int w = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (w >= n_rows * Hq) return;
-  const int row = w / Hq, h = w % Hq;
-  const int p0 = row_part_off[row], p1 = row_part_off[row + 1];
+  const int row = w / Hq, h = w % Hq, kvh = h / G, g = h % G;
+  const int Hkv = Hq / G;
+  const int p0 = rowkv_part_off[row * Hkv + kvh], p1 = rowkv_part_off[row * Hkv + kvh + 1];
+  mv::grid_dependency_wait();  // the partials are complete and visible from here on
   float m = -INFINITY;
-  for (int p = p0 + lane; p < p1; p += 32) m = fmaxf(m, part_ml[(int64_t(p) * Hq + h) * 2]);
+  for (int p = p0 + lane; p < p1; p += 32) m = fmaxf(m, part_ml[(int64_t(p) * G + g) * 2]);
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
   constexpr int E = D / 32;
@@ -463,8 +514,9 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const float* __restri
 #pragma unroll
   for (int e = 0; e < E; ++e) acc[e] = 0.f;
   float l = 0.f;
+#pragma unroll 4
   for (int p = p0; p < p1; ++p) {
-    const int64_t ps = int64_t(p) * Hq + h;
+    const int64_t ps = int64_t(p) * G + g;
     const float2 ml = *reinterpret_cast<const float2*>(part_ml + ps * 2);
     const float wgt = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m);
     l += wgt * ml.y;
@@ -483,19 +535,7 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const float* __restri
   for (int e = 0; e < E; e += 2) *reinterpret_cast<__nv_bfloat162*>(o + e) = __floats2bfloat162_rn(acc[e] * inv, acc[e + 1] * inv);
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
-      (void)cudaGetLastError();
-      n = 148;
-    }
-  }
-  return n;
-}
-
-struct TmapCache {  // the pools rarely change between calls: keep the last pair of tensor maps
+struct TmapCache {  // the pools rarely change between calls: keep the last pairs of tensor maps
   const void* k = nullptr;
   const void* v = nullptr;
   int64_t rows = 0;
@@ -516,7 +556,7 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
   }
   static thread_local TmapCache tc[4];
   static thread_local int tc_next = 0;
-  const int64_t rows = g->num_pages * g->n_kv_heads * 16;
+  const int64_t rows = g->num_pages * g->n_kv_heads * 16 * Cfg<D>::HALVES;  // 128-byte rows of the pool
   TmapCache* hit = nullptr;
   for (auto& c : tc)
     if (c.k == kp && c.v == vp && c.rows == rows && c.d == D) hit = &c;
@@ -524,35 +564,53 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
     hit = &tc[tc_next];
     tc_next = (tc_next + 1) % 4;
     hit->k = nullptr;
-    if (!mv::make_tmap_bf16_2d(&hit->tm_k, kp, uint64_t(rows), D, 16) || !mv::make_tmap_bf16_2d(&hit->tm_v, vp, uint64_t(rows), D, 16))
+    if (!mv::make_tmap_bf16_2d(&hit->tm_k, kp, uint64_t(rows), 64, 16 * Cfg<D>::HALVES) ||
+        !mv::make_tmap_bf16_2d(&hit->tm_v, vp, uint64_t(rows), 64, 16 * Cfg<D>::HALVES))
       return MV_ERR_CUDA;
     hit->k = kp; hit->v = vp; hit->rows = rows; hit->d = D;
   }
-  const size_t parts = size_t(P->stats.n_partials);
-  const size_t o_bytes = (parts * g->n_q_heads * D * sizeof(float) + 255) & ~size_t(255);
+  const int G = g->n_q_heads / g->n_kv_heads;
+  const size_t vecs = size_t(P->stats.n_partials) * size_t(G);
+  const size_t o_bytes = (vecs * D * sizeof(float) + 255) & ~size_t(255);
   DecodeArgs a;
   a.q = static_cast<const bf16*>(q);
-  a.page_idx = mv::table<int32_t>(P, P->layout.page_idx);
-  a.items = mv::table<mv::WorkItem>(P, P->layout.items);
+  a.stages = mv::table<mv::StageDesc>(P, P->layout.stages);
+  a.units = mv::table<mv::WorkUnit>(P, P->layout.units);
+  a.cta_unit_off = mv::table<int32_t>(P, P->layout.cta_unit_off);
   a.item_rows = mv::table<mv::ItemRow>(P, P->layout.item_rows);
   a.part_o = static_cast<float*>(ws);
   a.part_ml = reinterpret_cast<float*>(static_cast<char*>(ws) + o_bytes);
-  a.sched = const_cast<int32_t*>(mv::table<int32_t>(P, P->layout.sched));
+  a.status = const_cast<int32_t*>(mv::table<int32_t>(P, P->layout.sched)) + 2;
   a.Hq = g->n_q_heads;
-  a.Hkv = g->n_kv_heads;
-  a.G = g->n_q_heads / g->n_kv_heads;
-  a.n_units = int(P->stats.n_items) * g->n_kv_heads;
+  a.G = G;
   a.scale_log2 = mv::softmax_scale(g) * 1.4426950408889634f;
-  const int grid = std::min(a.n_units, 2 * sm_count());
-  decode_attn_kernel<D><<<grid, NTHREADS, Cfg<D>::SMEM, st>>>(a, hit->tm_k, hit->tm_v);
+  a.Hkv = g->n_kv_heads;
+  decode_attn_kernel<D><<<unsigned(P->stats.n_ctas), NTHREADS, Cfg<D>::SMEM, st>>>(a, hit->tm_k, hit->tm_v);
   mv::g_launches++;
   if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
+  // the merge kernel is launched with programmatic stream serialisation: it may become resident while the
+  // attention kernel is still running and waits (griddepcontrol.wait) for that grid to complete
   const int n_rows = int(P->stats.n_new_tokens);
   const int n_warps = n_rows * g->n_q_heads;
-  decode_merge_kernel<D><<<(n_warps + 3) / 4, 128, 0, st>>>(a.part_o, a.part_ml, mv::table<int32_t>(P, P->layout.row_part_off),
-                                                           static_cast<bf16*>(out), n_rows, g->n_q_heads);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(unsigned((n_warps + 3) / 4), 1, 1);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, decode_merge_kernel<D>, static_cast<const float*>(a.part_o),
+                                           static_cast<const float*>(a.part_ml), mv::table<int32_t>(P, P->layout.rowkv_part_off),
+                                           static_cast<bf16*>(out), n_rows, int(g->n_q_heads), G);
   mv::g_launches++;
-  return cudaGetLastError() == cudaSuccess ? MV_OK : MV_ERR_CUDA;
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return MV_ERR_CUDA;
+  }
+  return MV_OK;
 }
 
 }  // namespace
@@ -565,9 +623,11 @@ extern "C" mv_status mv_dag_decode_attn(const mv_plan* P, const mv_attn_geom* g,
   if (st != MV_OK) return st;
   if (P->stats.n_new_tokens == 0) return MV_OK;
   if (g->dtype != MV_BF16 || !P->stats.decode_ready) return MV_ERR_UNSUPPORTED;
-  if (P->stats.max_item_rows * (g->n_q_heads / g->n_kv_heads) > 64) return MV_ERR_UNSUPPORTED;
   if (!q_rot || !k_pages || !v_pages || !out) return MV_ERR_INVALID_ARG;
   if (!P->device_buf) return MV_ERR_WORKSPACE;
+  // the work units were cut for one KV head count and one group size
+  if (g->n_kv_heads != P->stats.sched_kv_heads || g->n_q_heads / g->n_kv_heads != P->stats.sched_group) return MV_ERR_UNSUPPORTED;
+  if (P->stats.max_item_rows * P->stats.sched_group > MAXQV) return MV_ERR_UNSUPPORTED;
   if (P->stats.max_page_id >= g->num_pages) return MV_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(k_pages) & 15) || (reinterpret_cast<uintptr_t>(v_pages) & 15)) return MV_ERR_INVALID_ARG;
   const size_t need = mv_workspace_bytes(P, g, MV_OP_DECODE_ATTN);

@@ -12,16 +12,28 @@ namespace mv {
 constexpr int kPrefillQTile = 128;   // query rows per prefill tile (tiles never straddle a node)
 constexpr int kPrefillKvTile = 64;   // granularity used only for the executed-pairs statistic
 
-// One decode work item per KV head: a page-aligned chunk of one node's KV and the rows that see it.
-struct WorkItem {
-  int32_t page_begin;  // index into the uploaded page_idx array of the chunk's first page
-  int32_t n_tokens;    // valid tokens in the chunk (the last page may be partial)
-  int32_t row_begin;   // index into item_rows of the first (row, partial slot) pair
-  int32_t n_rows;      // rows (new tokens) whose visible set contains this chunk
+// Decode work lists.  A request's frontier rows (at most 64 / group_size of them per row group) and all the KV
+// they see form one stream of 64-token STAGES, node after node; a stage belongs to one node and carries the
+// set of rows that see that node.  A work unit is a run of consecutive stages for ONE KV head; units are
+// listed CTA by CTA (cta_unit_off): the planner cuts the step's whole stream into equal shares.
+struct StageDesc {
+  int32_t page[4];    // physical pages of the stage (unused entries repeat page[0])
+  int32_t n_tokens;   // valid tokens, 1..64 (the node's last stage may be ragged)
+  uint32_t mask_lo, mask_hi;  // bit r: row r of the unit's row group sees this stage
+  int32_t pad;
+};
+struct WorkUnit {
+  int32_t stage_begin;  // index into the stage table
+  int32_t n_stages;
+  int32_t row_begin;    // index into item_rows of the unit's first (row, partial slot) pair
+  int32_t n_rows;       // rows of the row group
+  int32_t kvh;          // KV head
+  int32_t pad[3];
 };
 struct ItemRow {
   int32_t row;   // row index = index of the new token
-  int32_t part;  // split-KV partial slot this (item, row) pair writes
+  int32_t part;  // split-KV partial slot this (unit, row) pair writes (a slot holds group_size head vectors),
+                 // or -1 if the row sees none of the unit's stages
 };
 // One prefill query tile: rows [q_start, q_start+q_len) of one node and the KV ranges they may see.
 struct QTile {
@@ -34,7 +46,7 @@ struct KvRange {
 };
 
 struct DeviceLayout {  // byte offsets into the device table buffer (all multiples of 256)
-  size_t pos_id = 0, slot = 0, page_idx = 0, items = 0, item_rows = 0, row_part_off = 0, sched = 0,
+  size_t pos_id = 0, slot = 0, stages = 0, units = 0, cta_unit_off = 0, item_rows = 0, rowkv_part_off = 0, sched = 0,
          q_tiles = 0, kv_ranges = 0, total = 0;
 };
 
@@ -45,11 +57,12 @@ struct mv_plan {
   std::vector<int32_t> layer, pos_start, pos_id, qnode, qnode_tok_off, seg_off, seg_node, seg_len;
   std::vector<int64_t> slot, kv_len;
   // kernel tables
-  std::vector<int32_t> page_idx;
-  std::vector<mv::WorkItem> items;
+  std::vector<mv::StageDesc> stages;
+  std::vector<mv::WorkUnit> units;       // CTA by CTA
+  std::vector<int32_t> cta_unit_off;     // [n_ctas + 1]
   std::vector<mv::ItemRow> item_rows;
-  std::vector<int32_t> row_part_off;
-  int32_t sched_zero[64] = {};  // device-side scheduler words (work counter, finished-CTA counter), uploaded as zeros
+  std::vector<int32_t> rowkv_part_off;   // [n_rows * n_kv_heads + 1] CSR over the partial slots of a (row, KV head)
+  int32_t sched_zero[64] = {};  // device-side status words ([2] = status of bounded waits), uploaded as zeros
   std::vector<mv::QTile> q_tiles;
   std::vector<mv::KvRange> kv_ranges;
   mv_plan_stats stats{};

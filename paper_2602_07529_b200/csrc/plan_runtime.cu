@@ -47,10 +47,11 @@ extern "C" mv_status mv_plan_upload(mv_plan* P, void* device_buf, size_t device_
   const mv::DeviceLayout& L = P->layout;
   put(h, L.pos_id, P->pos_id);
   put(h, L.slot, P->slot);
-  put(h, L.page_idx, P->page_idx);
-  put(h, L.items, P->items);
+  put(h, L.stages, P->stages);
+  put(h, L.units, P->units);
+  put(h, L.cta_unit_off, P->cta_unit_off);
   put(h, L.item_rows, P->item_rows);
-  put(h, L.row_part_off, P->row_part_off);
+  put(h, L.rowkv_part_off, P->rowkv_part_off);
   std::memcpy(h + L.sched, P->sched_zero, sizeof(P->sched_zero));
   put(h, L.q_tiles, P->q_tiles);
   put(h, L.kv_ranges, P->kv_ranges);
@@ -75,9 +76,9 @@ extern "C" void mv_plan_destroy(mv_plan* P) {
 extern "C" size_t mv_workspace_bytes(const mv_plan* P, const mv_attn_geom* g, int op) {
   if (!P || !P->valid || !g) return 0;
   if (op == MV_OP_DECODE_ATTN) {
-    const size_t parts = size_t(P->stats.n_partials);
-    const size_t o = (parts * g->n_q_heads * g->head_dim * sizeof(float) + 255) & ~size_t(255);
-    const size_t ml = (parts * g->n_q_heads * 2 * sizeof(float) + 255) & ~size_t(255);
+    const size_t vecs = size_t(P->stats.n_partials) * size_t(P->stats.sched_group);  // one per (partial, head of the group)
+    const size_t o = (vecs * g->head_dim * sizeof(float) + 255) & ~size_t(255);
+    const size_t ml = (vecs * 2 * sizeof(float) + 255) & ~size_t(255);
     return o + ml + 256;
   }
   return 0;

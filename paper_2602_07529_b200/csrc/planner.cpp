@@ -18,7 +18,8 @@ namespace {
 using mv::ItemRow;
 using mv::KvRange;
 using mv::QTile;
-using mv::WorkItem;
+using mv::StageDesc;
+using mv::WorkUnit;
 
 struct Bits {  // dense bitset rows, n_words per node
   int n_words = 0;
@@ -42,7 +43,7 @@ mv_status check_batch(const mv_dag_batch* b) {
   if (b->vis_mode != MV_VIS_ANCESTORS && b->vis_mode != MV_VIS_LAYERWISE) return MV_ERR_INVALID_ARG;
   if (b->pos_mode != MV_POS_MAX_PARENT_END && b->pos_mode != MV_POS_FRONTIER_ALIGNED) return MV_ERR_INVALID_ARG;
   if (b->chunk_tokens < 0 || (b->chunk_tokens % b->page_size) != 0) return MV_ERR_INVALID_ARG;
-  if (b->n_kv_heads < 0 || b->group_size < 0) return MV_ERR_INVALID_ARG;
+  if (b->n_kv_heads < 0 || b->group_size < 0 || b->sched_ctas < 0) return MV_ERR_INVALID_ARG;
   if (b->node_off[0] != 0) return MV_ERR_INVALID_ARG;
   for (int r = 0; r < b->n_req; ++r)
     if (b->node_off[r + 1] < b->node_off[r]) return MV_ERR_INVALID_ARG;
@@ -103,9 +104,9 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   P->qnode_tok_off.assign(1, 0);
   P->seg_off.assign(1, 0);
   P->seg_node.clear(); P->seg_len.clear(); P->kv_len.clear();
-  P->items.clear(); P->item_rows.clear(); P->row_part_off.clear();
+  P->units.clear(); P->cta_unit_off.clear(); P->item_rows.clear(); P->rowkv_part_off.clear();
   P->q_tiles.clear(); P->kv_ranges.clear();
-  P->page_idx.assign(b->page_idx, b->page_idx + (n_nodes ? b->page_off[n_nodes] : 0));
+  P->stages.clear();
   mv_plan_stats S{};
   S.n_nodes = n_nodes;
   S.max_page_id = max_page;
@@ -122,30 +123,17 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   std::vector<int64_t> node_tok_start(n_nodes, 0);  // flattened index of a node's first NEW token
   std::vector<std::vector<int32_t>> rows_of_node;    // decode: rows that see each node (request local)
   int64_t unique_tokens = 0, per_row_tokens = 0, visible_pairs = 0, tile_pairs = 0;
-  std::vector<int32_t> row_parts;  // per row: number of partials
-  std::vector<int32_t> flat_rows;  // (row, local partial index) pairs of every item, in item creation order
   const int sched_kv_heads = b->n_kv_heads > 0 ? b->n_kv_heads : 8;
   const int sched_group = b->group_size > 0 ? b->group_size : 8;
   const int max_rows_per_item = std::max(1, 64 / sched_group);
 
-  // automatic chunk length: aim for a few work items per CTA slot, assuming 8 KV heads
-  int chunk = b->chunk_tokens;
-  if (chunk == 0 && decode_ready) {
-    int64_t total_unique = 0;
-    for (int r = 0; r < b->n_req; ++r) {
-      // cheap upper bound: all nodes with tokens in requests that have a frontier
-      const int lo = b->node_off[r], hi = b->node_off[r + 1];
-      bool has_new = false;
-      for (int g = lo; g < hi; ++g) has_new |= b->node_new[g] > 0;
-      if (!has_new) continue;
-      for (int g = lo; g < hi; ++g) total_unique += b->node_len[g] + b->node_new[g];
-    }
-    int64_t c = (total_unique * sched_kv_heads) / (148 * 2 * 6);
-    c = ((c + 63) / 64) * 64;
-    chunk = int(std::min<int64_t>(1024, std::max<int64_t>(256, c)));
-  }
-  if (chunk == 0) chunk = 256;
-  S.chunk_tokens = chunk;
+  // decode streams: one per (request, row group): a run of stages and the rows of the group; cut into work
+  // units after pass 1
+  struct Seg { int32_t stage_begin, n_stages, rows_begin, n_rows; };
+  std::vector<Seg> segs;
+  std::vector<int32_t> seg_rows;
+  constexpr int kStage = 64;  // tokens per stage of the decode kernel's pipeline
+  const int chunk = b->chunk_tokens;  // 0: units are cut only where a CTA's share ends
 
   int64_t new_tok_count = 0;
   for (int r = 0; r < b->n_req; ++r) {
@@ -204,7 +192,6 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       }
     }
     // canonical per-token and per-q-node tables
-    const int64_t first_row_of_req = new_tok_count;
     rows_of_node.assign(n, {});
     std::vector<char> seen_by_frontier(n, 0);
     for (int v = 0; v < n; ++v) {
@@ -237,36 +224,42 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     for (int u = 0; u < n; ++u)
       if (seen_by_frontier[u]) unique_tokens += b->node_len[lo + u] + b->node_new[lo + u];
 
-    // ---- decode work items of this request: (node chunk) x (rows that see the node)
+    // ---- decode streams of this request: per row group, the stages of every node at least one of its rows sees
     if (decode_ready) {
-      const int64_t n_rows_req = new_tok_count - first_row_of_req;
-      row_parts.resize(size_t(new_tok_count), 0);
-      (void)n_rows_req;
-      for (int u = 0; u < n; ++u) {
-        const auto& rows = rows_of_node[u];
-        const int32_t L = b->node_len[lo + u] + b->node_new[lo + u];
-        if (rows.empty() || L == 0) continue;
-        const int n_pages = (L + ps - 1) / ps;
-        const int n_chunks = (L + chunk - 1) / chunk;
-        const int pages_per_chunk = (n_pages + n_chunks - 1) / n_chunks;
-        for (int c = 0; c * pages_per_chunk < n_pages; ++c) {
-          const int pb = c * pages_per_chunk;
-          const int pe = std::min(n_pages, pb + pages_per_chunk);
-          // a row set larger than one tensor-core pass (64 q-vectors) is split; each part re-reads the chunk
-          for (size_t r0 = 0; r0 < rows.size(); r0 += size_t(max_rows_per_item)) {
-            const size_t r1 = std::min(rows.size(), r0 + size_t(max_rows_per_item));
-            WorkItem it;
-            it.page_begin = b->page_off[lo + u] + pb;
-            it.n_tokens = std::min(L, pe * ps) - pb * ps;
-            it.row_begin = int32_t(flat_rows.size() / 2);
-            it.n_rows = int32_t(r1 - r0);
-            P->items.push_back(it);
-            for (size_t k = r0; k < r1; ++k) {
-              flat_rows.push_back(rows[k]);
-              flat_rows.push_back(row_parts[rows[k]]++);  // partial index local to the row, made global below
+      std::vector<int32_t> req_rows;  // rows of the request, ascending (one per frontier node)
+      std::vector<int32_t> row_node;  // local node of each row
+      for (int v = 0; v < n; ++v)
+        if (b->node_new[lo + v] > 0) {
+          req_rows.push_back(int32_t(node_tok_start[lo + v]));
+          row_node.push_back(v);
+        }
+      for (size_t r0 = 0; r0 < req_rows.size(); r0 += size_t(max_rows_per_item)) {
+        const size_t r1 = std::min(req_rows.size(), r0 + size_t(max_rows_per_item));
+        Seg sg{int32_t(P->stages.size()), 0, int32_t(seg_rows.size()), int32_t(r1 - r0)};
+        for (int u = 0; u < n; ++u) {
+          const int32_t L = b->node_len[lo + u] + b->node_new[lo + u];
+          if (L == 0) continue;
+          uint64_t mask = 0;
+          for (size_t k = r0; k < r1; ++k)
+            if (vis.get(row_node[k], u)) mask |= uint64_t(1) << (k - r0);
+          if (mask == 0) continue;
+          const int32_t* pages = b->page_idx + b->page_off[lo + u];
+          const int n_pages = (L + ps - 1) / ps;
+          for (int32_t t0 = 0; t0 < L; t0 += kStage) {
+            StageDesc sd{};
+            sd.n_tokens = std::min<int32_t>(kStage, L - t0);
+            for (int j = 0; j < 4; ++j) {
+              const int pi = t0 / ps + j;
+              sd.page[j] = pages[pi < n_pages ? pi : t0 / ps];
             }
+            sd.mask_lo = uint32_t(mask);
+            sd.mask_hi = uint32_t(mask >> 32);
+            P->stages.push_back(sd);
           }
         }
+        sg.n_stages = int32_t(P->stages.size()) - sg.stage_begin;
+        seg_rows.insert(seg_rows.end(), req_rows.begin() + r0, req_rows.begin() + r1);
+        if (sg.n_stages > 0) segs.push_back(sg);
       }
     }
 
@@ -322,33 +315,99 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     }
   }
 
-  // ---- decode: global partial slots, longest-first item order
+  // ---- decode: cut the stream of (row-group stream, KV head) stage runs into n_ctas shares of equal cost
   if (decode_ready) {
     const int64_t n_rows = new_tok_count;
-    row_parts.resize(size_t(n_rows), 0);
-    P->row_part_off.assign(size_t(n_rows) + 1, 0);
-    for (int64_t r = 0; r < n_rows; ++r) P->row_part_off[r + 1] = P->row_part_off[r] + row_parts[r];
-    std::vector<int32_t> order(P->items.size());
-    std::iota(order.begin(), order.end(), 0);
-    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t c) {
-      return P->items[a].n_tokens > P->items[c].n_tokens;
-    });
-    std::vector<WorkItem> sorted;
-    sorted.reserve(order.size());
-    for (int32_t i : order) {
-      WorkItem it = P->items[i];
-      const int32_t src = it.row_begin;
-      it.row_begin = int32_t(P->item_rows.size());
-      for (int32_t k = 0; k < it.n_rows; ++k) {
-        const int32_t row = flat_rows[2 * size_t(src + k)], local = flat_rows[2 * size_t(src + k) + 1];
-        P->item_rows.push_back(ItemRow{row, P->row_part_off[row] + local});
+    const int n_ctas = b->sched_ctas > 0 ? b->sched_ctas : 296;
+    constexpr int64_t kUnitOverhead = 96;  // fixed cost of a unit (q staging, epilogue), in token equivalents
+    constexpr int64_t kStageOverhead = 8;  // fixed cost of a stage (barrier round trip), in token equivalents
+    const int max_unit_stages = chunk > 0 ? std::max(1, chunk / kStage) : (1 << 30);
+    std::vector<int64_t> cost_prefix(P->stages.size() + 1, 0);  // running stage cost over the stage table
+    for (size_t i = 0; i < P->stages.size(); ++i) cost_prefix[i + 1] = cost_prefix[i] + P->stages[i].n_tokens + kStageOverhead;
+    int64_t remaining = 0;  // cost not yet handed out
+    for (const Seg& sg : segs)
+      remaining += (cost_prefix[size_t(sg.stage_begin + sg.n_stages)] - cost_prefix[size_t(sg.stage_begin)] + kUnitOverhead) * sched_kv_heads;
+    // A CTA's share is recomputed from what is left whenever a CTA is opened, so that the overhead of the
+    // extra units the cuts themselves create never piles up on the last CTA.
+    auto share = [&](int c) {
+      const int64_t left = n_ctas - c;
+      return std::max<int64_t>((remaining + left * kUnitOverhead + left - 1) / left, 2 * kStage + kUnitOverhead);
+    };
+    P->cta_unit_off.assign(size_t(n_ctas) + 1, 0);
+    struct PartKey { int32_t rowkv, unit, k; };
+    std::vector<PartKey> keys;
+    int cta = 0;
+    int64_t acc = 0, target = share(0), max_acc = 0;
+    const int64_t first_share = target;
+    auto emit = [&](const Seg& sg, int kvh, int32_t st_off, int32_t take) {
+      WorkUnit wu{};
+      wu.stage_begin = sg.stage_begin + st_off;
+      wu.n_stages = take;
+      wu.row_begin = int32_t(P->item_rows.size());
+      wu.n_rows = sg.n_rows;
+      wu.kvh = kvh;
+      uint64_t seen = 0;  // rows that see at least one stage of the unit
+      for (int32_t i = 0; i < take; ++i) {
+        const StageDesc& sd = P->stages[size_t(wu.stage_begin + i)];
+        seen |= uint64_t(sd.mask_lo) | (uint64_t(sd.mask_hi) << 32);
       }
-      S.max_item_rows = std::max<int64_t>(S.max_item_rows, it.n_rows);
-      sorted.push_back(it);
+      for (int32_t k = 0; k < sg.n_rows; ++k) {
+        const int32_t row = seg_rows[size_t(sg.rows_begin + k)];
+        const bool has = (seen >> k) & 1;
+        if (has) keys.push_back(PartKey{row * sched_kv_heads + kvh, int32_t(P->units.size()), k});
+        P->item_rows.push_back(ItemRow{row, -1});
+      }
+      P->units.push_back(wu);
+      P->cta_unit_off[size_t(cta) + 1] = int32_t(P->units.size());
+      S.max_item_rows = std::max<int64_t>(S.max_item_rows, sg.n_rows);
+    };
+    for (const Seg& sg : segs) {
+      for (int kvh = 0; kvh < sched_kv_heads; ++kvh) {
+        int32_t off = 0;
+        remaining -= kUnitOverhead;  // the overhead of this run's first unit is charged below
+        while (off < sg.n_stages) {
+          const int64_t room = target - acc - kUnitOverhead;
+          const int64_t base = cost_prefix[size_t(sg.stage_begin + off)];
+          const int64_t rest = cost_prefix[size_t(sg.stage_begin + sg.n_stages)] - base;
+          if (cta < n_ctas - 1 && room < kStage / 2) {  // this CTA is full
+            ++cta;
+            acc = 0;
+            target = share(cta);
+            continue;
+          }
+          int32_t take = sg.n_stages - off;
+          if (cta < n_ctas - 1 && rest > room + kStage / 2) {
+            // the run of stages whose cost comes closest to the room (at least one stage): rounding to the
+            // nearest stage boundary keeps the shortfalls from drifting onto the last CTAs
+            const int64_t* lo_it = cost_prefix.data() + sg.stage_begin + off;
+            const int64_t* hi_it = cost_prefix.data() + sg.stage_begin + sg.n_stages + 1;
+            const int64_t* it = std::upper_bound(lo_it, hi_it, base + room);  // first prefix beyond the room
+            take = int32_t(it - lo_it) - 1;
+            if (it != hi_it && (*it - (base + room)) < ((base + room) - *(it - 1))) ++take;
+            take = std::max<int32_t>(1, std::min<int32_t>(take, sg.n_stages - off));
+          }
+          take = std::min(take, max_unit_stages);
+          emit(sg, kvh, off, take);
+          const int64_t c = cost_prefix[size_t(sg.stage_begin + off + take)] - base;
+          acc += c + kUnitOverhead;
+          max_acc = std::max(max_acc, acc);
+          remaining -= c;
+          off += take;
+        }
+      }
     }
-    P->items.swap(sorted);
-    S.n_items = int64_t(P->items.size());
-    S.n_partials = P->row_part_off[n_rows];
+    S.max_cta_cost = max_acc;
+    for (int c = 1; c <= n_ctas; ++c) P->cta_unit_off[c] = std::max(P->cta_unit_off[c], P->cta_unit_off[c - 1]);
+    // partial slots: contiguous per (row, KV head), in unit order
+    P->rowkv_part_off.assign(size_t(n_rows) * sched_kv_heads + 1, 0);
+    for (const PartKey& k : keys) P->rowkv_part_off[size_t(k.rowkv) + 1]++;
+    for (size_t i = 1; i < P->rowkv_part_off.size(); ++i) P->rowkv_part_off[i] += P->rowkv_part_off[i - 1];
+    std::vector<int32_t> next(P->rowkv_part_off.begin(), P->rowkv_part_off.end() - 1);
+    for (const PartKey& k : keys) P->item_rows[size_t(P->units[k.unit].row_begin + k.k)].part = next[k.rowkv]++;
+    S.n_items = int64_t(P->units.size());
+    S.n_partials = int64_t(keys.size());
+    S.n_ctas = n_ctas;
+    S.chunk_tokens = chunk > 0 ? chunk : first_share;
   }
   // ---- prefill: heaviest query tiles first
   if (prefill_ready) {
@@ -384,10 +443,11 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   auto place = [&](size_t bytes) { size_t o = off; off = align256(off + bytes); return o; };
   L.pos_id = place(P->pos_id.size() * sizeof(int32_t));
   L.slot = place(P->slot.size() * sizeof(int64_t));
-  L.page_idx = place(P->page_idx.size() * sizeof(int32_t));
-  L.items = place(P->items.size() * sizeof(WorkItem));
+  L.stages = place(P->stages.size() * sizeof(StageDesc));
+  L.units = place(P->units.size() * sizeof(WorkUnit));
+  L.cta_unit_off = place(P->cta_unit_off.size() * sizeof(int32_t));
   L.item_rows = place(P->item_rows.size() * sizeof(ItemRow));
-  L.row_part_off = place(P->row_part_off.size() * sizeof(int32_t));
+  L.rowkv_part_off = place(P->rowkv_part_off.size() * sizeof(int32_t));
   L.sched = place(sizeof(P->sched_zero));
   L.q_tiles = place(P->q_tiles.size() * sizeof(QTile));
   L.kv_ranges = place(P->kv_ranges.size() * sizeof(KvRange));

@@ -82,7 +82,8 @@ __global__ void __launch_bounds__(128) rope_write_kv_kernel(const T* q, const T*
     const int uu = is_q ? u : u - n_q_units;
     const int h = uu / CH, c = uu % CH;
     const T* src = is_q ? q + (int64_t(t) * Hq + h) * D : k + (int64_t(t) * Hkv + h) * D;
-    T* dst = is_q ? q_rot + (int64_t(t) * Hq + h) * D : k_pages + (((page * Hkv + h) << 4) + off) * D;
+    // pool element (page, head, token, c) lives in 64-element column block c / 64 of the (page, head) block
+    T* dst = is_q ? q_rot + (int64_t(t) * Hq + h) * D : k_pages + (page * Hkv + h) * (16 * D) + off * 64;
     T* dst2 = is_q ? nullptr : k_rot + (int64_t(t) * Hkv + h) * D;
     const bool w1 = is_q || k_pages != nullptr, w2 = !is_q && k_rot != nullptr;
     float lo[N], hi[N], olo[N], ohi[N];
@@ -95,8 +96,14 @@ __global__ void __launch_bounds__(128) rope_write_kv_kernel(const T* q, const T*
       ohi[i] = hi[i] * cc + lo[i] * ss;
     }
     if (w1) {
-      Vec16<T>::store(dst + c * N, olo);
-      Vec16<T>::store(dst + HALF + c * N, ohi);
+      if (is_q) {
+        Vec16<T>::store(dst + c * N, olo);
+        Vec16<T>::store(dst + HALF + c * N, ohi);
+      } else {
+        const int e0 = c * N, e1 = HALF + c * N;  // element indices inside the head vector
+        Vec16<T>::store(dst + (e0 >> 6) * 1024 + (e0 & 63), olo);
+        Vec16<T>::store(dst + (e1 >> 6) * 1024 + (e1 & 63), ohi);
+      }
     }
     if (w2) {
       Vec16<T>::store(dst2 + c * N, olo);
@@ -109,7 +116,8 @@ __global__ void __launch_bounds__(128) rope_write_kv_kernel(const T* q, const T*
   for (int u = threadIdx.x; u < Hkv * VCH; u += blockDim.x) {
     const int h = u / VCH, c = u % VCH;
     const uint4 val = *reinterpret_cast<const uint4*>(v + (int64_t(t) * Hkv + h) * D + c * N);
-    *reinterpret_cast<uint4*>(v_pages + (((page * Hkv + h) << 4) + off) * D + c * N) = val;
+    const int e = c * N;
+    *reinterpret_cast<uint4*>(v_pages + (page * Hkv + h) * (16 * D) + (e >> 6) * 1024 + off * 64 + (e & 63)) = val;
   }
 }
 

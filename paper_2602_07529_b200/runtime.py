@@ -15,6 +15,19 @@ def torch_dtype(geom: synth.Geometry):
     return torch.bfloat16 if geom.dtype == "bf16" else torch.float32
 
 
+def pool_shape(num_pages: int, geom: synth.Geometry):
+    """Shape of a K (or V) page pool: [pages][KV heads][head_dim / 64][page_size][64]."""
+    return (num_pages, geom.n_kv_heads, geom.head_dim // 64, geom.page_size, 64)
+
+
+def pool_tokens(pool, slot):
+    """Head vectors [n, KV heads, head_dim] stored at the pool slots ``slot`` (int64 tensor): a view-only gather that
+    undoes the 64-element column blocking of the pool."""
+    ps = pool.shape[3]
+    x = pool[slot // ps, :, :, slot % ps, :]            # [n, Hkv, head_dim / 64, 64]
+    return x.reshape(x.shape[0], x.shape[1], -1)
+
+
 def _dev_bytes(n: int, device):
     """256-byte aligned uint8 scratch of at least n bytes (torch's caching allocator aligns to 512)."""
     return torch.empty(max(int(n), 256), dtype=torch.uint8, device=device)
@@ -74,7 +87,7 @@ class DecodeState:
         g, b = wl.geom, wl.batch
         self.geom = B.geom_of(wl)
         dt = torch_dtype(g)
-        shape = (b.num_pages, g.n_kv_heads, g.page_size, g.head_dim)
+        shape = pool_shape(b.num_pages, g)
         fill = float("nan") if canary else 0.0
         self.pools = [(torch.full(shape, fill, dtype=dt, device=device), torch.full(shape, fill, dtype=dt, device=device))
                       for _ in range(n_pool_copies)]
@@ -111,7 +124,7 @@ class PrefillState:
         self.q, self.k, self.v = _stack_values(wl, "all", device)
         self.pod = PlanOnDevice(b, device, geom=g)
         self.plan = self.pod.plan
-        shape = (b.num_pages, g.n_kv_heads, g.page_size, g.head_dim)
+        shape = pool_shape(b.num_pages, g)
         self.k_pages = torch.zeros(shape, dtype=dt, device=device)
         self.v_pages = torch.zeros(shape, dtype=dt, device=device)
         self.q_rot = torch.empty_like(self.q)

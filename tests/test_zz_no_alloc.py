@@ -42,8 +42,8 @@ def test_static_scratch_matches_workspace_entry_point_twice():
 
 def test_static_scratch_rejects_oversized_plans():
     from paper_2602_07529_b200 import binding as B, runtime
-    wl = synth.config2(n_req=1, prefix=4096, branches=5, branch_len=40)
-    st = runtime.DecodeState(wl, chunk_tokens=16)            # 16-token chunks: hundreds of partials per row
+    wl = synth.config2(n_req=1, prefix=16384, branches=16, branch_len=40)
+    st = runtime.DecodeState(wl, chunk_tokens=16)            # one-stage work units: hundreds of partials per row
     assert st.plan.workspace_bytes(st.geom, B.OP_DECODE_ATTN) > B.mv_static_workspace_bytes()
     kp, vp = st.pools[0]
     with pytest.raises(B.MvError) as e:
