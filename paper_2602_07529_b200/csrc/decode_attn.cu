@@ -59,19 +59,19 @@ struct Cfg {
   // dynamic shared memory: stages | q | meta (see Smem)
   static constexpr int OFF_Q = NSTAGES * STAGE_BYTES;
   static constexpr int OFF_META = OFF_Q + Q_BYTES;
-  static constexpr int SMEM = OFF_META + 896;  // D = 128: 115,584 B, so that two CTAs share an SM
+  static constexpr int SMEM = OFF_META + 1024;  // D = 128: 115,712 B, the most that lets two CTAs share an SM
 };
 
 struct Meta {                       // tail of the dynamic shared memory
   float2 ml[4][16];                 // epilogue: (max, sum) of every row of every consumer warp    512 B
   int32_t pv[MAXQV];                // partial vector index (partial * G + head in group) or -1    256 B
   int32_t n_stages, n_qv;
-  int32_t st_tokens[NSTAGES];       // per stage buffer: valid tokens
-  uint32_t st_mask_lo[NSTAGES], st_mask_hi[NSTAGES];  // per stage buffer: rows that see the stage
+  uint32_t st_tokens[NSTAGES];      // per stage buffer: valid tokens of the four page slots, a byte each
+  uint2 st_mask[NSTAGES][4];        // per stage buffer and page slot: rows that see the slot's node (lo, hi)
   uint64_t full[NSTAGES], empty[NSTAGES], q_full, q_empty;
   int abort;
 };
-static_assert(sizeof(Meta) <= 896, "meta area");
+static_assert(sizeof(Meta) <= 1024, "meta area");
 
 // Byte offset of 16-byte chunk `chunk` of token row `row` inside a K (or V) stage tile as TMA lays it out: a
 // stage is four page blocks; a page block is [column block chunk / 8][16 tokens][128 B], and inside a
@@ -106,7 +106,7 @@ struct UnitRegs {  // a unit's descriptor, loaded ahead of use
   int stage_begin = 0, n_stages = 0, row_begin = 0, n_rows = 0, kvh = 0;
 };
 struct StageRegs {  // one stage descriptor per lane (a window of 32 stages)
-  int4 a = make_int4(0, 0, 0, 0), b = make_int4(0, 0, 0, 0);
+  int4 a = make_int4(0, 0, 0, 0), b = make_int4(0, 0, 0, 0), c = make_int4(0, 0, 0, 0), d = make_int4(0, 0, 0, 0);
 };
 
 template <int D>
@@ -132,8 +132,10 @@ __device__ __forceinline__ void producer(const DecodeArgs& a, int u_begin, int u
     StageRegs r;
     if (first + lane < w.n_stages) {
       const int4* p = reinterpret_cast<const int4*>(a.stages + w.stage_begin + first + lane);
-      r.a = __ldg(p);
-      r.b = __ldg(p + 1);
+      r.a = __ldg(p);      // pages
+      r.b = __ldg(p + 1);  // tokens per slot, slots in use, mask_lo[0..1]
+      r.c = __ldg(p + 2);  // mask_lo[2..3], mask_hi[0..1]
+      r.d = __ldg(p + 3);  // mask_hi[2..3]
     }
     return r;
   };
@@ -183,19 +185,20 @@ __device__ __forceinline__ void producer(const DecodeArgs& a, int u_begin, int u
       const int src = s & 31;
       const int4 da = make_int4(__shfl_sync(0xffffffffu, win.a.x, src), __shfl_sync(0xffffffffu, win.a.y, src),
                                 __shfl_sync(0xffffffffu, win.a.z, src), __shfl_sync(0xffffffffu, win.a.w, src));
-      const int n_tok = __shfl_sync(0xffffffffu, win.b.x, src);
-      const int m_lo = __shfl_sync(0xffffffffu, win.b.y, src), m_hi = __shfl_sync(0xffffffffu, win.b.z, src);
+      const int n_pages = __shfl_sync(0xffffffffu, win.b.y, src);
       const int b = issued % NSTAGES;
-      const int n_pages = (n_tok + 15) >> 4;
       const uint32_t bar = sy.full + 8 * b;
-      if (lane == 0) {
-        wait_or_flag(sy, sy.empty + 8 * b, ((issued / NSTAGES) & 1) ^ 1);  // every consumer warp has released the buffer
-        meta->st_tokens[b] = n_tok;
-        meta->st_mask_lo[b] = uint32_t(m_lo);
-        meta->st_mask_hi[b] = uint32_t(m_hi);
-        mv::mbar_arrive_expect_tx(bar, uint32_t(n_pages) * 16 * D * 2 * 2);  // releases the stores above
+      if (lane == 0) wait_or_flag(sy, sy.empty + 8 * b, ((issued / NSTAGES) & 1) ^ 1);  // every consumer warp has released the buffer
+      __syncwarp();
+      if (lane == src) {  // the lane that holds the descriptor publishes the page slots' token counts and row masks
+        meta->st_tokens[b] = uint32_t(win.b.x);
+        meta->st_mask[b][0] = make_uint2(uint32_t(win.b.z), uint32_t(win.c.z));
+        meta->st_mask[b][1] = make_uint2(uint32_t(win.b.w), uint32_t(win.c.w));
+        meta->st_mask[b][2] = make_uint2(uint32_t(win.c.x), uint32_t(win.d.x));
+        meta->st_mask[b][3] = make_uint2(uint32_t(win.c.y), uint32_t(win.d.y));
       }
       __syncwarp();
+      if (lane == 0) mv::mbar_arrive_expect_tx(bar, uint32_t(n_pages) * 16 * D * 2 * 2);  // releases the stores above
       // lane j < 8: page j / 2 of the stage, K or V; one box = the whole contiguous (page, head) block
       const int p = (lane >> 1) & 3, kv = lane & 1;
       const int page = p == 0 ? da.x : p == 1 ? da.y : p == 2 ? da.z : da.w;
@@ -242,16 +245,32 @@ __device__ __forceinline__ void consume_unit(const DecodeArgs& a, int n_stages, 
     const uint32_t kb = smem_base + b * Cfg<D>::STAGE_BYTES, vb = kb + Cfg<D>::KV_BYTES;
     ++consumed;
     const bool last = (s == n_stages - 1);
-    const int tok_lim = meta->st_tokens[b] - tok_w;  // valid tokens of this warp's slice
-    const uint64_t seen_by = (uint64_t(meta->st_mask_hi[b]) << 32) | meta->st_mask_lo[b];  // rows that see the stage's node
-    if (tok_lim > 0 && (seen_by & tile_rows) != 0) {  // warp-uniform: some row of this m-tile sees the stage
-      if (tok_lim < WT) {
-        // ragged end of the node: rows past the last token hold whatever the page (or an older stage) left
-        // there; V must be zero where P is zero, or 0 * NaN would poison the output
-        const int r0 = tok_w + tok_lim, nz = (WT - tok_lim) * Cfg<D>::CPR;
-        for (int i = lane; i < nz; i += 32) {
-          const int r = r0 + i / Cfg<D>::CPR, c = i % Cfg<D>::CPR;
-          *reinterpret_cast<uint4*>(smem + (vb - smem_base) + tile_off<D>(r, c)) = make_uint4(0, 0, 0, 0);
+    // this warp's slice of the stage is NT / 2 page slots; each has its own valid-token count and row mask
+    constexpr int NS = NT / 2;
+    const int slot0 = tok_w >> 4;
+    const uint32_t tok4 = meta->st_tokens[b] >> (8 * slot0);
+    uint64_t seen_by[NS];
+    int ntok[NS];
+    bool any_work = false, plain = true;
+#pragma unroll
+    for (int j = 0; j < NS; ++j) {
+      const uint2 mk = meta->st_mask[b][slot0 + j];
+      seen_by[j] = (uint64_t(mk.y) << 32) | mk.x;
+      ntok[j] = int((tok4 >> (8 * j)) & 0xffu);
+      any_work |= ntok[j] > 0 && (seen_by[j] & tile_rows) != 0;
+      plain &= ntok[j] == 16 && (seen_by[j] & tile_rows) == tile_rows;
+    }
+    if (any_work) {  // warp-uniform: some row of this m-tile sees some token of the slice
+      if (!plain) {
+        // rows past a page's last token hold whatever the pool (or an older stage) left there; V must be
+        // zero where P is zero, or 0 * NaN would poison the output
+#pragma unroll
+        for (int j = 0; j < NS; ++j) {
+          const int nz = (16 - ntok[j]) * Cfg<D>::CPR;
+          for (int i = lane; i < nz; i += 32) {
+            const int r = tok_w + j * 16 + ntok[j] + i / Cfg<D>::CPR, c = i % Cfg<D>::CPR;
+            *reinterpret_cast<uint4*>(smem + (vb - smem_base) + tile_off<D>(r, c)) = make_uint4(0, 0, 0, 0);
+          }
         }
         __syncwarp();
       }
@@ -271,7 +290,7 @@ __device__ __forceinline__ void consume_unit(const DecodeArgs& a, int n_stages, 
       }
       // scale to log2 units, mask the ragged tail, online softmax
       float mx0 = -INFINITY, mx1 = -INFINITY;
-      if (tok_lim >= WT && (seen_by & tile_rows) == tile_rows) {  // every row of the m-tile sees every token
+      if (plain) {  // every row of the m-tile sees every token of the slice
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
@@ -279,14 +298,15 @@ __device__ __forceinline__ void consume_unit(const DecodeArgs& a, int n_stages, 
           mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
           mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
         }
-      } else {  // the DAG mask (a row that does not see the node) and the ragged end of the node
-        const bool vis0 = row0 >= 0 && ((seen_by >> row0) & 1), vis1 = row1 >= 0 && ((seen_by >> row1) & 1);
+      } else {  // the DAG mask (a row that does not see the page's node) and the ragged last page of a node
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
+          const int j = nt >> 1;
+          const bool vis0 = row0 >= 0 && ((seen_by[j] >> row0) & 1), vis1 = row1 >= 0 && ((seen_by[j] >> row1) & 1);
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const int col = nt * 8 + (lane & 3) * 2 + (e & 1);
-            sacc[nt][e] = (col < tok_lim && (e < 2 ? vis0 : vis1)) ? sacc[nt][e] * a.scale_log2 : -INFINITY;
+            const int col = (nt & 1) * 8 + (lane & 3) * 2 + (e & 1);  // token inside the page
+            sacc[nt][e] = (col < ntok[j] && (e < 2 ? vis0 : vis1)) ? sacc[nt][e] * a.scale_log2 : -INFINITY;
           }
           mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
           mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
@@ -339,7 +359,7 @@ __device__ __forceinline__ void consume_unit(const DecodeArgs& a, int n_stages, 
       }
     }
     if (!last || KS == 1) {  // hand the stage back; with kv splits the unit's last stage is kept as epilogue scratch
-      if (last) mv::fence_proxy_async();  // a ragged stage was patched with ordinary stores; TMA refills it next
+      mv::fence_proxy_async();  // a ragged page may have been patched with ordinary stores; TMA refills the buffer next
       __syncwarp();
       if (lane == 0) mv::mbar_arrive(sy.empty + 8 * b);
     }

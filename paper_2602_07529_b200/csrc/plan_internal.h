@@ -13,15 +13,17 @@ constexpr int kPrefillQTile = 128;   // query rows per prefill tile (tiles never
 constexpr int kPrefillKvTile = 64;   // granularity used only for the executed-pairs statistic
 
 // Decode work lists.  A request's frontier rows (at most 64 / group_size of them per row group) and all the KV
-// they see form one stream of 64-token STAGES, node after node; a stage belongs to one node and carries the
-// set of rows that see that node.  A work unit is a run of consecutive stages for ONE KV head; units are
+// they see form one stream of pages, node after node, packed four to a 64-token STAGE; every page slot
+// carries the set of rows that see its node (the DAG mask at page granularity) and its count of valid tokens.  A work unit is a run of consecutive stages for ONE KV head; units are
 // listed CTA by CTA (cta_unit_off): the planner cuts the step's whole stream into equal shares.
-struct StageDesc {
-  int32_t page[4];    // physical pages of the stage (unused entries repeat page[0])
-  int32_t n_tokens;   // valid tokens, 1..64 (the node's last stage may be ragged)
-  uint32_t mask_lo, mask_hi;  // bit r: row r of the unit's row group sees this stage
-  int32_t pad;
+struct StageDesc {     // 64 bytes
+  int32_t page[4];     // physical pages of the stage's four page slots (absent slots repeat page[0])
+  uint32_t n_tokens4;  // valid tokens of each page slot, one byte per slot (16 except on a node's last page)
+  int32_t n_pages;     // page slots in use, 1..4 (fewer than 4 only on the last stage of a stream)
+  uint32_t mask_lo[4], mask_hi[4];  // per page slot: bit r set = row r of the unit's row group sees the page's node
+  int32_t pad[2];
 };
+static_assert(sizeof(StageDesc) == 64, "stage descriptor layout");
 struct WorkUnit {
   int32_t stage_begin;  // index into the stage table
   int32_t n_stages;

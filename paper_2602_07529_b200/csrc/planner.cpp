@@ -236,6 +236,13 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       for (size_t r0 = 0; r0 < req_rows.size(); r0 += size_t(max_rows_per_item)) {
         const size_t r1 = std::min(req_rows.size(), r0 + size_t(max_rows_per_item));
         Seg sg{int32_t(P->stages.size()), 0, int32_t(seg_rows.size()), int32_t(r1 - r0)};
+        StageDesc sd{};  // the stage being filled, page slot by page slot
+        auto flush = [&]() {
+          if (sd.n_pages == 0) return;
+          for (int j = sd.n_pages; j < 4; ++j) sd.page[j] = sd.page[0];
+          P->stages.push_back(sd);
+          sd = StageDesc{};
+        };
         for (int u = 0; u < n; ++u) {
           const int32_t L = b->node_len[lo + u] + b->node_new[lo + u];
           if (L == 0) continue;
@@ -244,19 +251,16 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
             if (vis.get(row_node[k], u)) mask |= uint64_t(1) << (k - r0);
           if (mask == 0) continue;
           const int32_t* pages = b->page_idx + b->page_off[lo + u];
-          const int n_pages = (L + ps - 1) / ps;
-          for (int32_t t0 = 0; t0 < L; t0 += kStage) {
-            StageDesc sd{};
-            sd.n_tokens = std::min<int32_t>(kStage, L - t0);
-            for (int j = 0; j < 4; ++j) {
-              const int pi = t0 / ps + j;
-              sd.page[j] = pages[pi < n_pages ? pi : t0 / ps];
-            }
-            sd.mask_lo = uint32_t(mask);
-            sd.mask_hi = uint32_t(mask >> 32);
-            P->stages.push_back(sd);
+          for (int32_t t0 = 0; t0 < L; t0 += ps) {
+            const int j = sd.n_pages++;
+            sd.page[j] = pages[t0 / ps];
+            sd.n_tokens4 |= uint32_t(std::min<int32_t>(ps, L - t0)) << (8 * j);
+            sd.mask_lo[j] = uint32_t(mask);
+            sd.mask_hi[j] = uint32_t(mask >> 32);
+            if (sd.n_pages == 4) flush();
           }
         }
+        flush();
         sg.n_stages = int32_t(P->stages.size()) - sg.stage_begin;
         seg_rows.insert(seg_rows.end(), req_rows.begin() + r0, req_rows.begin() + r1);
         if (sg.n_stages > 0) segs.push_back(sg);
@@ -320,10 +324,9 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     const int64_t n_rows = new_tok_count;
     const int n_ctas = b->sched_ctas > 0 ? b->sched_ctas : 296;
     constexpr int64_t kUnitOverhead = 96;  // fixed cost of a unit (q staging, epilogue), in token equivalents
-    constexpr int64_t kStageOverhead = 8;  // fixed cost of a stage (barrier round trip), in token equivalents
     const int max_unit_stages = chunk > 0 ? std::max(1, chunk / kStage) : (1 << 30);
     std::vector<int64_t> cost_prefix(P->stages.size() + 1, 0);  // running stage cost over the stage table
-    for (size_t i = 0; i < P->stages.size(); ++i) cost_prefix[i + 1] = cost_prefix[i] + P->stages[i].n_tokens + kStageOverhead;
+    for (size_t i = 0; i < P->stages.size(); ++i) cost_prefix[i + 1] = cost_prefix[i] + 16 * P->stages[i].n_pages + 16;  // a slot's fixed cost + its pages
     int64_t remaining = 0;  // cost not yet handed out
     for (const Seg& sg : segs)
       remaining += (cost_prefix[size_t(sg.stage_begin + sg.n_stages)] - cost_prefix[size_t(sg.stage_begin)] + kUnitOverhead) * sched_kv_heads;
@@ -349,7 +352,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       uint64_t seen = 0;  // rows that see at least one stage of the unit
       for (int32_t i = 0; i < take; ++i) {
         const StageDesc& sd = P->stages[size_t(wu.stage_begin + i)];
-        seen |= uint64_t(sd.mask_lo) | (uint64_t(sd.mask_hi) << 32);
+        for (int j = 0; j < sd.n_pages; ++j) seen |= uint64_t(sd.mask_lo[j]) | (uint64_t(sd.mask_hi[j]) << 32);
       }
       for (int32_t k = 0; k < sg.n_rows; ++k) {
         const int32_t row = seg_rows[size_t(sg.rows_begin + k)];
