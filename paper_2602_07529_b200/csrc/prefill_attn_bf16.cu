@@ -234,6 +234,7 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
 namespace mv {
 mv_status prefill_f32(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out,
                       cudaStream_t st);
+mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out, cudaStream_t st);
 }
 
 extern "C" mv_status mv_dag_prefill_attn(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_rot,
@@ -249,5 +250,9 @@ extern "C" mv_status mv_dag_prefill_attn(const mv_plan* P, const mv_attn_geom* g
   if (!P->device_buf) return MV_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (g->dtype == MV_F32) return mv::prefill_f32(P, g, q_rot, k_rot, v, out, s);
+  // head_dim 128 with an even group size runs on tcgen05 (two heads of a KV head per CTA); TMA needs 16-byte
+  // aligned tensors.  Everything else takes the mma.sync kernel below.
+  const bool aligned = ((reinterpret_cast<uintptr_t>(q_rot) | reinterpret_cast<uintptr_t>(k_rot) | reinterpret_cast<uintptr_t>(v)) & 15) == 0;
+  if (g->head_dim == 128 && (g->n_q_heads / g->n_kv_heads) % 2 == 0 && aligned) return mv::prefill_tc(P, g, q_rot, k_rot, v, out, s);
   return g->head_dim == 128 ? launch<128>(P, g, q_rot, k_rot, v, out, s) : launch<64>(P, g, q_rot, k_rot, v, out, s);
 }

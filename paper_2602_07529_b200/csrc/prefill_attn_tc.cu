@@ -1,0 +1,371 @@
+// Topology-masked prefill attention on the 5th-generation tensor cores (Eq. 2 with the DAG mask of Eq. 3 in
+// visibility-set form), head_dim 128, bf16 in, fp32 accumulation in tensor memory.
+//
+// A CTA owns one query tile (128 rows of one node) for TWO query heads of the same KV head, so the two
+// problems walk the same KV tiles with the same mask and every K / V tile that TMA brings in feeds four
+// 128 x 128 x 128 products.  Only the KV ranges the tile's node may see are walked (tile skipping); the
+// causal test applies only inside the node's own range and only on tiles that touch the diagonal; ragged
+// range ends are masked by a column bound.
+//
+// Warp roles (384 threads): warp 0 = TMA producer (Q tiles once, then a ring of K and V tiles), warp 1 =
+// MMA issuer (one thread: S_i = Q_i K^T into tensor memory, O_i += P_i V with P_i read from tensor memory),
+// warps 4-7 and 8-11 = softmax groups of head 0 and head 1 (one thread per query row: online softmax in
+// log2 units, P written back over S as packed bf16, O rescaled in tensor memory only when the row maximum
+// moved by more than 2^8, final normalisation and store).  The issuer alternates the two heads, so one
+// group's softmax overlaps the other head's products.  Every mbarrier wait is bounded (status word).
+#include "common.cuh"
+#include "umma.cuh"
+
+namespace {
+
+using bf16 = __nv_bfloat16;
+constexpr int D = 128;
+constexpr int BQ = 128;                 // query rows per tile
+constexpr int BK = 128;                 // keys per KV tile
+constexpr int TILE_BYTES = BK * D * 2;  // 32 KB: [2 column blocks][128 rows][128 B]
+constexpr int RING = 5;                 // K and V tiles in flight (K0 V0 K1 V1 ...)
+constexpr int NTHREADS = 384;
+constexpr int OFF_Q = 0;                        // Q0, Q1
+constexpr int OFF_RING = 2 * TILE_BYTES;        // ring entries
+constexpr int OFF_BAR = OFF_RING + RING * TILE_BYTES;
+constexpr int SMEM_BYTES = OFF_BAR + 256;
+constexpr float RESCALE_THRESHOLD = 8.f;  // log2 units: P stays below 2^8, well inside bf16 and fp32 range
+
+struct Bars {  // shared-memory addresses
+  uint32_t q_full, kv_full, kv_empty, s_full, p_full, o_done;
+};
+
+struct PrefillArgs {
+  const mv::QTile* q_tiles;
+  const mv::KvRange* ranges;
+  bf16* out;
+  int32_t* status;
+  int Hq, G;
+  float scale_log2;
+};
+
+// The KV tiles of a query tile, in the order every role walks them: ranges in table order, 128 keys at a time;
+// a causal range stops after the tile's last query.
+struct TileIter {
+  const mv::KvRange* rg;
+  int n_ranges, q_last;
+  int ri = 0, pos = 0, end = 0, causal = 0;
+  __device__ TileIter(const mv::KvRange* r, int n, int ql) : rg(r), n_ranges(n), q_last(ql) {}
+  // start key, valid keys (1..128), causal flag of the next tile; false when the walk is over
+  __device__ bool next(int& start, int& n, int& c) {
+    while (pos >= end) {
+      if (ri >= n_ranges) return false;
+      const mv::KvRange r = rg[ri++];
+      pos = r.kv_start;
+      end = r.kv_start + r.kv_len;
+      causal = r.causal;
+      if (causal) end = min(end, q_last + 1);
+    }
+    start = pos;
+    n = min(BK, end - pos);
+    c = causal;
+    pos += BK;
+    return true;
+  }
+};
+
+struct Waiter {  // bounded waits: after one ran out every later wait returns at once, so the CTA still ends
+  volatile int* abort;
+  int32_t* status;
+  __device__ __forceinline__ void wait(uint32_t bar, uint32_t parity) const {
+    if (*abort) return;
+    if (!mv::mbar_wait_bounded(bar, parity)) {
+      *abort = 1;
+      atomicExch(status, int(MV_ERR_TIMEOUT));
+    }
+  }
+};
+
+__device__ __forceinline__ void producer_warp(const mv::QTile& qt, const PrefillArgs& a, int h0, int kvh, uint32_t smem_base,
+                                              const Bars& br, const Waiter& w, const CUtensorMap* tm_q, const CUtensorMap* tm_k,
+                                              const CUtensorMap* tm_v) {
+  if ((threadIdx.x & 31) != 0) return;
+  mv::mbar_arrive_expect_tx(br.q_full, 2 * TILE_BYTES);
+  for (int i = 0; i < 2; ++i)
+    for (int h = 0; h < 2; ++h)
+      mv::tma_load_2d(smem_base + OFF_Q + i * TILE_BYTES + h * (TILE_BYTES / 2), tm_q, (h0 + i) * D + h * 64, qt.q_start, br.q_full);
+  TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.q_start + qt.q_len - 1);
+  int start, n, c, e = 0;  // e: ring entries issued so far
+  while (it.next(start, n, c)) {
+    for (int kv = 0; kv < 2; ++kv, ++e) {
+      const int slot = e % RING;
+      w.wait(br.kv_empty + 8 * slot, ((e / RING) & 1) ^ 1);
+      const uint32_t bar = br.kv_full + 8 * slot;
+      mv::mbar_arrive_expect_tx(bar, TILE_BYTES);
+      const uint32_t dst = smem_base + OFF_RING + slot * TILE_BYTES;
+      for (int h = 0; h < 2; ++h) mv::tma_load_2d(dst + h * (TILE_BYTES / 2), kv ? tm_v : tm_k, kvh * D + h * 64, start, bar);
+    }
+  }
+}
+
+// S_i = Q_i K^T: both operands K-major, eight 16-element k-steps
+__device__ __forceinline__ void issue_qk(uint32_t s_tmem, uint32_t q_smem, uint32_t k_smem) {
+  constexpr uint32_t idesc = mv::um::idesc_bf16(BQ, BK, 0, 0);
+#pragma unroll
+  for (int k = 0; k < D / 16; ++k) {
+    const uint32_t off = (k >> 2) * (TILE_BYTES / 2) + (k & 3) * 32;
+    mv::um::mma_ss(s_tmem, mv::um::smem_desc(q_smem + off, 16, 1024), mv::um::smem_desc(k_smem + off, 16, 1024), idesc, k > 0);
+  }
+}
+// O_i (+)= P_i V: P from tensor memory (two bf16 per column), V MN-major, eight 16-key k-steps
+__device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_smem, bool accumulate) {
+  constexpr uint32_t idesc = mv::um::idesc_bf16(BQ, D, 0, 1);
+#pragma unroll
+  for (int k = 0; k < BK / 16; ++k)
+    mv::um::mma_ts(o_tmem, p_tmem + k * 8, mv::um::smem_desc(v_smem + k * 2048, TILE_BYTES / 2, 1024), idesc, accumulate || k > 0);
+}
+
+__device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs& a, uint32_t smem_base, uint32_t tmem, const Bars& br,
+                                         const Waiter& w) {
+  if ((threadIdx.x & 31) != 0) return;
+  TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.q_start + qt.q_len - 1);
+  int start, n, c;
+  int n_tiles = 0;
+  while (it.next(start, n, c)) ++n_tiles;
+  if (n_tiles == 0) return;
+  const uint32_t q0 = smem_base + OFF_Q, q1 = q0 + TILE_BYTES;
+  const uint32_t s0 = tmem, s1 = tmem + 128, o0 = tmem + 256, o1 = tmem + 384;
+  auto slot_addr = [&](int e) { return smem_base + OFF_RING + (e % RING) * TILE_BYTES; };
+  auto wait_full = [&](int e) { w.wait(br.kv_full + 8 * (e % RING), (e / RING) & 1); };
+  auto release = [&](int e) { mv::um::commit(br.kv_empty + 8 * (e % RING)); };
+  w.wait(br.q_full, 0);
+  wait_full(0);
+  mv::um::fence_after();
+  issue_qk(s0, q0, slot_addr(0));
+  mv::um::commit(br.s_full);
+  issue_qk(s1, q1, slot_addr(0));
+  mv::um::commit(br.s_full + 8);
+  release(0);
+  for (int j = 0; j < n_tiles; ++j) {
+    const int ev = 2 * j + 1, ek = 2 * j + 2;  // ring entries of V_j and K_{j+1}
+    const bool more = j + 1 < n_tiles;
+    wait_full(ev);
+    w.wait(br.p_full, j & 1);
+    mv::um::fence_after();
+    issue_pv(o0, s0, slot_addr(ev), j > 0);
+    mv::um::commit(br.o_done);
+    if (more) {
+      wait_full(ek);
+      mv::um::fence_after();
+      issue_qk(s0, q0, slot_addr(ek));
+      mv::um::commit(br.s_full);
+    }
+    w.wait(br.p_full + 8, j & 1);
+    mv::um::fence_after();
+    issue_pv(o1, s1, slot_addr(ev), j > 0);
+    mv::um::commit(br.o_done + 8);
+    release(ev);
+    if (more) {
+      issue_qk(s1, q1, slot_addr(ek));
+      mv::um::commit(br.s_full + 8);
+      release(ek);
+    }
+  }
+}
+
+// One softmax group = 128 threads = the 128 query rows of head `i` (0 or 1) of the CTA.
+__device__ __forceinline__ void softmax_group(const mv::QTile& qt, const PrefillArgs& a, int i, int head, uint32_t tmem, const Bars& br,
+                                              const Waiter& w) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = (warp & 3) * 32 + lane;                   // query row of the tile = tensor-memory lane
+  const int qi = qt.q_start + r;                          // flattened index of the query
+  const uint32_t lane_base = tmem + (uint32_t((warp & 3) * 32) << 16);
+  const uint32_t s_t = lane_base + i * 128, o_t = lane_base + 256 + i * 128;
+  const uint32_t s_full = br.s_full + 8 * i, p_full = br.p_full + 8 * i, o_done = br.o_done + 8 * i;
+  TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.q_start + qt.q_len - 1);
+  float m = -INFINITY, l = 0.f;  // running maximum (log2 units) and sum of this row
+  int start, n, causal, j = 0;
+  while (it.next(start, n, causal)) {
+    w.wait(s_full, j & 1);
+    mv::um::fence_after();
+    uint32_t s[BK];
+#pragma unroll
+    for (int c = 0; c < BK / 32; ++c) mv::um::ld32(s_t + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+    mv::um::wait_ld();
+    // scale to log2 units; mask the ragged end of the range and, on diagonal tiles, keys after the query
+    const bool need_mask = (n < BK) || (causal && start + BK - 1 > qt.q_start);
+    float mx = -INFINITY;
+    if (!need_mask) {
+#pragma unroll
+      for (int c = 0; c < BK; ++c) {
+        const float v = __uint_as_float(s[c]) * a.scale_log2;
+        s[c] = __float_as_uint(v);
+        mx = fmaxf(mx, v);
+      }
+    } else {
+      const int lim = causal ? min(n, qi - start + 1) : n;  // keys [0, lim) of the tile are visible to this row
+#pragma unroll
+      for (int c = 0; c < BK; ++c) {
+        const float v = c < lim ? __uint_as_float(s[c]) * a.scale_log2 : -INFINITY;
+        s[c] = __float_as_uint(v);
+        mx = fmaxf(mx, v);
+      }
+    }
+    // the row's reference maximum moves only when it would otherwise let P grow past 2^8
+    const bool move = mx > m + RESCALE_THRESHOLD || (m == -INFINITY && mx > -INFINITY);
+    if (j > 0 && __any_sync(0xffffffffu, move)) {
+      const float f = (move && m != -INFINITY) ? mv::fast_exp2(m - mx) : 1.f;
+      w.wait(o_done, (j - 1) & 1);  // O_i holds tiles 0 .. j-1 and no product is writing it
+      mv::um::fence_after();
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o[32];
+        mv::um::ld32(o_t + c * 32, o);
+        mv::um::wait_ld();
+#pragma unroll
+        for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * f);
+        mv::um::st32(o_t + c * 32, o);
+      }
+      l *= f;
+    }
+    if (move) m = mx;
+    const float mref = (m == -INFINITY) ? 0.f : m;
+    float sum = 0.f;
+    uint32_t pk[BK / 2];
+#pragma unroll
+    for (int c = 0; c < BK / 2; ++c) {
+      const float p0 = mv::fast_exp2(__uint_as_float(s[2 * c]) - mref), p1 = mv::fast_exp2(__uint_as_float(s[2 * c + 1]) - mref);
+      sum += p0 + p1;
+      pk[c] = mv::pack_bf16(p0, p1);
+    }
+    l += sum;
+    mv::um::st32(s_t, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+    mv::um::st32(s_t + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+    mv::um::wait_st();
+    mv::um::fence_before();
+    mv::mbar_arrive(p_full);  // P_i (and a rescaled O_i) are in place for this tile's second product
+    ++j;
+  }
+  if (j == 0) return;
+  w.wait(o_done, (j - 1) & 1);
+  mv::um::fence_after();
+  const float inv = 1.f / l;
+  bf16* dst = a.out + (int64_t(qi) * a.Hq + head) * D;
+#pragma unroll
+  for (int c = 0; c < D / 32; ++c) {
+    uint32_t o[32];
+    mv::um::ld32(o_t + c * 32, o);
+    mv::um::wait_ld();
+    if (r < qt.q_len) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint4 v;
+        v.x = mv::pack_bf16(__uint_as_float(o[8 * k]) * inv, __uint_as_float(o[8 * k + 1]) * inv);
+        v.y = mv::pack_bf16(__uint_as_float(o[8 * k + 2]) * inv, __uint_as_float(o[8 * k + 3]) * inv);
+        v.z = mv::pack_bf16(__uint_as_float(o[8 * k + 4]) * inv, __uint_as_float(o[8 * k + 5]) * inv);
+        v.w = mv::pack_bf16(__uint_as_float(o[8 * k + 6]) * inv, __uint_as_float(o[8 * k + 7]) * inv);
+        *reinterpret_cast<uint4*>(dst + c * 32 + k * 8) = v;
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1) prefill_tc_kernel(const PrefillArgs a, const __grid_constant__ CUtensorMap tm_q,
+                                                                 const __grid_constant__ CUtensorMap tm_k,
+                                                                 const __grid_constant__ CUtensorMap tm_v) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const uint32_t smem_base = mv::smem_u32(smem);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 200);
+  int* abort_flag = reinterpret_cast<int*>(smem + OFF_BAR + 208);
+  Bars br;
+  br.q_full = mv::smem_u32(&bars[0]);
+  br.kv_full = mv::smem_u32(&bars[1]);
+  br.kv_empty = mv::smem_u32(&bars[1 + RING]);
+  br.s_full = mv::smem_u32(&bars[1 + 2 * RING]);
+  br.p_full = mv::smem_u32(&bars[3 + 2 * RING]);
+  br.o_done = mv::smem_u32(&bars[5 + 2 * RING]);
+  if ((smem_base & 1023u) != 0) {  // the swizzle pattern is anchored at 1024-byte boundaries
+    if (tid == 0) atomicExch(a.status, int(MV_ERR_UNSUPPORTED));
+    return;
+  }
+  if (tid == 0) {
+    *abort_flag = 0;
+    mv::mbar_init(br.q_full, 1);
+    for (int i = 0; i < RING; ++i) {
+      mv::mbar_init(br.kv_full + 8 * i, 1);
+      mv::mbar_init(br.kv_empty + 8 * i, 1);  // one tcgen05.commit
+    }
+    for (int i = 0; i < 2; ++i) {
+      mv::mbar_init(br.s_full + 8 * i, 1);    // one tcgen05.commit
+      mv::mbar_init(br.p_full + 8 * i, 128);  // every thread of the softmax group
+      mv::mbar_init(br.o_done + 8 * i, 1);    // one tcgen05.commit
+    }
+    mv::mbar_fence_init();
+    mv::fence_proxy_async();
+  }
+  if (warp == 2) {  // the whole tensor memory of the SM: S0 S1 O0 O1, 128 columns each
+    mv::um::tmem_alloc(mv::smem_u32(tmem_slot), 512);
+    mv::um::tmem_relinquish();
+  }
+  mv::um::fence_before();
+  __syncthreads();
+  mv::um::fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const mv::QTile qt = a.q_tiles[blockIdx.x];
+  const int h0 = blockIdx.y * 2, kvh = h0 / a.G;
+  Waiter w{abort_flag, a.status};
+  if (warp < 4) {
+    mv::um::reg_dec<48>();
+    if (warp == 0) producer_warp(qt, a, h0, kvh, smem_base, br, w, &tm_q, &tm_k, &tm_v);
+    else if (warp == 1) mma_warp(qt, a, smem_base, tmem, br, w);
+  } else {
+    mv::um::reg_inc<224>();
+    const int i = (warp - 4) >> 2;
+    softmax_group(qt, a, i, h0 + i, tmem, br, w);
+  }
+  mv::um::fence_before();
+  __syncthreads();
+  if (warp == 2) mv::um::tmem_dealloc(tmem, 512);
+}
+
+struct TcMaps {  // the last problem's tensor maps (pointers and token count rarely change between calls)
+  const void *q = nullptr, *k = nullptr, *v = nullptr;
+  int64_t T = 0;
+  int Hq = 0, Hkv = 0;
+  CUtensorMap tm_q, tm_k, tm_v;
+};
+
+}  // namespace
+
+namespace mv {
+// Tensor-core prefill for head_dim 128 and an even group size; the caller has validated the arguments.
+mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return MV_ERR_CUDA;
+    }
+    attr_set = true;
+  }
+  const int64_t T = P->stats.n_new_tokens;
+  static thread_local TcMaps tc;
+  if (!(tc.q == q && tc.k == k && tc.v == v && tc.T == T && tc.Hq == g->n_q_heads && tc.Hkv == g->n_kv_heads)) {
+    tc.q = nullptr;
+    if (!mv::make_tmap_bf16_2d(&tc.tm_q, q, uint64_t(T), uint64_t(g->n_q_heads) * D, BQ) ||
+        !mv::make_tmap_bf16_2d(&tc.tm_k, k, uint64_t(T), uint64_t(g->n_kv_heads) * D, BK) ||
+        !mv::make_tmap_bf16_2d(&tc.tm_v, v, uint64_t(T), uint64_t(g->n_kv_heads) * D, BK))
+      return MV_ERR_CUDA;
+    tc.q = q; tc.k = k; tc.v = v; tc.T = T; tc.Hq = g->n_q_heads; tc.Hkv = g->n_kv_heads;
+  }
+  PrefillArgs a;
+  a.q_tiles = mv::table<mv::QTile>(P, P->layout.q_tiles);
+  a.ranges = mv::table<mv::KvRange>(P, P->layout.kv_ranges);
+  a.out = static_cast<bf16*>(out);
+  a.status = const_cast<int32_t*>(mv::table<int32_t>(P, P->layout.sched)) + 2;
+  a.Hq = g->n_q_heads;
+  a.G = g->n_q_heads / g->n_kv_heads;
+  a.scale_log2 = mv::softmax_scale(g) * 1.4426950408889634f;
+  dim3 grid(unsigned(P->stats.n_q_tiles), unsigned(g->n_q_heads / 2));
+  prefill_tc_kernel<<<grid, NTHREADS, SMEM_BYTES, st>>>(a, tc.tm_q, tc.tm_k, tc.tm_v);
+  mv::g_launches++;
+  return cudaGetLastError() == cudaSuccess ? MV_OK : MV_ERR_CUDA;
+}
+}  // namespace mv
