@@ -103,20 +103,19 @@ __device__ __forceinline__ void producer_warp(const mv::QTile& qt, const Prefill
   }
 }
 
-// S_i = Q_i K^T: both operands K-major, eight 16-element k-steps
-__device__ __forceinline__ void issue_qk(uint32_t s_tmem, uint32_t q_smem, uint32_t k_smem) {
-  constexpr uint32_t idesc = mv::um::idesc_bf16(BQ, BK, 0, 0);
+// S_i = Q_i K^T over the first n_cols keys of the tile (a multiple of 32): both operands K-major, eight k-steps
+__device__ __forceinline__ void issue_qk(uint32_t s_tmem, uint32_t q_smem, uint32_t k_smem, int n_cols) {
+  const uint32_t idesc = mv::um::idesc_bf16(BQ, n_cols, 0, 0);
 #pragma unroll
   for (int k = 0; k < D / 16; ++k) {
     const uint32_t off = (k >> 2) * (TILE_BYTES / 2) + (k & 3) * 32;
     mv::um::mma_ss(s_tmem, mv::um::smem_desc(q_smem + off, 16, 1024), mv::um::smem_desc(k_smem + off, 16, 1024), idesc, k > 0);
   }
 }
-// O_i (+)= P_i V: P from tensor memory (two bf16 per column), V MN-major, eight 16-key k-steps
-__device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_smem, bool accumulate) {
+// O_i (+)= P_i V over the first k_steps * 16 keys: P from tensor memory (two bf16 per column), V MN-major
+__device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_smem, bool accumulate, int k_steps) {
   constexpr uint32_t idesc = mv::um::idesc_bf16(BQ, D, 0, 1);
-#pragma unroll
-  for (int k = 0; k < BK / 16; ++k)
+  for (int k = 0; k < k_steps; ++k)
     mv::um::mma_ts(o_tmem, p_tmem + k * 8, mv::um::smem_desc(v_smem + k * 2048, TILE_BYTES / 2, 1024), idesc, accumulate || k > 0);
 }
 
@@ -124,47 +123,48 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
                                          const Waiter& w) {
   if ((threadIdx.x & 31) != 0) return;
   TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.q_start + qt.q_len - 1);
-  int start, n, c;
-  int n_tiles = 0;
-  while (it.next(start, n, c)) ++n_tiles;
-  if (n_tiles == 0) return;
+  int start, n_cur, n_next = 0, c;
+  if (!it.next(start, n_cur, c)) return;
+  bool more = it.next(start, n_next, c);
   const uint32_t q0 = smem_base + OFF_Q, q1 = q0 + TILE_BYTES;
   const uint32_t s0 = tmem, s1 = tmem + 128, o0 = tmem + 256, o1 = tmem + 384;
   auto slot_addr = [&](int e) { return smem_base + OFF_RING + (e % RING) * TILE_BYTES; };
   auto wait_full = [&](int e) { w.wait(br.kv_full + 8 * (e % RING), (e / RING) & 1); };
   auto release = [&](int e) { mv::um::commit(br.kv_empty + 8 * (e % RING)); };
+  auto cols = [](int n) { return ((n + 15) >> 4) << 4; };  // score columns computed; the softmax groups mask the rest
   w.wait(br.q_full, 0);
   wait_full(0);
   mv::um::fence_after();
-  issue_qk(s0, q0, slot_addr(0));
+  issue_qk(s0, q0, slot_addr(0), cols(n_cur));
   mv::um::commit(br.s_full);
-  issue_qk(s1, q1, slot_addr(0));
+  issue_qk(s1, q1, slot_addr(0), cols(n_cur));
   mv::um::commit(br.s_full + 8);
   release(0);
-  for (int j = 0; j < n_tiles; ++j) {
+  for (int j = 0;; ++j) {
     const int ev = 2 * j + 1, ek = 2 * j + 2;  // ring entries of V_j and K_{j+1}
-    const bool more = j + 1 < n_tiles;
+    const int k_steps = (n_cur + 15) >> 4;
     wait_full(ev);
     w.wait(br.p_full, j & 1);
     mv::um::fence_after();
-    issue_pv(o0, s0, slot_addr(ev), j > 0);
+    issue_pv(o0, s0, slot_addr(ev), j > 0, k_steps);
     mv::um::commit(br.o_done);
     if (more) {
       wait_full(ek);
       mv::um::fence_after();
-      issue_qk(s0, q0, slot_addr(ek));
+      issue_qk(s0, q0, slot_addr(ek), cols(n_next));
       mv::um::commit(br.s_full);
     }
     w.wait(br.p_full + 8, j & 1);
     mv::um::fence_after();
-    issue_pv(o1, s1, slot_addr(ev), j > 0);
+    issue_pv(o1, s1, slot_addr(ev), j > 0, k_steps);
     mv::um::commit(br.o_done + 8);
     release(ev);
-    if (more) {
-      issue_qk(s1, q1, slot_addr(ek));
-      mv::um::commit(br.s_full + 8);
-      release(ek);
-    }
+    if (!more) break;
+    issue_qk(s1, q1, slot_addr(ek), cols(n_next));
+    mv::um::commit(br.s_full + 8);
+    release(ek);
+    n_cur = n_next;
+    more = it.next(start, n_next, c);
   }
 }
 
@@ -183,29 +183,28 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
   while (it.next(start, n, causal)) {
     w.wait(s_full, j & 1);
     mv::um::fence_after();
+    // all 128 columns are read: on a ragged tile the issuer computed only the leading ones, the rest holds an
+    // older tile's scores and is masked below
     uint32_t s[BK];
 #pragma unroll
     for (int c = 0; c < BK / 32; ++c) mv::um::ld32(s_t + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
     mv::um::wait_ld();
-    // scale to log2 units; mask the ragged end of the range and, on diagonal tiles, keys after the query
-    const bool need_mask = (n < BK) || (causal && start + BK - 1 > qt.q_start);
-    float mx = -INFINITY;
+    // mask the ragged end of the range and, on diagonal tiles, keys after the query; row maximum of the raw
+    // scores with four independent chains (the softmax scale is positive, so it commutes with the maximum)
+    const bool need_mask = n < BK || (causal && start + BK - 1 > qt.q_start);
+    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
     if (!need_mask) {
 #pragma unroll
-      for (int c = 0; c < BK; ++c) {
-        const float v = __uint_as_float(s[c]) * a.scale_log2;
-        s[c] = __float_as_uint(v);
-        mx = fmaxf(mx, v);
-      }
+      for (int c = 0; c < BK; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(s[c]));
     } else {
       const int lim = causal ? min(n, qi - start + 1) : n;  // keys [0, lim) of the tile are visible to this row
 #pragma unroll
       for (int c = 0; c < BK; ++c) {
-        const float v = c < lim ? __uint_as_float(s[c]) * a.scale_log2 : -INFINITY;
-        s[c] = __float_as_uint(v);
-        mx = fmaxf(mx, v);
+        if (c >= lim) s[c] = __float_as_uint(-INFINITY);
+        mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(s[c]));
       }
     }
+    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
     // the row's reference maximum moves only when it would otherwise let P grow past 2^8
     const bool move = mx > m + RESCALE_THRESHOLD || (m == -INFINITY && mx > -INFINITY);
     if (j > 0 && __any_sync(0xffffffffu, move)) {
@@ -225,17 +224,17 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
     }
     if (move) m = mx;
     const float mref = (m == -INFINITY) ? 0.f : m;
-    float sum = 0.f;
-    uint32_t pk[BK / 2];
+    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int c = 0; c < BK / 2; ++c) {
-      const float p0 = mv::fast_exp2(__uint_as_float(s[2 * c]) - mref), p1 = mv::fast_exp2(__uint_as_float(s[2 * c + 1]) - mref);
-      sum += p0 + p1;
-      pk[c] = mv::pack_bf16(p0, p1);
+    for (int c = 0; c < BK / 2; ++c) {  // P over S in place: columns 2c, 2c+1 -> packed column c
+      const float p0 = mv::fast_exp2(fmaf(__uint_as_float(s[2 * c]), a.scale_log2, -mref));
+      const float p1 = mv::fast_exp2(fmaf(__uint_as_float(s[2 * c + 1]), a.scale_log2, -mref));
+      sum4[c & 3] += p0 + p1;
+      s[c] = mv::pack_bf16(p0, p1);
     }
-    l += sum;
-    mv::um::st32(s_t, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-    mv::um::st32(s_t + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+    l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+    mv::um::st32(s_t, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+    mv::um::st32(s_t + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
     mv::um::wait_st();
     mv::um::fence_before();
     mv::mbar_arrive(p_full);  // P_i (and a rescaled O_i) are in place for this tile's second product
