@@ -40,6 +40,7 @@ struct DecodeArgs {
   const mv::StageDesc* stages;
   const mv::WorkUnit* units;
   const int32_t* cta_unit_off;
+  const mv::WorkUnit* cta_head;  // each CTA's first unit with its unit range in pad[0], pad[1]
   const mv::ItemRow* item_rows;
   float* part_o;    // [n_partials * G][D]
   float* part_ml;   // [n_partials * G][2]  (max in log2 units, sum)
@@ -110,9 +111,19 @@ struct StageRegs {  // one stage descriptor per lane (a window of 32 stages)
 };
 
 template <int D>
-__device__ __forceinline__ void producer(const DecodeArgs& a, int u_begin, int u_end, uint32_t smem_base, Meta* meta, const Sync& sy,
-                                         const CUtensorMap* tm_k, const CUtensorMap* tm_v) {
+__device__ __forceinline__ void producer(const DecodeArgs& a, uint32_t smem_base, Meta* meta, const Sync& sy, const CUtensorMap* tm_k,
+                                         const CUtensorMap* tm_v) {
   const int lane = threadIdx.x & 31;
+  // one load at a known address gives the CTA's unit range and its first unit
+  UnitRegs wu;
+  int u_begin, u_end;
+  {
+    const int4* p = reinterpret_cast<const int4*>(a.cta_head + blockIdx.x);
+    const int4 x = __ldg(p), y = __ldg(p + 1);
+    wu.stage_begin = x.x; wu.n_stages = x.y; wu.row_begin = x.z; wu.n_rows = x.w; wu.kvh = y.x;
+    u_begin = y.y;
+    u_end = y.z;
+  }
   int issued = 0;  // stages issued so far (buffer = issued % NSTAGES)
   // Table reads run ahead of their use so that no load sits on the issue path: the descriptor of unit u + 2,
   // and the row list and first stage window of unit u + 1, are requested while unit u is being issued.
@@ -139,7 +150,7 @@ __device__ __forceinline__ void producer(const DecodeArgs& a, int u_begin, int u
     }
     return r;
   };
-  UnitRegs wu = load_unit(u_begin), wu1 = load_unit(u_begin + 1);
+  UnitRegs wu1 = load_unit(u_begin + 1);
   mv::ItemRow ir0 = load_rows(wu, 0), ir1 = load_rows(wu, 32);
   StageRegs win = load_window(wu, 0);
   for (int u = u_begin; u < u_end; ++u) {
@@ -495,12 +506,12 @@ __global__ void __launch_bounds__(NTHREADS, 2) decode_attn_kernel(const DecodeAr
     mv::fence_proxy_async();
   }
   __syncthreads();
-  const int u_begin = a.cta_unit_off[blockIdx.x], u_end = a.cta_unit_off[blockIdx.x + 1];
   if (warp == 4) {
-    producer<D>(a, u_begin, u_end, smem_base, meta, sy, &tm_k, &tm_v);
+    producer<D>(a, smem_base, meta, sy, &tm_k, &tm_v);
     mv::grid_dependency_launch_dependents();
     return;
   }
+  const int u_begin = a.cta_unit_off[blockIdx.x], u_end = a.cta_unit_off[blockIdx.x + 1];
   int consumed = 0;
   for (int u = u_begin; u < u_end; ++u) {
     wait_or_flag(sy, sy.q_full, (u - u_begin) & 1);
@@ -525,29 +536,44 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const float* __restri
   const int Hkv = Hq / G;
   const int p0 = rowkv_part_off[row * Hkv + kvh], p1 = rowkv_part_off[row * Hkv + kvh + 1];
   mv::grid_dependency_wait();  // the partials are complete and visible from here on
-  float m = -INFINITY;
-  for (int p = p0 + lane; p < p1; p += 32) m = fmaxf(m, part_ml[(int64_t(p) * G + g) * 2]);
-#pragma unroll
-  for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+  // online merge, four partials per step: the loads of a step do not depend on one another, so a (row, head)
+  // with up to four partials costs one round trip to L2
   constexpr int E = D / 32;
+  float m = -INFINITY, l = 0.f;
   float acc[E];
 #pragma unroll
   for (int e = 0; e < E; ++e) acc[e] = 0.f;
-  float l = 0.f;
-#pragma unroll 4
-  for (int p = p0; p < p1; ++p) {
-    const int64_t ps = int64_t(p) * G + g;
-    const float2 ml = *reinterpret_cast<const float2*>(part_ml + ps * 2);
-    const float wgt = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - m);
-    l += wgt * ml.y;
-    const float* po = part_o + ps * D + lane * E;
-    if (E == 4) {
-      const float4 t = *reinterpret_cast<const float4*>(po);
-      acc[0] += wgt * t.x; acc[1] += wgt * t.y; acc[2] += wgt * t.z; acc[3 % E] += wgt * t.w;
-    } else {
-      const float2 t = *reinterpret_cast<const float2*>(po);
-      acc[0] += wgt * t.x; acc[1] += wgt * t.y;
+  for (int pb = p0; pb < p1; pb += 4) {
+    float2 ml[4];
+    float t[4][E];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const bool ok = pb + k < p1;
+      const int64_t ps = int64_t(ok ? pb + k : pb) * G + g;
+      ml[k] = *reinterpret_cast<const float2*>(part_ml + ps * 2);
+      if (!ok) ml[k].x = -INFINITY;
+      const float* po = part_o + ps * D + lane * E;
+      if (E == 4) {
+        const float4 v = *reinterpret_cast<const float4*>(po);
+        t[k][0] = v.x; t[k][1] = v.y; t[k][2 % E] = v.z; t[k][3 % E] = v.w;
+      } else {
+        const float2 v = *reinterpret_cast<const float2*>(po);
+        t[k][0] = v.x; t[k][1] = v.y;
+      }
     }
+    const float mn = fmaxf(fmaxf(m, fmaxf(ml[0].x, ml[1].x)), fmaxf(ml[2].x, ml[3].x));
+    const float f = (m == -INFINITY) ? 0.f : exp2f(m - mn);
+    l *= f;
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[e] *= f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float wgt = (ml[k].x == -INFINITY) ? 0.f : exp2f(ml[k].x - mn);
+      l += wgt * ml[k].y;
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[e] += wgt * t[k][e];
+    }
+    m = mn;
   }
   const float inv = 1.f / l;
   bf16* o = out + (int64_t(row) * Hq + h) * D + lane * E;
@@ -597,6 +623,7 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
   a.stages = mv::table<mv::StageDesc>(P, P->layout.stages);
   a.units = mv::table<mv::WorkUnit>(P, P->layout.units);
   a.cta_unit_off = mv::table<int32_t>(P, P->layout.cta_unit_off);
+  a.cta_head = mv::table<mv::WorkUnit>(P, P->layout.cta_head);
   a.item_rows = mv::table<mv::ItemRow>(P, P->layout.item_rows);
   a.part_o = static_cast<float*>(ws);
   a.part_ml = reinterpret_cast<float*>(static_cast<char*>(ws) + o_bytes);

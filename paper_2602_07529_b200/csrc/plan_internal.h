@@ -48,7 +48,7 @@ struct KvRange {
 };
 
 struct DeviceLayout {  // byte offsets into the device table buffer (all multiples of 256)
-  size_t pos_id = 0, slot = 0, stages = 0, units = 0, cta_unit_off = 0, item_rows = 0, rowkv_part_off = 0, sched = 0,
+  size_t pos_id = 0, slot = 0, stages = 0, units = 0, cta_unit_off = 0, cta_head = 0, item_rows = 0, rowkv_part_off = 0, sched = 0,
          q_tiles = 0, kv_ranges = 0, total = 0;
 };
 
@@ -62,6 +62,7 @@ struct mv_plan {
   std::vector<mv::StageDesc> stages;
   std::vector<mv::WorkUnit> units;       // CTA by CTA
   std::vector<int32_t> cta_unit_off;     // [n_ctas + 1]
+  std::vector<mv::WorkUnit> cta_head;    // [n_ctas] copy of each CTA's first unit; pad[0], pad[1] = its unit range
   std::vector<mv::ItemRow> item_rows;
   std::vector<int32_t> rowkv_part_off;   // [n_rows * n_kv_heads + 1] CSR over the partial slots of a (row, KV head)
   int32_t sched_zero[64] = {};  // device-side status words ([2] = status of bounded waits), uploaded as zeros

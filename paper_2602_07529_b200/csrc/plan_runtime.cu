@@ -50,6 +50,7 @@ extern "C" mv_status mv_plan_upload(mv_plan* P, void* device_buf, size_t device_
   put(h, L.stages, P->stages);
   put(h, L.units, P->units);
   put(h, L.cta_unit_off, P->cta_unit_off);
+  put(h, L.cta_head, P->cta_head);
   put(h, L.item_rows, P->item_rows);
   put(h, L.rowkv_part_off, P->rowkv_part_off);
   std::memcpy(h + L.sched, P->sched_zero, sizeof(P->sched_zero));

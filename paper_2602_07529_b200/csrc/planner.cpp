@@ -104,7 +104,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   P->qnode_tok_off.assign(1, 0);
   P->seg_off.assign(1, 0);
   P->seg_node.clear(); P->seg_len.clear(); P->kv_len.clear();
-  P->units.clear(); P->cta_unit_off.clear(); P->item_rows.clear(); P->rowkv_part_off.clear();
+  P->units.clear(); P->cta_unit_off.clear(); P->cta_head.clear(); P->item_rows.clear(); P->rowkv_part_off.clear();
   P->q_tiles.clear(); P->kv_ranges.clear();
   P->stages.clear();
   mv_plan_stats S{};
@@ -401,6 +401,13 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     }
     S.max_cta_cost = max_acc;
     for (int c = 1; c <= n_ctas; ++c) P->cta_unit_off[c] = std::max(P->cta_unit_off[c], P->cta_unit_off[c - 1]);
+    P->cta_head.assign(size_t(n_ctas), WorkUnit{});
+    for (int c = 0; c < n_ctas; ++c) {
+      const int32_t ub = P->cta_unit_off[c], ue = P->cta_unit_off[c + 1];
+      if (ub < ue) P->cta_head[size_t(c)] = P->units[size_t(ub)];
+      P->cta_head[size_t(c)].pad[0] = ub;
+      P->cta_head[size_t(c)].pad[1] = ue;
+    }
     // partial slots: contiguous per (row, KV head), in unit order
     P->rowkv_part_off.assign(size_t(n_rows) * sched_kv_heads + 1, 0);
     for (const PartKey& k : keys) P->rowkv_part_off[size_t(k.rowkv) + 1]++;
@@ -449,6 +456,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   L.stages = place(P->stages.size() * sizeof(StageDesc));
   L.units = place(P->units.size() * sizeof(WorkUnit));
   L.cta_unit_off = place(P->cta_unit_off.size() * sizeof(int32_t));
+  L.cta_head = place(P->cta_head.size() * sizeof(WorkUnit));
   L.item_rows = place(P->item_rows.size() * sizeof(ItemRow));
   L.rowkv_part_off = place(P->rowkv_part_off.size() * sizeof(int32_t));
   L.sched = place(sizeof(P->sched_zero));
