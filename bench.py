@@ -315,7 +315,7 @@ def run_ours(args):
                    "parallelism": (f"{world} ranks, one batch each, sharded by request, no collective" if world > 1 else "single")},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                     "peak_source": peaks["source"], "kernel": "decode_attn_kernel + decode_merge_kernel (one mv_dag_decode_attn call)",
+                     "peak_source": peaks["source"], "kernel": "decode_attn_kernel + decode_merge_kernel (one mv_dag_decode_attn call; the traffic figure is decode_attn_kernel alone)",
                      "algorithmic_bytes": algo_bytes, "launch_ms_mean": decode_ms, "launch_ms_min": decode_ms_min,
                      "frac_of_nominal_8TBs": achieved / 8000.0, "naive_per_row_GBs": naive_bytes / (decode_ms * 1e-3) / 1e9,
                      "decode_query_tokens_per_s": rows / (decode_ms * 1e-3)},
