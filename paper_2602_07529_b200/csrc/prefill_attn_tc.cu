@@ -50,12 +50,16 @@ struct TileIter {
   const mv::KvRange* rg;
   int n_ranges, q_last;
   int ri = 0, pos = 0, end = 0, causal = 0;
-  __device__ TileIter(const mv::KvRange* r, int n, int ql) : rg(r), n_ranges(n), q_last(ql) {}
+  mv::KvRange nxt;  // the range after the current one, read one range ahead so that no load sits on the walk
+  __device__ TileIter(const mv::KvRange* r, int n, int ql) : rg(r), n_ranges(n), q_last(ql) {
+    nxt = n > 0 ? r[0] : mv::KvRange{0, 0, 0, 0};
+  }
   // start key, valid keys (1..128), causal flag of the next tile; false when the walk is over
   __device__ bool next(int& start, int& n, int& c) {
     while (pos >= end) {
       if (ri >= n_ranges) return false;
-      const mv::KvRange r = rg[ri++];
+      const mv::KvRange r = nxt;
+      if (++ri < n_ranges) nxt = rg[ri];
       pos = r.kv_start;
       end = r.kv_start + r.kv_len;
       causal = r.causal;
@@ -103,20 +107,25 @@ __device__ __forceinline__ void producer_warp(const mv::QTile& qt, const Prefill
   }
 }
 
-// S_i = Q_i K^T over the first n_cols keys of the tile (a multiple of 32): both operands K-major, eight k-steps
-__device__ __forceinline__ void issue_qk(uint32_t s_tmem, uint32_t q_smem, uint32_t k_smem, int n_cols) {
+// S_i = Q_i K^T over the first n_cols keys of the tile (a multiple of 16): both operands K-major, eight k-steps.
+// A descriptor's start address sits in its low bits in 16-byte units, so a k-step is one addition.
+__device__ __forceinline__ void issue_qk(uint32_t s_tmem, uint64_t q_desc, uint64_t k_desc, int n_cols) {
   const uint32_t idesc = mv::um::idesc_bf16(BQ, n_cols, 0, 0);
+  mv::um::mma_ss<false>(s_tmem, q_desc, k_desc, idesc);
 #pragma unroll
-  for (int k = 0; k < D / 16; ++k) {
-    const uint32_t off = (k >> 2) * (TILE_BYTES / 2) + (k & 3) * 32;
-    mv::um::mma_ss(s_tmem, mv::um::smem_desc(q_smem + off, 16, 1024), mv::um::smem_desc(k_smem + off, 16, 1024), idesc, k > 0);
+  for (int k = 1; k < D / 16; ++k) {
+    const uint32_t off = ((k >> 2) * (TILE_BYTES / 2) + (k & 3) * 32) >> 4;
+    mv::um::mma_ss<true>(s_tmem, q_desc + off, k_desc + off, idesc);
   }
 }
 // O_i (+)= P_i V over the first k_steps * 16 keys: P from tensor memory (two bf16 per column), V MN-major
-__device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_smem, bool accumulate, int k_steps) {
+__device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint64_t v_desc, bool accumulate, int k_steps) {
   constexpr uint32_t idesc = mv::um::idesc_bf16(BQ, D, 0, 1);
-  for (int k = 0; k < k_steps; ++k)
-    mv::um::mma_ts(o_tmem, p_tmem + k * 8, mv::um::smem_desc(v_smem + k * 2048, TILE_BYTES / 2, 1024), idesc, accumulate || k > 0);
+  if (accumulate) mv::um::mma_ts<true>(o_tmem, p_tmem, v_desc, idesc);
+  else mv::um::mma_ts<false>(o_tmem, p_tmem, v_desc, idesc);
+#pragma unroll
+  for (int k = 1; k < BK / 16; ++k)
+    if (k < k_steps) mv::um::mma_ts<true>(o_tmem, p_tmem + k * 8, v_desc + uint32_t((k * 2048) >> 4), idesc);
 }
 
 __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs& a, uint32_t smem_base, uint32_t tmem, const Bars& br,
@@ -126,18 +135,19 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
   int start, n_cur, n_next = 0, c;
   if (!it.next(start, n_cur, c)) return;
   bool more = it.next(start, n_next, c);
-  const uint32_t q0 = smem_base + OFF_Q, q1 = q0 + TILE_BYTES;
+  const uint64_t q0 = mv::um::smem_desc(smem_base + OFF_Q, 16, 1024), q1 = mv::um::smem_desc(smem_base + OFF_Q + TILE_BYTES, 16, 1024);
   const uint32_t s0 = tmem, s1 = tmem + 128, o0 = tmem + 256, o1 = tmem + 384;
-  auto slot_addr = [&](int e) { return smem_base + OFF_RING + (e % RING) * TILE_BYTES; };
+  auto k_desc = [&](int e) { return mv::um::smem_desc(smem_base + OFF_RING + (e % RING) * TILE_BYTES, 16, 1024); };
+  auto v_desc = [&](int e) { return mv::um::smem_desc(smem_base + OFF_RING + (e % RING) * TILE_BYTES, TILE_BYTES / 2, 1024); };
   auto wait_full = [&](int e) { w.wait(br.kv_full + 8 * (e % RING), (e / RING) & 1); };
   auto release = [&](int e) { mv::um::commit(br.kv_empty + 8 * (e % RING)); };
   auto cols = [](int n) { return ((n + 15) >> 4) << 4; };  // score columns computed; the softmax groups mask the rest
   w.wait(br.q_full, 0);
   wait_full(0);
   mv::um::fence_after();
-  issue_qk(s0, q0, slot_addr(0), cols(n_cur));
+  issue_qk(s0, q0, k_desc(0), cols(n_cur));
   mv::um::commit(br.s_full);
-  issue_qk(s1, q1, slot_addr(0), cols(n_cur));
+  issue_qk(s1, q1, k_desc(0), cols(n_cur));
   mv::um::commit(br.s_full + 8);
   release(0);
   for (int j = 0;; ++j) {
@@ -146,21 +156,21 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
     wait_full(ev);
     w.wait(br.p_full, j & 1);
     mv::um::fence_after();
-    issue_pv(o0, s0, slot_addr(ev), j > 0, k_steps);
+    issue_pv(o0, s0, v_desc(ev), j > 0, k_steps);
     mv::um::commit(br.o_done);
     if (more) {
       wait_full(ek);
       mv::um::fence_after();
-      issue_qk(s0, q0, slot_addr(ek), cols(n_next));
+      issue_qk(s0, q0, k_desc(ek), cols(n_next));
       mv::um::commit(br.s_full);
     }
     w.wait(br.p_full + 8, j & 1);
     mv::um::fence_after();
-    issue_pv(o1, s1, slot_addr(ev), j > 0, k_steps);
+    issue_pv(o1, s1, v_desc(ev), j > 0, k_steps);
     mv::um::commit(br.o_done + 8);
     release(ev);
     if (!more) break;
-    issue_qk(s1, q1, slot_addr(ek), cols(n_next));
+    issue_qk(s1, q1, k_desc(ek), cols(n_next));
     mv::um::commit(br.s_full + 8);
     release(ek);
     n_cur = n_next;
