@@ -26,6 +26,11 @@
 
 #include "common.cuh"
 
+namespace mv {
+mv_status decode_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* kp, const void* vp, void* ws,
+                    cudaStream_t st);
+}
+
 namespace {
 
 using bf16 = __nv_bfloat16;
@@ -632,9 +637,19 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
   a.G = G;
   a.scale_log2 = mv::softmax_scale(g) * 1.4426950408889634f;
   a.Hkv = g->n_kv_heads;
-  decode_attn_kernel<D><<<unsigned(P->stats.n_ctas), NTHREADS, Cfg<D>::SMEM, st>>>(a, hit->tm_k, hit->tm_v);
-  mv::g_launches++;
-  if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
+#ifndef MV_DECODE_TC_MIN_QV
+#define MV_DECODE_TC_MIN_QV 17
+#endif
+  // units of more than one m16 tile of q-vectors go to the tcgen05 kernel (head_dim 128): there the legacy
+  // tensor path and the shared-memory re-reads of every consumer warp would set the pace instead of HBM
+  if (D == 128 && P->stats.max_item_rows * G >= MV_DECODE_TC_MIN_QV) {
+    const mv_status ts = mv::decode_tc(P, g, q, kp, vp, ws, st);
+    if (ts != MV_OK) return ts;
+  } else {
+    decode_attn_kernel<D><<<unsigned(P->stats.n_ctas), NTHREADS, Cfg<D>::SMEM, st>>>(a, hit->tm_k, hit->tm_v);
+    mv::g_launches++;
+    if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
+  }
   // the merge kernel is launched with programmatic stream serialisation: it may become resident while the
   // attention kernel is still running and waits (griddepcontrol.wait) for that grid to complete
   const int n_rows = int(P->stats.n_new_tokens);
