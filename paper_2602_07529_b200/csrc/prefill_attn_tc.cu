@@ -205,7 +205,7 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
     if (!need_mask) {
 #pragma unroll
-      for (int c = 0; c < BK; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(s[c]));
+      for (int c = 0; c < BK; c += 2) mx4[(c >> 1) & 3] = mv::max3(mx4[(c >> 1) & 3], __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
     } else {
       const int lim = causal ? min(n, qi - start + 1) : n;  // keys [0, lim) of the tile are visible to this row
 #pragma unroll
@@ -234,15 +234,22 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
     }
     if (move) m = mx;
     const float mref = (m == -INFINITY) ? 0.f : m;
-    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+    // packed-pair arithmetic: one FMA and one add per two scores, so that instruction issue does not pace the group
+    const uint64_t scale2 = mv::pack_f32x2(a.scale_log2, a.scale_log2), nmref2 = mv::pack_f32x2(-mref, -mref);
+    uint64_t sum2[4] = {0, 0, 0, 0};  // four independent chains of (even column, odd column) sums
 #pragma unroll
     for (int c = 0; c < BK / 2; ++c) {  // P over S in place: columns 2c, 2c+1 -> packed column c
-      const float p0 = mv::fast_exp2(fmaf(__uint_as_float(s[2 * c]), a.scale_log2, -mref));
-      const float p1 = mv::fast_exp2(fmaf(__uint_as_float(s[2 * c + 1]), a.scale_log2, -mref));
-      sum4[c & 3] += p0 + p1;
+      float x0, x1;
+      mv::unpack_f32x2(mv::fma_f32x2(mv::pack_f32x2(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1])), scale2, nmref2), x0, x1);
+      const float p0 = mv::fast_exp2(x0), p1 = mv::fast_exp2(x1);
+      sum2[c & 3] = mv::add_f32x2(sum2[c & 3], mv::pack_f32x2(p0, p1));
       s[c] = mv::pack_bf16(p0, p1);
     }
-    l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+    {
+      float e, o;
+      mv::unpack_f32x2(mv::add_f32x2(mv::add_f32x2(sum2[0], sum2[1]), mv::add_f32x2(sum2[2], sum2[3])), e, o);
+      l += e + o;
+    }
     mv::um::st32(s_t, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
     mv::um::st32(s_t + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
     mv::um::wait_st();
