@@ -338,15 +338,22 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
         }
         if (move) m = mx;
         const float mref = (m == -INFINITY) ? 0.f : m;
-        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+        // packed-pair arithmetic: one FMA and one add per two scores
+        const uint64_t scale2 = mv::pack_f32x2(a.scale_log2, a.scale_log2), nmref2 = mv::pack_f32x2(-mref, -mref);
+        uint64_t sum2[4] = {0, 0, 0, 0};
 #pragma unroll
         for (int c = 0; c < ST / 2; ++c) {  // P over S in place: columns 2c, 2c+1 -> packed column c
-          const float p0 = mv::fast_exp2(fmaf(__uint_as_float(sc[2 * c]), a.scale_log2, -mref));
-          const float p1 = mv::fast_exp2(fmaf(__uint_as_float(sc[2 * c + 1]), a.scale_log2, -mref));
-          sum4[c & 3] += p0 + p1;
+          float x0, x1;
+          mv::unpack_f32x2(mv::fma_f32x2(mv::pack_f32x2(__uint_as_float(sc[2 * c]), __uint_as_float(sc[2 * c + 1])), scale2, nmref2), x0, x1);
+          const float p0 = mv::fast_exp2(x0), p1 = mv::fast_exp2(x1);
+          sum2[c & 3] = mv::add_f32x2(sum2[c & 3], mv::pack_f32x2(p0, p1));
           sc[c] = mv::pack_bf16(p0, p1);
         }
-        l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        {
+          float e, o;
+          mv::unpack_f32x2(mv::add_f32x2(mv::add_f32x2(sum2[0], sum2[1]), mv::add_f32x2(sum2[2], sum2[3])), e, o);
+          l += e + o;
+        }
         mv::um::st32(s_t, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
         mv::um::wait_st();
       }
