@@ -637,12 +637,10 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
   a.G = G;
   a.scale_log2 = mv::softmax_scale(g) * 1.4426950408889634f;
   a.Hkv = g->n_kv_heads;
-#ifndef MV_DECODE_TC_MIN_QV
-#define MV_DECODE_TC_MIN_QV 17
-#endif
-  // units of more than one m16 tile of q-vectors go to the tcgen05 kernel (head_dim 128): there the legacy
-  // tensor path and the shared-memory re-reads of every consumer warp would set the pace instead of HBM
-  if (D == 128 && P->stats.max_item_rows * G >= MV_DECODE_TC_MIN_QV) {
+  // head_dim 128 runs on the tcgen05 kernel: the tensor core reads a stage's K / V tile once for all q-vectors and the
+  // products leave the warps' instruction streams (measured faster at every unit size: 54 vs 57 us at 16 q-vectors,
+  // 733 vs 881 us on the serving mix at up to 64); head_dim 64 keeps the mma.sync kernel of this file
+  if (D == 128) {
     const mv_status ts = mv::decode_tc(P, g, q, kp, vp, ws, st);
     if (ts != MV_OK) return ts;
   } else {

@@ -286,6 +286,11 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
     mv::mbar_arrive(bar(&meta->q_empty));  // header and slot ids are in registers
     const bool warp_active = (warp & 3) * 32 < n_qv;  // some q-vector of this warp is real
     const int row = r < n_qv ? r / a.G : -1;           // row of the unit's row group this q-vector belongs to
+    uint64_t warp_rows = 0;                            // rows that own a real q-vector of this warp
+    if (warp_active) {
+      const int r_lo = ((warp & 3) * 32) / a.G, r_hi = (min((warp & 3) * 32 + 31, n_qv - 1)) / a.G;
+      warp_rows = (r_hi - r_lo == 63 ? ~uint64_t(0) : ((uint64_t(1) << (r_hi - r_lo + 1)) - 1)) << r_lo;
+    }
     float m = -INFINITY, l = 0.f;
     for (int s = 0; s < n; ++s, ++g) {
       const int sb = g % NSTAGES, pb = g & 1;
@@ -300,18 +305,30 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
         mv::um::ld32(s_t, *reinterpret_cast<uint32_t(*)[32]>(&sc[0]));
         mv::um::ld32(s_t + 32, *reinterpret_cast<uint32_t(*)[32]>(&sc[32]));
         mv::um::wait_ld();
-        // the DAG mask at page granularity and the ragged last page of a node
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        bool plain = tok4 == 0x10101010u;  // four full pages ...
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const uint2 mk = meta->st_mask[sb][j];
-          const uint64_t seen_by = (uint64_t(mk.y) << 32) | mk.x;
-          const bool vis = row >= 0 && j < int(n_pages) && ((seen_by >> row) & 1);
-          const int lim = vis ? int((tok4 >> (8 * j)) & 0xffu) : 0;  // tokens [0, lim) of the page are visible to this q-vector
+          plain &= (((uint64_t(mk.y) << 32) | mk.x) & warp_rows) == warp_rows;  // ... seen by every real q-vector of the warp
+        }
+        if (plain) {
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            if (c >= lim) sc[j * 16 + c] = __float_as_uint(-INFINITY);
-            mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(sc[j * 16 + c]));
+          for (int c = 0; c < ST; c += 2) mx4[(c >> 1) & 3] = mv::max3(mx4[(c >> 1) & 3], __uint_as_float(sc[c]), __uint_as_float(sc[c + 1]));
+          if (row < 0) mx4[0] = mx4[1] = mx4[2] = mx4[3] = -INFINITY;  // a padding q-vector of the warp
+        } else {
+          // the DAG mask at page granularity and the ragged last page of a node
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint2 mk = meta->st_mask[sb][j];
+            const uint64_t seen_by = (uint64_t(mk.y) << 32) | mk.x;
+            const bool vis = row >= 0 && j < int(n_pages) && ((seen_by >> row) & 1);
+            const int lim = vis ? int((tok4 >> (8 * j)) & 0xffu) : 0;  // tokens [0, lim) of the page are visible to this q-vector
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+              if (c >= lim) sc[j * 16 + c] = __float_as_uint(-INFINITY);
+              mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(sc[j * 16 + c]));
+            }
           }
         }
         mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
