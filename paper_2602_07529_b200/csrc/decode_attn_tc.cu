@@ -130,40 +130,9 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
     const UnitRegs wu2 = load_unit(u + 2);
     const mv::ItemRow nir0 = load_rows(wu1, 0), nir1 = load_rows(wu1, 32);
     const StageRegs nwin = load_window(wu1, 0);
-    // ---- q-vectors (K-major tile, 128-byte swizzle: what the tensor core expects) and partial-slot ids
-    const int n_qv = wu.n_rows * a.G;
-    if (lane == 0) wait_or_flag(h, bar(&meta->q_empty), (ui & 1) ^ 1);
-    __syncwarp();
-    for (int x = lane; x < MAXQV; x += 32) {
-      const int r = min(x / a.G, MAXQV - 1);
-      const int p_lo = __shfl_sync(0xffffffffu, ir0.part, r & 31), p_hi = __shfl_sync(0xffffffffu, ir1.part, r & 31);
-      const int part = r < 32 ? p_lo : p_hi;
-      meta->pv[x] = (x < n_qv && part >= 0) ? part * a.G + x % a.G : -1;
-    }
-    if (lane == 0) {
-      meta->n_stages = wu.n_stages;
-      meta->n_qv = n_qv;
-    }
-    for (int i0 = 0; i0 < MAXQV * 16; i0 += 32) {  // all 64 rows: rows past n_qv are zero-filled
-      const int i = i0 + lane;
-      const int x = i >> 4, c = i & 15;
-      const int r = min(x / a.G, MAXQV - 1);
-      const int r_lo = __shfl_sync(0xffffffffu, ir0.row, r & 31), r_hi = __shfl_sync(0xffffffffu, ir1.row, r & 31);
-      const int row = r < 32 ? r_lo : r_hi;
-      const bool ok = x < n_qv;
-      const bf16* src = a.q + (ok ? (int64_t(row) * a.Hq + wu.kvh * a.G + x % a.G) * D + c * 8 : 0);
-      const uint32_t dst = h.q_smem + (c >> 3) * (Q_BYTES / 2) + x * 128 + (((c & 7) ^ (x & 7)) << 4);
-      mv::cp_async_16(dst, src, ok ? 16 : 0);
-    }
-    mv::cp_async_mbar_arrive_noinc(bar(&meta->q_full));
-    __syncwarp();
-    if (lane == 0) {
-      mv::fence_proxy_async();  // the copies above are read by the tensor core (async proxy)
-      mv::mbar_arrive(bar(&meta->q_full));
-    }
-    // ---- KV stages, 32 descriptors per window
+    // ---- KV stages, 32 descriptors per window (called with s = 0, 1, 2, ... in order)
     StageRegs nxt;
-    for (int s = 0; s < wu.n_stages; ++s) {
+    auto issue_stage = [&](int s) {
       if ((s & 31) == 0) {
         if (s > 0) win = nxt;
         nxt = load_window(wu, s + 32);
@@ -196,7 +165,44 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
         mv::tma_load_2d(dst, kv ? tm_v : tm_k, 0, row, fb);
       }
       ++issued;
+    };
+    // at the start of the share the first stages go out before the q tile is staged: they do not depend on it, and
+    // this puts the first TMA one table read after the launch
+    const int pre = ui == 0 ? min(wu.n_stages, NSTAGES) : 0;
+    for (int s = 0; s < pre; ++s) issue_stage(s);
+    // ---- q-vectors (K-major tile, 128-byte swizzle: what the tensor core expects) and partial-slot ids
+    const int n_qv = wu.n_rows * a.G;
+    if (lane == 0) wait_or_flag(h, bar(&meta->q_empty), (ui & 1) ^ 1);
+    __syncwarp();
+    for (int x = lane; x < MAXQV; x += 32) {
+      const int r = min(x / a.G, MAXQV - 1);
+      const int p_lo = __shfl_sync(0xffffffffu, ir0.part, r & 31), p_hi = __shfl_sync(0xffffffffu, ir1.part, r & 31);
+      const int part = r < 32 ? p_lo : p_hi;
+      meta->pv[x] = (x < n_qv && part >= 0) ? part * a.G + x % a.G : -1;
     }
+    if (lane == 0) {
+      meta->n_stages = wu.n_stages;
+      meta->n_qv = n_qv;
+    }
+    // rows past n_qv are left as they are: the tensor core computes on them, nobody reads those results
+    for (int i0 = 0; i0 < ((n_qv + 1) & ~1) * 16; i0 += 32) {
+      const int i = i0 + lane;
+      const int x = i >> 4, c = i & 15;
+      const int r = min(x / a.G, MAXQV - 1);
+      const int r_lo = __shfl_sync(0xffffffffu, ir0.row, r & 31), r_hi = __shfl_sync(0xffffffffu, ir1.row, r & 31);
+      const int row = r < 32 ? r_lo : r_hi;
+      const bool ok = x < n_qv;
+      const bf16* src = a.q + (ok ? (int64_t(row) * a.Hq + wu.kvh * a.G + x % a.G) * D + c * 8 : 0);
+      const uint32_t dst = h.q_smem + (c >> 3) * (Q_BYTES / 2) + x * 128 + (((c & 7) ^ (x & 7)) << 4);
+      mv::cp_async_16(dst, src, ok ? 16 : 0);
+    }
+    mv::cp_async_mbar_arrive_noinc(bar(&meta->q_full));
+    __syncwarp();
+    if (lane == 0) {
+      mv::fence_proxy_async();  // the copies above are read by the tensor core (async proxy)
+      mv::mbar_arrive(bar(&meta->q_full));
+    }
+    for (int s = pre; s < wu.n_stages; ++s) issue_stage(s);
     wu = wu1; wu1 = wu2; ir0 = nir0; ir1 = nir1; win = nwin;
   }
 }
