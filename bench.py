@@ -34,7 +34,7 @@ METRIC = "dag_decode_attn_query_tokens_per_s"
 UNIT = "query-tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_attn_kernel launch on this workload, taken from the
 # ncu capture summarised in profiles/ (None until a capture exists for the current kernel).
-NCU_TRAFFIC_BYTES = {"config2": 213_300_000}
+NCU_TRAFFIC_BYTES = {"config2": 210_400_000}
 
 
 def _peaks():
@@ -315,7 +315,7 @@ def run_ours(args):
                    "parallelism": (f"{world} ranks, one batch each, sharded by request, no collective" if world > 1 else "single")},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                     "peak_source": peaks["source"], "kernel": "decode_attn_kernel + decode_merge_kernel (one mv_dag_decode_attn call; the traffic figure is decode_attn_kernel alone)",
+                     "peak_source": peaks["source"], "kernel": "decode_tc_kernel + decode_merge_kernel (one mv_dag_decode_attn call; the traffic figure is decode_tc_kernel alone)",
                      "algorithmic_bytes": algo_bytes, "launch_ms_mean": decode_ms, "launch_ms_min": decode_ms_min,
                      "frac_of_nominal_8TBs": achieved / 8000.0, "naive_per_row_GBs": naive_bytes / (decode_ms * 1e-3) / 1e9,
                      "decode_query_tokens_per_s": rows / (decode_ms * 1e-3)},
