@@ -254,6 +254,45 @@ def test_decode_many_siblings_more_than_64_qvectors():
     check_decode(wl, _np(st.step()))
 
 
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (6, 2), (12, 2), (3, 1)])
+def test_decode_odd_group_sizes_head_dim_128(hq, hkv):
+    """Group sizes 1, 3 and 6 on the tensor-memory kernel: q-vectors of a row do not fill a 16-row tile evenly."""
+    rt = _rt()
+    geom = synth.Geometry(hq, hkv, 128, 16, "bf16")
+    for seed in (3, 4):
+        wl = synth.random_dag_workload(seed, "decode", n_req=3, max_nodes=10, max_len=200, geom=geom)
+        st = rt.DecodeState(wl, canary=True)
+        got = _np(st.step())
+        assert st.plan.read_status() == 0
+        check_decode(wl, got)
+
+
+def test_decode_many_rows_group_size_one():
+    """70 sibling rows with one head per KV head: two row groups of 64 and 6 rows, each re-reading the prefix."""
+    rt = _rt()
+    wl = synth.config2(n_req=1, prefix=300, branches=70, branch_len=20)
+    wl.geom = synth.Geometry(2, 2, 128, 16, "bf16")
+    st = rt.DecodeState(wl, canary=True)
+    got = _np(st.step())
+    assert st.plan.read_status() == 0
+    assert st.plan.stats()["max_item_rows"] == 64
+    check_decode(wl, got)
+
+
+def test_decode_single_token_nodes_and_long_units():
+    """Nodes of one token (a lone ragged page each) and a unit longer than one descriptor window (more than 32 stages)."""
+    rt = _rt()
+    geom = synth.Geometry(8, 2, 128, 16, "bf16")
+    req = [([], 2500, 0), ([0], 1, 0), ([1], 1, 0), ([2], 0, 1), ([0], 1, 1), ([0], 17, 1)]
+    wl = synth.Workload("edge", "decode", geom, synth.build_batch([req], rng=np.random.default_rng(5)), 11)
+    st = rt.DecodeState(wl, canary=True)
+    st.plan.replan(wl.batch, 0, geom.n_kv_heads, geom.group, 2)   # two shares: one unit spans ~40 stages
+    st.plan.upload(st.pod.tables)
+    got = _np(st.step())
+    assert st.plan.read_status() == 0
+    check_decode(wl, got)
+
+
 def test_decode_config2_full_sampled():
     rt = _rt()
     wl = synth.config2()
