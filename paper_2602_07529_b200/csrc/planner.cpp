@@ -132,6 +132,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   struct Seg { int32_t stage_begin, n_stages, rows_begin, n_rows; };
   std::vector<Seg> segs;
   std::vector<int32_t> seg_rows;
+  std::vector<char> stage_plain;  // per stage: four full pages seen by the whole row group
   constexpr int kStage = 64;  // tokens per stage of the decode kernel's pipeline
   const int chunk = b->chunk_tokens;  // 0: units are cut only where a CTA's share ends
 
@@ -240,6 +241,11 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
         auto flush = [&]() {
           if (sd.n_pages == 0) return;
           for (int j = sd.n_pages; j < 4; ++j) sd.page[j] = sd.page[0];
+          // plain = four full pages that every row of the group sees: the kernels' unmasked softmax path
+          const uint64_t all_rows = (r1 - r0) == 64 ? ~uint64_t(0) : ((uint64_t(1) << (r1 - r0)) - 1);
+          bool plain = sd.n_pages == 4 && sd.n_tokens4 == 0x10101010u;
+          for (int j = 0; j < 4 && plain; ++j) plain = ((uint64_t(sd.mask_hi[j]) << 32) | sd.mask_lo[j]) == all_rows;
+          stage_plain.push_back(plain ? 1 : 0);
           P->stages.push_back(sd);
           sd = StageDesc{};
         };
@@ -323,10 +329,15 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   if (decode_ready) {
     const int64_t n_rows = new_tok_count;
     const int n_ctas = b->sched_ctas > 0 ? b->sched_ctas : 296;
-    constexpr int64_t kUnitOverhead = 96;  // fixed cost of a unit (q staging, epilogue), in token equivalents
+    // Cost model in token equivalents, fitted to per-share times measured on the device (a full unmasked stage takes
+    // about 1.4 us of a half-CTA's time = 80; a unit's q hand-over and epilogue 2.4 us; a stage whose pages are not all
+    // full and seen by every row takes the masked softmax path, +0.3 us).
+    constexpr int64_t kUnitOverhead = 140;
     const int max_unit_stages = chunk > 0 ? std::max(1, chunk / kStage) : (1 << 30);
     std::vector<int64_t> cost_prefix(P->stages.size() + 1, 0);  // running stage cost over the stage table
-    for (size_t i = 0; i < P->stages.size(); ++i) cost_prefix[i + 1] = cost_prefix[i] + 16 * P->stages[i].n_pages + 16;  // a slot's fixed cost + its pages
+    for (size_t i = 0; i < P->stages.size(); ++i) {
+      cost_prefix[i + 1] = cost_prefix[i] + 16 * P->stages[i].n_pages + 16 + (stage_plain[i] ? 0 : 18);
+    }
     int64_t remaining = 0;  // cost not yet handed out
     for (const Seg& sg : segs)
       remaining += (cost_prefix[size_t(sg.stage_begin + sg.n_stages)] - cost_prefix[size_t(sg.stage_begin)] + kUnitOverhead) * sched_kv_heads;
