@@ -34,6 +34,11 @@ struct Bits {  // dense bitset rows, n_words per node
   bool get(int v, int u) const { return (row(v)[u >> 6] >> (u & 63)) & 1; }
 };
 
+// a decode stream: one per (request, row group): a run of stages and the rows of the group
+struct Seg { int32_t stage_begin, n_stages, rows_begin, n_rows; };
+// a partial slot to be numbered: (row, KV head), unit, row of the unit
+struct PartKey { int32_t rowkv, unit, k; };
+
 size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
 mv_status check_batch(const mv_dag_batch* b) {
@@ -118,10 +123,26 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   }
 
   // ---- pass 1 (per request): layers, visibility, positions, canonical tables
-  Bits vis;
-  std::vector<int32_t> pos_end, layer_end;
-  std::vector<int64_t> node_tok_start(n_nodes, 0);  // flattened index of a node's first NEW token
-  std::vector<std::vector<int32_t>> rows_of_node;    // decode: rows that see each node (request local)
+  // scratch that keeps its capacity from one call to the next (planning runs once per decode step); bound to local
+  // references once, since every access to a thread-local object of a shared library is a call
+  struct Scratch {
+    Bits vis;
+    std::vector<int32_t> pos_end, layer_end, req_rows, row_node, seg_rows, next_part;
+    std::vector<int64_t> node_tok_start, cost_prefix;
+    std::vector<char> seen_by_frontier, stage_plain;
+    std::vector<Seg> segs;
+    std::vector<PartKey> keys;
+  };
+  static thread_local Scratch scratch;
+  Scratch& sc = scratch;
+  Bits& vis = sc.vis;
+  std::vector<int32_t>&pos_end = sc.pos_end, &layer_end = sc.layer_end, &req_rows = sc.req_rows, &row_node = sc.row_node,
+                      &seg_rows = sc.seg_rows, &next_part = sc.next_part;
+  std::vector<int64_t>&node_tok_start = sc.node_tok_start, &cost_prefix = sc.cost_prefix;
+  std::vector<char>&seen_by_frontier = sc.seen_by_frontier, &stage_plain = sc.stage_plain;
+  std::vector<Seg>& segs = sc.segs;
+  std::vector<PartKey>& keys = sc.keys;
+  node_tok_start.assign(size_t(n_nodes), 0);  // flattened index of a node's first NEW token
   int64_t unique_tokens = 0, per_row_tokens = 0, visible_pairs = 0, tile_pairs = 0;
   const int sched_kv_heads = b->n_kv_heads > 0 ? b->n_kv_heads : 8;
   const int sched_group = b->group_size > 0 ? b->group_size : 8;
@@ -129,10 +150,9 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
 
   // decode streams: one per (request, row group): a run of stages and the rows of the group; cut into work
   // units after pass 1
-  struct Seg { int32_t stage_begin, n_stages, rows_begin, n_rows; };
-  std::vector<Seg> segs;
-  std::vector<int32_t> seg_rows;
-  std::vector<char> stage_plain;  // per stage: four full pages seen by the whole row group
+  segs.clear();
+  seg_rows.clear();
+  stage_plain.clear();  // per stage: four full pages seen by the whole row group
   constexpr int kStage = 64;  // tokens per stage of the decode kernel's pipeline
   const int chunk = b->chunk_tokens;  // 0: units are cut only where a CTA's share ends
 
@@ -193,8 +213,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       }
     }
     // canonical per-token and per-q-node tables
-    rows_of_node.assign(n, {});
-    std::vector<char> seen_by_frontier(n, 0);
+    seen_by_frontier.assign(size_t(n), 0);
     for (int v = 0; v < n; ++v) {
       const int g = lo + v;
       node_tok_start[g] = new_tok_count;
@@ -214,7 +233,6 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
         P->seg_len.push_back(ln);
         kv += ln;
         seen_by_frontier[u] = 1;
-        if (decode_ready) rows_of_node[u].push_back(int32_t(new_tok_count));
       }
       P->seg_off.push_back(int32_t(P->seg_node.size()));
       P->kv_len.push_back(kv);
@@ -227,8 +245,8 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
 
     // ---- decode streams of this request: per row group, the stages of every node at least one of its rows sees
     if (decode_ready) {
-      std::vector<int32_t> req_rows;  // rows of the request, ascending (one per frontier node)
-      std::vector<int32_t> row_node;  // local node of each row
+      req_rows.clear();  // rows of the request, ascending (one per frontier node)
+      row_node.clear();  // local node of each row
       for (int v = 0; v < n; ++v)
         if (b->node_new[lo + v] > 0) {
           req_rows.push_back(int32_t(node_tok_start[lo + v]));
@@ -238,13 +256,13 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
         const size_t r1 = std::min(req_rows.size(), r0 + size_t(max_rows_per_item));
         Seg sg{int32_t(P->stages.size()), 0, int32_t(seg_rows.size()), int32_t(r1 - r0)};
         StageDesc sd{};  // the stage being filled, page slot by page slot
+        const uint64_t group_rows = (r1 - r0) == 64 ? ~uint64_t(0) : ((uint64_t(1) << (r1 - r0)) - 1);
         auto flush = [&]() {
           if (sd.n_pages == 0) return;
           for (int j = sd.n_pages; j < 4; ++j) sd.page[j] = sd.page[0];
           // plain = four full pages that every row of the group sees: the kernels' unmasked softmax path
-          const uint64_t all_rows = (r1 - r0) == 64 ? ~uint64_t(0) : ((uint64_t(1) << (r1 - r0)) - 1);
           bool plain = sd.n_pages == 4 && sd.n_tokens4 == 0x10101010u;
-          for (int j = 0; j < 4 && plain; ++j) plain = ((uint64_t(sd.mask_hi[j]) << 32) | sd.mask_lo[j]) == all_rows;
+          for (int j = 0; j < 4 && plain; ++j) plain = ((uint64_t(sd.mask_hi[j]) << 32) | sd.mask_lo[j]) == group_rows;
           stage_plain.push_back(plain ? 1 : 0);
           P->stages.push_back(sd);
           sd = StageDesc{};
@@ -257,7 +275,29 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
             if (vis.get(row_node[k], u)) mask |= uint64_t(1) << (k - r0);
           if (mask == 0) continue;
           const int32_t* pages = b->page_idx + b->page_off[lo + u];
-          for (int32_t t0 = 0; t0 < L; t0 += ps) {
+          int32_t t0 = 0;
+          // open stage first, then whole stages of four full pages at once, then the tail page by page
+          for (; t0 < L && sd.n_pages != 0; t0 += ps) {
+            const int j = sd.n_pages++;
+            sd.page[j] = pages[t0 / ps];
+            sd.n_tokens4 |= uint32_t(std::min<int32_t>(ps, L - t0)) << (8 * j);
+            sd.mask_lo[j] = uint32_t(mask);
+            sd.mask_hi[j] = uint32_t(mask >> 32);
+            if (sd.n_pages == 4) flush();
+          }
+          for (; t0 + 4 * ps <= L; t0 += 4 * ps) {
+            StageDesc full{};
+            for (int j = 0; j < 4; ++j) {
+              full.page[j] = pages[t0 / ps + j];
+              full.mask_lo[j] = uint32_t(mask);
+              full.mask_hi[j] = uint32_t(mask >> 32);
+            }
+            full.n_tokens4 = 0x10101010u;
+            full.n_pages = 4;
+            stage_plain.push_back(mask == group_rows ? 1 : 0);
+            P->stages.push_back(full);
+          }
+          for (; t0 < L; t0 += ps) {
             const int j = sd.n_pages++;
             sd.page[j] = pages[t0 / ps];
             sd.n_tokens4 |= uint32_t(std::min<int32_t>(ps, L - t0)) << (8 * j);
@@ -334,7 +374,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     // full and seen by every row takes the masked softmax path, +0.3 us).
     constexpr int64_t kUnitOverhead = 140;
     const int max_unit_stages = chunk > 0 ? std::max(1, chunk / kStage) : (1 << 30);
-    std::vector<int64_t> cost_prefix(P->stages.size() + 1, 0);  // running stage cost over the stage table
+    cost_prefix.assign(P->stages.size() + 1, 0);  // running stage cost over the stage table
     for (size_t i = 0; i < P->stages.size(); ++i) {
       cost_prefix[i + 1] = cost_prefix[i] + 16 * P->stages[i].n_pages + 16 + (stage_plain[i] ? 0 : 18);
     }
@@ -348,8 +388,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       return std::max<int64_t>((remaining + left * kUnitOverhead + left - 1) / left, 2 * kStage + kUnitOverhead);
     };
     P->cta_unit_off.assign(size_t(n_ctas) + 1, 0);
-    struct PartKey { int32_t rowkv, unit, k; };
-    std::vector<PartKey> keys;
+    keys.clear();
     int cta = 0;
     int64_t acc = 0, target = share(0), max_acc = 0;
     const int64_t first_share = target;
@@ -361,7 +400,8 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       wu.n_rows = sg.n_rows;
       wu.kvh = kvh;
       uint64_t seen = 0;  // rows that see at least one stage of the unit
-      for (int32_t i = 0; i < take; ++i) {
+      const uint64_t all_rows = sg.n_rows == 64 ? ~uint64_t(0) : ((uint64_t(1) << sg.n_rows) - 1);
+      for (int32_t i = 0; i < take && seen != all_rows; ++i) {
         const StageDesc& sd = P->stages[size_t(wu.stage_begin + i)];
         for (int j = 0; j < sd.n_pages; ++j) seen |= uint64_t(sd.mask_lo[j]) | (uint64_t(sd.mask_hi[j]) << 32);
       }
@@ -423,8 +463,8 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     P->rowkv_part_off.assign(size_t(n_rows) * sched_kv_heads + 1, 0);
     for (const PartKey& k : keys) P->rowkv_part_off[size_t(k.rowkv) + 1]++;
     for (size_t i = 1; i < P->rowkv_part_off.size(); ++i) P->rowkv_part_off[i] += P->rowkv_part_off[i - 1];
-    std::vector<int32_t> next(P->rowkv_part_off.begin(), P->rowkv_part_off.end() - 1);
-    for (const PartKey& k : keys) P->item_rows[size_t(P->units[k.unit].row_begin + k.k)].part = next[k.rowkv]++;
+    next_part.assign(P->rowkv_part_off.begin(), P->rowkv_part_off.end() - 1);
+    for (const PartKey& k : keys) P->item_rows[size_t(P->units[k.unit].row_begin + k.k)].part = next_part[k.rowkv]++;
     S.n_items = int64_t(P->units.size());
     S.n_partials = int64_t(keys.size());
     S.n_ctas = n_ctas;
