@@ -66,6 +66,7 @@ struct Half {  // what every role of one half needs
   uint32_t q_smem, stage_smem;  // this half's q tile and first stage
   Meta* meta;
   uint32_t tmem;         // this half's 256 tensor-memory columns: S buffers at +0 and +64, O at +128
+  int lane0;             // tensor-memory lane (= row of the 128-row products) of the half's q-vector 0
   int share;             // index of the share this half works through
   int32_t* status;
 };
@@ -217,8 +218,9 @@ __device__ __forceinline__ void issuer(const TcArgs& a, const Half& h) {
     u_begin = y.y;
     u_end = y.z;
   }
-  // the q tile: 64 rows per column block; the tensor core reads 128, the rest is whatever follows (never used)
-  const uint64_t q_desc = mv::um::smem_desc(h.q_smem, 16, 1024);
+  // the q tile holds 64 rows per column block: rows lane0 .. lane0 + 63 of the 128-row operand; the tensor core reads
+  // the neighbouring 8 KB of shared memory as the other 64 rows, and nobody reads what it computes from them
+  const uint64_t q_desc = mv::um::smem_desc(h.q_smem - uint32_t(h.lane0) * 128u, 16, 1024);
   constexpr uint32_t idesc_qk = mv::um::idesc_bf16(128, ST, 0, 0), idesc_pv = mv::um::idesc_bf16(128, D, 0, 1);
   int g = 0;  // stages consumed so far (ring position)
   int t = 0;  // stages whose scores were issued so far (S buffer = t & 1)
@@ -269,10 +271,13 @@ __device__ __forceinline__ void issuer(const TcArgs& a, const Half& h) {
   }
 }
 
-// ---- softmax group of one half: thread r = q-vector r of the unit (r < 64; warps 2 and 3 of the group idle along) ----
+// ---- softmax group of one half: the thread on tensor-memory lane lane0 + r owns q-vector r of the unit (r < 64); the
+// group's other two warps idle along.  Half 0 keeps its q-vectors on lanes 0..63, half 1 on lanes 64..127, so that the
+// two halves' busy warps sit on different quarters of the SM (a warp reaches the 32 lanes of its index modulo 4).
 __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r = (warp & 3) * 32 + lane;  // tensor-memory lane = q-vector of the unit
+  const int wb = (warp & 3) * 32 - h.lane0;  // q-vector of the warp's lane 0 (negative or >= 64: an idle warp)
+  const int r = wb + lane;
   const int gt = threadIdx.x & 127;      // index inside the group
   Meta* meta = h.meta;
   const uint32_t lane_base = h.tmem + (uint32_t((warp & 3) * 32) << 16);
@@ -288,13 +293,13 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
     const int ui = u - u_begin;
     wait_or_flag(h, bar(&meta->q_full), ui & 1);
     const int n = meta->n_stages, n_qv = meta->n_qv;
-    const int pv = r < MAXQV ? meta->pv[r] : -1;
+    const int pv = (r >= 0 && r < MAXQV) ? meta->pv[r] : -1;
     mv::mbar_arrive(bar(&meta->q_empty));  // header and slot ids are in registers
-    const bool warp_active = (warp & 3) * 32 < n_qv;  // some q-vector of this warp is real
-    const int row = r < n_qv ? r / a.G : -1;           // row of the unit's row group this q-vector belongs to
-    uint64_t warp_rows = 0;                            // rows that own a real q-vector of this warp
+    const bool warp_active = wb >= 0 && wb < n_qv;            // some q-vector of this warp is real
+    const int row = (r >= 0 && r < n_qv) ? r / a.G : -1;      // row of the unit's row group this q-vector belongs to
+    uint64_t warp_rows = 0;                                   // rows that own a real q-vector of this warp
     if (warp_active) {
-      const int r_lo = ((warp & 3) * 32) / a.G, r_hi = (min((warp & 3) * 32 + 31, n_qv - 1)) / a.G;
+      const int r_lo = wb / a.G, r_hi = (min(wb + 31, n_qv - 1)) / a.G;
       warp_rows = (r_hi - r_lo == 63 ? ~uint64_t(0) : ((uint64_t(1) << (r_hi - r_lo + 1)) - 1)) << r_lo;
     }
     float m = -INFINITY, l = 0.f;
@@ -463,6 +468,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) decode_tc_kernel(const TcArgs a, 
   h.stage_smem = smem_base + OFF_STAGES + hi * NSTAGES * STAGE_BYTES;
   h.meta = reinterpret_cast<Meta*>(smem + OFF_META + hi * META_BYTES);
   h.tmem = tmem_slot + hi * 256;
+  h.lane0 = hi * 64;
   h.share = blockIdx.x * 2 + hi;
   h.status = a.status;
   if (h.share < n_shares) {
