@@ -167,9 +167,10 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
       }
       ++issued;
     };
-    // at the start of the share the first stages go out before the q tile is staged: they do not depend on it, and
-    // this puts the first TMA one table read after the launch
-    const int pre = ui == 0 ? min(wu.n_stages, NSTAGES) : 0;
+    // The unit's first stages go out before its q tile is staged: they do not depend on it.  At the start of the share
+    // this puts the first TMA one table read after the launch; between units it keeps the ring full while the producer
+    // waits for the previous unit to let go of the q tile (each stage still waits for its own buffer to come free).
+    const int pre = min(wu.n_stages, NSTAGES);
     for (int s = 0; s < pre; ++s) issue_stage(s);
     // ---- q-vectors (K-major tile, 128-byte swizzle: what the tensor core expects) and partial-slot ids
     const int n_qv = wu.n_rows * a.G;
