@@ -176,6 +176,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
                : "memory");
 }
+// The same load with an L2 eviction-priority policy (see l2_policy_evict_first).
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;\n"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar), "l"(policy)
+               : "memory");
+}
+// Policy for data that is read once: its lines are the first to leave L2, so that what is read again (q, the plan
+// tables, the split-KV partials) stays.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(p));
+  return p;
+}
 // Arrival on `bar` that fires once all cp.async copies this thread issued before it have landed; it counts
 // against the barrier's expected arrivals (no increment of the pending count).
 __device__ __forceinline__ void cp_async_mbar_arrive_noinc(uint32_t bar) {

@@ -130,6 +130,7 @@ __device__ __forceinline__ void producer(const DecodeArgs& a, uint32_t smem_base
     u_end = y.z;
   }
   int issued = 0;  // stages issued so far (buffer = issued % NSTAGES)
+  const uint64_t kv_policy = mv::l2_policy_evict_first();  // the KV stream is read once per call
   // Table reads run ahead of their use so that no load sits on the issue path: the descriptor of unit u + 2,
   // and the row list and first stage window of unit u + 1, are requested while unit u is being issued.
   auto load_unit = [&](int u) {
@@ -221,7 +222,7 @@ __device__ __forceinline__ void producer(const DecodeArgs& a, uint32_t smem_base
       if (lane < 8 && p < n_pages) {
         const int row = (page * a.Hkv + wu.kvh) * (16 * Cfg<D>::HALVES);
         const uint32_t dst = smem_base + b * Cfg<D>::STAGE_BYTES + kv * Cfg<D>::KV_BYTES + p * Cfg<D>::PAGE_BYTES;
-        mv::tma_load_2d(dst, kv ? tm_v : tm_k, 0, row, bar);
+        mv::tma_load_2d_hint(dst, kv ? tm_v : tm_k, 0, row, bar, kv_policy);
       }
       ++issued;
     }

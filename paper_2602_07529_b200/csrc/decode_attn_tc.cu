@@ -123,6 +123,7 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
     return r;
   };
   int issued = 0;
+  const uint64_t kv_policy = mv::l2_policy_evict_first();  // the KV stream is read once per call
   UnitRegs wu1 = load_unit(u_begin + 1);
   mv::ItemRow ir0 = load_rows(wu, 0), ir1 = load_rows(wu, 32);
   StageRegs win = load_window(wu, 0);
@@ -163,7 +164,7 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
       if (lane < 16 && p < n_pages) {
         const int row = ((page * a.Hkv + wu.kvh) * 2 + cb) * 16;
         const uint32_t dst = h.stage_smem + b * STAGE_BYTES + kv * KV_BYTES + cb * (KV_BYTES / 2) + p * 2048;
-        mv::tma_load_2d(dst, kv ? tm_v : tm_k, 0, row, fb);
+        mv::tma_load_2d_hint(dst, kv ? tm_v : tm_k, 0, row, fb, kv_policy);
       }
       ++issued;
     };
