@@ -27,7 +27,9 @@ EXPORTS = ["mv_plan_dag", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_
            "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
            "mv_dag_prefill_attn", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_status_string",
            "mv_launch_count", "mv_plan_read_status", "mv_dag_decode_attn_static",
-           "mv_static_workspace_bytes"]
+           "mv_static_workspace_bytes",
+           "mv_sched_create", "mv_sched_destroy", "mv_sched_add_request", "mv_sched_step", "mv_sched_rows",
+           "mv_sched_commit", "mv_sched_page_refs", "mv_sched_get_stats"]
 
 
 class MvError(RuntimeError):
@@ -54,6 +56,12 @@ class _Stats(C.Structure):
         "n_nodes", "n_new_tokens", "n_qnodes", "n_segs", "decode_ready", "prefill_ready", "n_items", "n_partials",
         "chunk_tokens", "unique_kv_tokens", "per_row_kv_tokens", "n_q_tiles", "visible_pairs", "tile_pairs",
         "max_page_id", "max_item_rows", "sched_kv_heads", "sched_group", "n_ctas", "max_cta_cost")]
+
+
+class _SchedStats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "requests_live", "transitions_fired", "forks", "joins", "markings_advanced", "decode_steps", "rows_emitted",
+        "pages_in_use", "pages_peak")]
 
 
 def _load():
@@ -86,6 +94,15 @@ def _load():
     lib.mv_plan_read_status.argtypes = [vp, vp, C.POINTER(i32)]
     lib.mv_launch_count.argtypes = []
     lib.mv_launch_count.restype = i64
+    lib.mv_sched_create.argtypes = [i32, i32, C.POINTER(vp)]
+    lib.mv_sched_destroy.argtypes = [vp]
+    lib.mv_sched_destroy.restype = None
+    lib.mv_sched_add_request.argtypes = [vp, i32, vp, vp, vp, C.POINTER(i32)]
+    lib.mv_sched_step.argtypes = [vp, C.POINTER(_DagBatch), C.POINTER(i32)]
+    lib.mv_sched_rows.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i32)]
+    lib.mv_sched_commit.argtypes = [vp, vp]
+    lib.mv_sched_page_refs.argtypes = [vp, vp, i32, vp]
+    lib.mv_sched_get_stats.argtypes = [vp, C.POINTER(_SchedStats)]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is C.c_int and name not in ("mv_plan_destroy",):
@@ -247,3 +264,73 @@ def mv_launch_count() -> int:
 
 def mv_status_string(status: int) -> str:
     return lib.mv_status_string(int(status)).decode()
+
+
+class Scheduler:
+    """Frontier scheduler (``mv_sched_*``): argument marshalling only."""
+
+    def __init__(self, page_size: int, num_pages: int):
+        self._h = C.c_void_p(None)
+        _check(lib.mv_sched_create(page_size, num_pages, C.byref(self._h)), "mv_sched_create")
+        self.c_batch = _DagBatch()
+
+    def add_request(self, parents, tokens) -> int:
+        off = np.zeros(len(parents) + 1, np.int32)
+        off[1:] = np.cumsum([len(p) for p in parents])
+        idx = _i32([q for p in parents for q in p])
+        tok = _i32(tokens)
+        rid = C.c_int32(-1)
+        _check(lib.mv_sched_add_request(self._h, len(parents), off.ctypes.data, idx.ctypes.data if idx.size else None,
+                                        tok.ctypes.data, C.byref(rid)), "mv_sched_add_request")
+        return int(rid.value)
+
+    def step(self):
+        """Emits the next decode step.  Returns None when nothing is running, else a dict of numpy copies of the
+        batch arrays plus ``row_req`` / ``row_node``; ``self.c_batch`` is the struct mv_plan_dag takes."""
+        n_rows = C.c_int32(0)
+        _check(lib.mv_sched_step(self._h, C.byref(self.c_batch), C.byref(n_rows)), "mv_sched_step")
+        if n_rows.value == 0:
+            return None
+        b = self.c_batch
+        n_req = int(b.n_req)
+
+        def arr(ptr, n):
+            return np.ctypeslib.as_array(C.cast(ptr, C.POINTER(C.c_int32)), shape=(n,)).copy() if n else np.zeros(0, np.int32)
+        node_off = arr(b.node_off, n_req + 1)
+        n_nodes = int(node_off[-1])
+        parent_off = arr(b.parent_off, n_nodes + 1)
+        page_off = arr(b.page_off, n_nodes + 1)
+        rq, nd, n = C.c_void_p(), C.c_void_p(), C.c_int32(0)
+        _check(lib.mv_sched_rows(self._h, C.byref(rq), C.byref(nd), C.byref(n)), "mv_sched_rows")
+        return dict(n_req=n_req, node_off=node_off, node_len=arr(b.node_len, n_nodes), node_new=arr(b.node_new, n_nodes),
+                    parent_off=parent_off, parent_idx=arr(b.parent_idx, int(parent_off[-1])), page_off=page_off,
+                    page_idx=arr(b.page_idx, int(page_off[-1])), row_req=arr(rq.value, n.value), row_node=arr(nd.value, n.value))
+
+    def commit(self, finished=None):
+        f = None
+        if finished is not None:
+            f = np.ascontiguousarray(np.asarray(finished, dtype=np.uint8))
+        _check(lib.mv_sched_commit(self._h, f.ctypes.data if f is not None else None), "mv_sched_commit")
+
+    def page_refs(self, pages) -> np.ndarray:
+        p = _i32(pages)
+        out = np.zeros(p.size, np.int32)
+        _check(lib.mv_sched_page_refs(self._h, p.ctypes.data if p.size else None, p.size, out.ctypes.data if p.size else None),
+               "mv_sched_page_refs")
+        return out
+
+    def stats(self) -> dict:
+        st = _SchedStats()
+        _check(lib.mv_sched_get_stats(self._h, C.byref(st)), "mv_sched_get_stats")
+        return {n: int(getattr(st, n)) for n, _ in _SchedStats._fields_}
+
+    def destroy(self):
+        if self._h:
+            lib.mv_sched_destroy(self._h)
+            self._h = C.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libmedverse_attn.so")
-SOURCES = ["planner.cpp", "plan_runtime.cu", "rope_write_kv.cu", "decode_attn.cu", "decode_attn_tc.cu", "prefill_attn_f32.cu",
+SOURCES = ["planner.cpp", "scheduler.cpp", "plan_runtime.cu", "rope_write_kv.cu", "decode_attn.cu", "decode_attn_tc.cu", "prefill_attn_f32.cu",
            "prefill_attn_bf16.cu", "prefill_attn_tc.cu", "decode_step_host.cu", "tma_util.cu"]
 
 
@@ -25,7 +25,7 @@ def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "medverse_attn.h")]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", f) for f in os.listdir(os.path.join(ROOT, "include"))]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

@@ -25,7 +25,8 @@ def _compare(batch):
 
 
 def test_library_exports_every_declared_symbol():
-    hdr = open(os.path.join(ROOT, "include", "medverse_attn.h")).read()
+    inc = os.path.join(ROOT, "include")
+    hdr = "".join(open(os.path.join(inc, f)).read() for f in sorted(os.listdir(inc)) if f.endswith(".h"))
     declared = set(re.findall(r"\b(mv_[a-z_]+)\s*\(", hdr))
     assert declared, "no declarations parsed"
     assert declared == set(B.EXPORTS)

@@ -1,0 +1,166 @@
+"""The frontier scheduler (mv_sched_*, through the C ABI) against its oracle, step by step and bit for bit; its
+batches handed to the attention planner; its cost per step.  No GPU."""
+import ctypes as C
+import time
+
+import numpy as np
+import pytest
+
+from oracle import frontier_oracle as FO
+from oracle import medverse_oracle as MO
+from paper_2602_07529_b200 import binding as B, synth
+
+KEYS = ("node_off", "node_len", "node_new", "parent_off", "parent_idx", "page_off", "page_idx", "row_req", "row_node")
+
+
+def _random_dag(rng, n, max_parents=3, n_roots=1):
+    parents = [[] for _ in range(n)]
+    for v in range(n_roots, n):
+        k = int(rng.integers(1, min(max_parents, v) + 1))
+        parents[v] = sorted(rng.choice(v, size=k, replace=False).tolist())
+    return parents
+
+
+def _same_step(got, want):
+    assert (got is None) == (want is None)
+    if got is None:
+        return
+    assert got["n_req"] == want["n_req"]
+    for k in KEYS:
+        assert np.array_equal(got[k], np.asarray(want[k], dtype=np.int32)), k
+
+
+def _same_state(s, o, num_pages):
+    refs = s.page_refs(np.arange(num_pages))
+    want = np.array([o.refs.get(p, 0) for p in range(num_pages)], np.int32)
+    assert np.array_equal(refs, want)
+    st = s.stats()
+    for k, v in o.stats.items():
+        assert st[k] == v, k
+    assert st["requests_live"] == sum(1 for rq in o.requests if not rq.done)
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_streams_match_the_oracle_step_by_step(seed):
+    rng = np.random.default_rng(100 + seed)
+    num_pages = 512
+    s, o = B.Scheduler(16, num_pages), FO.Scheduler(16, num_pages)
+    pending = []
+    for _ in range(int(rng.integers(2, 6))):
+        n = int(rng.integers(2, 12))
+        parents = _random_dag(rng, n, n_roots=int(rng.integers(1, 3)) if n > 3 else 1)
+        tokens = [int(rng.integers(0, 70)) if not parents[v] else int(rng.integers(1, 40)) for v in range(n)]
+        pending.append((parents, tokens))
+    # two requests at once, the others join while the first ones run
+    for parents, tokens in pending[:2]:
+        assert s.add_request(parents, tokens) == o.add_request(parents, tokens)
+    pending = pending[2:]
+    steps = 0
+    while True:
+        _same_state(s, o, num_pages)
+        got, want = s.step(), o.step()
+        _same_step(got, want)
+        if got is None:
+            if not pending:
+                break
+            parents, tokens = pending.pop()
+            assert s.add_request(parents, tokens) == o.add_request(parents, tokens)
+            continue
+        finished = (rng.random(len(got["row_req"])) < 0.05).astype(np.uint8) if seed % 2 else None
+        s.commit(finished)
+        o.commit(finished)
+        steps += 1
+        if pending and steps % 7 == 0:
+            parents, tokens = pending.pop()
+            assert s.add_request(parents, tokens) == o.add_request(parents, tokens)
+    _same_state(s, o, num_pages)
+    assert s.stats()["pages_in_use"] == 0 and steps > 0
+
+
+def test_scheduler_steps_feed_the_attention_planner():
+    # every emitted batch is a valid decode batch: the planner accepts it and agrees with the attention oracle's
+    # layers and positions; rows of one frontier that fork from one node start at the same position (Sec. 4.2)
+    s = B.Scheduler(16, 256)
+    R, A, Bn, Cn, Dn = range(5)
+    s.add_request([[], [R], [R], [A, Bn], [R]], [37, 5, 9, 3, 2])
+    n_steps = 0
+    while True:
+        b = s.step()
+        if b is None:
+            break
+        # the struct the scheduler filled goes to the planner as it is (the caller only adds its scheduling hints)
+        s.c_batch.n_kv_heads, s.c_batch.group_size = 8, 4
+        h = C.c_void_p(None)
+        assert B.lib.mv_plan_dag(C.byref(s.c_batch), C.byref(h)) == 0
+        B.lib.mv_plan_destroy(h)
+        # and the same arrays through the binding's own batch type, to read the tables back
+        batch = synth.DagBatch(b["n_req"], b["node_off"], b["node_len"], b["node_new"], b["parent_off"], b["parent_idx"],
+                               b["page_off"], b["page_idx"], 16, 256, synth.VIS_ANCESTORS, synth.POS_MAX_PARENT_END)
+        plan = B.Plan(batch, 0, 8, 4)
+        st = plan.stats()
+        assert st["decode_ready"] == 1 and st["n_new_tokens"] == len(b["row_req"])
+        n = int(b["node_off"][1])
+        parents = [b["parent_idx"][b["parent_off"][v]:b["parent_off"][v + 1]].tolist() for v in range(n)]
+        layer = MO.node_layers(parents)
+        assert np.array_equal(plan.table("layer"), np.asarray(layer, np.int32))
+        total = (b["node_len"] + b["node_new"]).tolist()
+        start = MO.position_starts(parents, total, layer)
+        want_pos = [int(start[v]) + int(b["node_len"][v]) for v in range(n) if b["node_new"][v]]
+        assert plan.table("pos_id").tolist() == want_pos
+        if n_steps == 0:  # A, B and D fork from R: same first position, right after the context
+            assert want_pos == [37, 37, 37]
+        s.commit()
+        n_steps += 1
+    assert n_steps == 9 + 3  # the frontier {A, B, D} lasts as long as B; then the join C
+
+
+def test_error_paths_leave_the_state_unchanged():
+    s = B.Scheduler(16, 4)
+    with pytest.raises(B.MvError) as e:
+        s.add_request([[], [1]], [3, 1])
+    assert e.value.status == 2  # a parent must precede its child
+    with pytest.raises(B.MvError) as e:
+        s.add_request([[], [0]], [3, 0])
+    assert e.value.status == 1  # a step emits at least one token
+    with pytest.raises(B.MvError) as e:
+        s.add_request([[], [0]], [100, 1])
+    assert e.value.status == 3 and s.stats()["pages_in_use"] == 0  # the context does not fit
+    with pytest.raises(B.MvError) as e:
+        s.commit()
+    assert e.value.status == 1  # nothing was emitted
+    s.add_request([[], [0], [0]], [33, 40, 40])  # 3 pages of context, one page left
+    with pytest.raises(B.MvError) as e:
+        s.step()
+    assert e.value.status == 3 and s.stats()["pages_in_use"] == 3 and s.stats()["decode_steps"] == 0
+    assert s.page_refs([0, 1, 2, 3]).tolist() == [3, 3, 3, 0]
+
+
+def test_step_is_idempotent_until_committed_and_requests_wait_for_the_commit():
+    s = B.Scheduler(16, 64)
+    s.add_request([[], [0]], [5, 3])
+    a, b = s.step(), s.step()
+    for k in KEYS:
+        assert np.array_equal(a[k], b[k])
+    assert s.stats()["decode_steps"] == 1 and s.stats()["pages_in_use"] == 2
+    with pytest.raises(B.MvError):
+        s.add_request([[], [0]], [5, 3])
+    s.commit()
+    assert s.add_request([[], [0]], [5, 3]) == 1
+
+
+def test_scheduling_cost_per_step_is_small_against_a_decode_step():
+    # 16 requests of one context and four sibling steps each (the shape of the timed decode workload): the paper puts
+    # parsing and scheduling below 0.01 % and Fork / Join near 1 % of a request's latency (Table 2); here one
+    # mv_sched_step + mv_sched_commit must stay far below the ~50 us the attention of such a step takes on the GPU
+    s = B.Scheduler(16, 16 * (128 + 4 * 8))
+    for _ in range(16):
+        s.add_request([[], [0], [0], [0], [0]], [2048, 100, 100, 100, 100])
+    n_rows = C.c_int32(0)
+    t0 = time.perf_counter()
+    steps = 0
+    for _ in range(90):
+        assert B.lib.mv_sched_step(s._h, C.byref(s.c_batch), C.byref(n_rows)) == 0 and n_rows.value == 64
+        assert B.lib.mv_sched_commit(s._h, None) == 0
+        steps += 1
+    us = (time.perf_counter() - t0) / steps * 1e6
+    assert us < 25.0, us
