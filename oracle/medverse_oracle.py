@@ -317,3 +317,44 @@ def decode_request(batch, r, q_raw, k_raw, v, base=10000.0, scale=None, rows=Non
         allow = np.ones((1, kk.shape[0]), dtype=bool)
         out[ri] = masked_attention(qq, kk, vv, allow, scale)[0]
     return out
+
+
+def append_request(batch, r, q_raw, k_raw, v, base=10000.0, scale=None, rows=None):
+    """Several new tokens per node against the existing cache (Sec. 4.3: what follows a Join or the Phase I -> II
+    hand-over, where generation "proceeds from the merged KV state" with more than one token to write at once).
+
+    Nodes that receive tokens in the same call must not see one another (they are one frontier).  k_raw / v
+    [n_tot, Hkv, d]: raw values of every token of every node in (node, token) order, a node's new tokens last inside
+    it.  q_raw [n_new, Hq, d]: one raw query per new token, (node, token) order.  New token j of node w sees every
+    token of every other node of vis(w), and tokens 0 .. node_len(w) + j of w itself (causal inside the own node,
+    Eq. 2; the DAG mask of Eq. 3 across nodes).  Each token is embedded at its adaptive index (Sec. 4.2).
+    Returns o [n_new, Hq, d] float64 (rows not requested are left as NaN).
+    """
+    lo, hi, parents, layer, vis, tot, start = _request_layout(batch, r)
+    tok_off = np.concatenate([[0], np.cumsum(tot)]).astype(np.int64)
+    fresh = [vl for vl in range(hi - lo) if int(batch["node_new"][lo + vl]) > 0]
+    for w in fresh:
+        for u in vis[w]:
+            if u != w and u in fresh:
+                raise ValueError("nodes that receive tokens in one call must not see one another")
+    q_raw = np.asarray(q_raw)
+    out = np.full(q_raw.shape, np.nan, np.float64)
+    ri = 0
+    for w in fresh:
+        old = int(batch["node_len"][lo + w])
+        for j in range(int(batch["node_new"][lo + w])):
+            if rows is None or ri in rows:
+                ks, vs, pos = [], [], []
+                for u in vis[w]:
+                    a = int(tok_off[u])
+                    n_vis = (old + j + 1) if u == w else int(tok_off[u + 1]) - a
+                    ks.append(k_raw[a:a + n_vis])
+                    vs.append(v[a:a + n_vis])
+                    pos.extend(range(start[u], start[u] + n_vis))
+                kk = rope_rotate(np.concatenate(ks, 0), pos, base)
+                qq = rope_rotate(q_raw[ri:ri + 1], [start[w] + old + j], base)
+                allow = np.ones((1, kk.shape[0]), dtype=bool)
+                out[ri] = masked_attention(qq, kk, np.concatenate(vs, 0), allow, scale)[0]
+            ri += 1
+    return out
+

@@ -365,3 +365,61 @@ def test_config1_visible_pair_count():
     allow = O.allowed_mask(tok_node, tok_index, vis)
     expect = 128 * 129 // 2 + 3 * (32 * 128 + 32 * 33 // 2) + 16 * (240 - 16) + 16 * 17 // 2
     assert int(allow.sum()) == expect
+
+
+# ------------------------------------------------------------------ several new tokens per node against the cache
+
+def _append_case(seed, k_new):
+    rng = np.random.default_rng(seed)
+    # context, two siblings that receive k_new tokens each, an older finished branch that only one of them sees
+    reqs = [[([], 19, 0), ([0], 7, 0), ([0, 1], int(rng.integers(0, 20)), k_new), ([0], int(rng.integers(1, 20)), k_new)]]
+    b = synth.build_batch(reqs, rng=rng)
+    tot = int((b.node_len + b.node_new).sum())
+    q = _rand((2 * k_new, 4, 16), seed + 1)
+    k = _rand((tot, 2, 16), seed + 2)
+    v = _rand((tot, 2, 16), seed + 3)
+    return reqs, b, q, k, v
+
+
+def test_append_of_one_token_is_the_decode_step():
+    reqs, b, q, k, v = _append_case(11, 1)
+    bd = batch_dict(b)
+    assert max_abs(O.append_request(bd, 0, q, k, v), O.decode_request(bd, 0, q, k, v)) == 0.0
+
+
+def test_append_of_k_tokens_equals_k_decode_steps():
+    """Writing k tokens of a node at once gives every one of them what k single-token steps would have given."""
+    for seed, k_new in ((21, 3), (22, 17)):
+        reqs, b, q, k, v = _append_case(seed, k_new)
+        got = O.append_request(batch_dict(b), 0, q, k, v)
+        tok_off = np.concatenate([[0], np.cumsum(b.node_len + b.node_new)])
+        fresh = [n for n in range(4) if b.node_new[n] > 0]
+        for j in range(k_new):
+            step = [(p, ln + (j if nw else 0), 1 if nw else 0) for p, ln, nw in reqs[0]]
+            bj = batch_dict(synth.build_batch([step]))
+            keep = np.concatenate([np.arange(tok_off[n], tok_off[n] + b.node_len[n] + (j + 1 if b.node_new[n] else 0)) for n in range(4)])
+            qj = np.stack([q[i * k_new + j] for i in range(len(fresh))])
+            want = O.decode_request(bj, 0, qj, k[keep], v[keep])
+            for i in range(len(fresh)):
+                assert max_abs(got[i * k_new + j], want[i]) < 1e-12
+
+
+def test_append_rows_equal_the_dense_mask_formulation():
+    """The same rows from the flattened-sequence oracle with the dense mask of Eq. 3."""
+    reqs, b, q, k, v = _append_case(31, 9)
+    got = O.append_request(batch_dict(b), 0, q, k, v)
+    hist = batch_dict(b.as_history())
+    tok_off = np.concatenate([[0], np.cumsum(b.node_len + b.node_new)])
+    rows = np.concatenate([np.arange(tok_off[n + 1] - b.node_new[n], tok_off[n + 1]) for n in range(4) if b.node_new[n] > 0])
+    qfull = np.zeros((int(tok_off[-1]), 4, 16), np.float32)
+    qfull[rows] = q
+    # siblings that receive tokens in the same call do not see each other in either formulation
+    want = O.prefill_request(hist, 0, qfull, k, v)[rows]
+    assert max_abs(got, want) < 1e-12
+
+
+def test_append_refuses_nodes_that_see_each_other():
+    b = batch_dict(synth.build_batch([[([], 5, 2), ([0], 0, 3)]]))
+    with pytest.raises(ValueError):
+        O.append_request(b, 0, _rand((5, 4, 16), 1), _rand((10, 2, 16), 2), _rand((10, 2, 16), 3))
+
