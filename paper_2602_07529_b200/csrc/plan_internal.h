@@ -10,6 +10,7 @@
 namespace mv {
 
 constexpr int kPrefillQTile = 128;   // query rows per prefill tile (tiles never straddle a node)
+constexpr int kMaxAppendTokens = 256;  // most new tokens per node that the decode path takes (beyond that: prefill only)
 constexpr int kPrefillKvTile = 64;   // granularity used only for the executed-pairs statistic
 
 // Decode work lists.  A request's frontier rows (at most 64 / group_size of them per row group) and all the KV

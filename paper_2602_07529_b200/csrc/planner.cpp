@@ -118,7 +118,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
 
   bool decode_ready = true, prefill_ready = true;
   for (int g = 0; g < n_nodes; ++g) {
-    if (b->node_new[g] > 1) decode_ready = false;
+    if (b->node_new[g] > mv::kMaxAppendTokens) decode_ready = false;
     if (b->node_len[g] != 0) prefill_ready = false;
   }
 
@@ -127,7 +127,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   // references once, since every access to a thread-local object of a shared library is a call
   struct Scratch {
     Bits vis;
-    std::vector<int32_t> pos_end, layer_end, req_rows, row_node, seg_rows, next_part;
+    std::vector<int32_t> pos_end, layer_end, req_rows, row_node, row_tok, seg_rows, next_part;
     std::vector<int64_t> node_tok_start, cost_prefix;
     std::vector<char> seen_by_frontier, stage_plain;
     std::vector<Seg> segs;
@@ -136,7 +136,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   static thread_local Scratch scratch;
   Scratch& sc = scratch;
   Bits& vis = sc.vis;
-  std::vector<int32_t>&pos_end = sc.pos_end, &layer_end = sc.layer_end, &req_rows = sc.req_rows, &row_node = sc.row_node,
+  std::vector<int32_t>&pos_end = sc.pos_end, &layer_end = sc.layer_end, &req_rows = sc.req_rows, &row_node = sc.row_node, &row_tok = sc.row_tok,
                       &seg_rows = sc.seg_rows, &next_part = sc.next_part;
   std::vector<int64_t>&node_tok_start = sc.node_tok_start, &cost_prefix = sc.cost_prefix;
   std::vector<char>&seen_by_frontier = sc.seen_by_frontier, &stage_plain = sc.stage_plain;
@@ -243,14 +243,22 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     for (int u = 0; u < n; ++u)
       if (seen_by_frontier[u]) unique_tokens += b->node_len[lo + u] + b->node_new[lo + u];
 
+    // the decode path applies when the nodes that receive tokens form one frontier: none of them sees another
+    for (int v = 0; v < n && decode_ready; ++v) {
+      if (b->node_new[lo + v] == 0) continue;
+      for (int u = 0; u < n; ++u)
+        if (u != v && b->node_new[lo + u] > 0 && vis.get(v, u)) decode_ready = false;
+    }
     // ---- decode streams of this request: per row group, the stages of every node at least one of its rows sees
     if (decode_ready) {
-      req_rows.clear();  // rows of the request, ascending (one per frontier node)
+      req_rows.clear();  // rows of the request, ascending: one per new token, node after node
       row_node.clear();  // local node of each row
+      row_tok.clear();   // which of its node's new tokens the row is
       for (int v = 0; v < n; ++v)
-        if (b->node_new[lo + v] > 0) {
-          req_rows.push_back(int32_t(node_tok_start[lo + v]));
+        for (int32_t j = 0; j < b->node_new[lo + v]; ++j) {
+          req_rows.push_back(int32_t(node_tok_start[lo + v]) + j);
           row_node.push_back(v);
+          row_tok.push_back(j);
         }
       for (size_t r0 = 0; r0 < req_rows.size(); r0 += size_t(max_rows_per_item)) {
         const size_t r1 = std::min(req_rows.size(), r0 + size_t(max_rows_per_item));
@@ -270,11 +278,42 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
         for (int u = 0; u < n; ++u) {
           const int32_t L = b->node_len[lo + u] + b->node_new[lo + u];
           if (L == 0) continue;
-          uint64_t mask = 0;
+          uint64_t mask = 0, own = 0;  // rows that see node u; those among them that are new tokens of u itself
           for (size_t k = r0; k < r1; ++k)
-            if (vis.get(row_node[k], u)) mask |= uint64_t(1) << (k - r0);
+            if (vis.get(row_node[k], u)) {
+              mask |= uint64_t(1) << (k - r0);
+              if (row_node[k] == u) own |= uint64_t(1) << (k - r0);
+            }
           if (mask == 0) continue;
           const int32_t* pages = b->page_idx + b->page_off[lo + u];
+          if (own != 0 && b->node_new[lo + u] > 1) {
+            // Several new tokens of u in this group: token j sees u's tokens 0 .. node_len + j (causal inside the own
+            // node).  A page is listed once per distinct count of visible tokens among the group's rows, each time
+            // with the rows that see exactly that many (rows of other nodes cannot see u: it receives tokens).
+            const int32_t old_len = b->node_len[lo + u];
+            for (int32_t t0 = 0; t0 < L; t0 += ps) {
+              size_t k = r0;
+              while (k < r1) {
+                if (row_node[k] != u) { ++k; continue; }
+                const int32_t lim = std::max<int32_t>(0, std::min<int32_t>(ps, old_len + row_tok[k] + 1 - t0));
+                uint64_t run = 0;
+                size_t k2 = k;
+                for (; k2 < r1 && row_node[k2] == u &&
+                       std::max<int32_t>(0, std::min<int32_t>(ps, old_len + row_tok[k2] + 1 - t0)) == lim; ++k2)
+                  run |= uint64_t(1) << (k2 - r0);
+                if (lim > 0) {
+                  const int j = sd.n_pages++;
+                  sd.page[j] = pages[t0 / ps];
+                  sd.n_tokens4 |= uint32_t(lim) << (8 * j);
+                  sd.mask_lo[j] = uint32_t(run);
+                  sd.mask_hi[j] = uint32_t(run >> 32);
+                  if (sd.n_pages == 4) flush();
+                }
+                k = k2;
+              }
+            }
+            continue;
+          }
           int32_t t0 = 0;
           // open stage first, then whole stages of four full pages at once, then the tail page by page
           for (; t0 < L && sd.n_pages != 0; t0 += ps) {

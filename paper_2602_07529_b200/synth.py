@@ -138,12 +138,13 @@ def config1() -> Workload:
 
 
 def config2(seed: int = 1002, n_req: int = 16, prefix: int = 2048, branches: int = 4,
-            branch_len: int = 256) -> Workload:
-    """Multi-branch decode step, Llama-3-8B attention geometry, bf16 KV."""
+            branch_len: int = 256, new_tokens: int = 1) -> Workload:
+    """Multi-branch decode step, Llama-3-8B attention geometry, bf16 KV (new_tokens > 1: every branch receives that
+    many tokens at once, a node append)."""
     rng = np.random.default_rng(seed)
     reqs = []
     for _ in range(n_req):
-        req = [([], prefix, 0)] + [([0], branch_len, 1) for _ in range(branches)]
+        req = [([], prefix, 0)] + [([0], branch_len, new_tokens) for _ in range(branches)]
         reqs.append(req)
     batch = build_batch(reqs, rng=rng)
     geom = Geometry(32, 8, 128, 16, "bf16", 10000.0, 1.0 / math.sqrt(128.0))
@@ -231,8 +232,9 @@ def config5(seed: int = 1005, n_req: int = 128, prefix_lo: int = 512, prefix_hi:
 
 def random_dag_workload(seed: int, kind: str = "decode", n_req: int = 3, max_nodes: int = 9,
                         max_len: int = 70, geom: Geometry | None = None, vis_mode=VIS_ANCESTORS,
-                        pos_mode=POS_MAX_PARENT_END, allow_empty: bool = True) -> Workload:
-    """Small arbitrary DAGs (any node may have any earlier nodes as parents) for parity sweeps."""
+                        pos_mode=POS_MAX_PARENT_END, allow_empty: bool = True, max_new: int = 1) -> Workload:
+    """Small arbitrary DAGs (any node may have any earlier nodes as parents) for parity sweeps.  kind "decode": the
+    leaves receive tokens, one each, or 1 .. max_new each (node append) when max_new > 1."""
     rng = np.random.default_rng(seed)
     reqs = []
     for _ in range(n_req):
@@ -249,7 +251,7 @@ def random_dag_workload(seed: int, kind: str = "decode", n_req: int = 3, max_nod
         for v in range(n):
             ln = int(rng.integers(0 if allow_empty else 1, max_len + 1))
             if kind == "decode":
-                req.append((parents[v], ln, 0 if has_child[v] else 1))
+                req.append((parents[v], ln, 0 if has_child[v] else (1 if max_new <= 1 else int(rng.integers(1, max_new + 1)))))
             else:
                 req.append((parents[v], 0, max(ln, 0 if allow_empty else 1)))
         if kind == "prefill" and sum(x[2] for x in req) == 0:
