@@ -121,8 +121,8 @@ typedef enum {
 
 typedef struct {
   int64_t n_nodes, n_new_tokens, n_qnodes, n_segs;
-  int64_t decode_ready;        /* 1 if mv_dag_decode_attn applies: the nodes that receive tokens do not see one
-                                  another and receive at most 256 tokens each (one each in a plain decode step)  */
+  int64_t decode_ready;        /* 1 if mv_dag_decode_attn applies: every node receives at most one token, or at
+                                  most 256 each with no receiving node visible to another of its request        */
   int64_t prefill_ready;       /* 1 if no node holds older tokens (mv_dag_prefill_attn applies)            */
   int64_t n_items;             /* decode: work units = (KV slice of a node, KV head, row set)                */
   int64_t n_partials;          /* decode: split-KV partial results, each holding group_size head vectors    */
@@ -198,8 +198,9 @@ mv_status mv_rope_write_kv(const mv_plan* plan, const mv_attn_geom* geom, const 
  * (prefix, common ancestors) are read once per KV head and serve all those rows and the whole GQA group.
  * Node append (what follows a Join or the Phase I -> II hand-over of Sec. 4.3, where more than one token is
  * written to a node at once): a node may receive up to 256 new tokens, one row each in (node, token) order; new
- * token j of v then sees v's tokens 0 .. node_len(v) + j and every other visible node in full.  Nodes that
- * receive tokens in one call must not see one another, else the plan is not decode_ready.
+ * token j of v then sees v's tokens 0 .. node_len(v) + j and every other visible node in full.  In a request
+ * where some node receives several tokens, the nodes that receive tokens must not see one another, else the
+ * plan is not decode_ready.
  *   q_rot   device [n_rows][n_q_heads][head_dim]  bf16
  *   k_pages, v_pages  device pools, bf16
  *   out     device [n_rows][n_q_heads][head_dim]  bf16

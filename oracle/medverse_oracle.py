@@ -323,7 +323,8 @@ def append_request(batch, r, q_raw, k_raw, v, base=10000.0, scale=None, rows=Non
     """Several new tokens per node against the existing cache (Sec. 4.3: what follows a Join or the Phase I -> II
     hand-over, where generation "proceeds from the merged KV state" with more than one token to write at once).
 
-    Nodes that receive tokens in the same call must not see one another (they are one frontier).  k_raw / v
+    When some node receives more than one token, the nodes that receive tokens must not see one another (they are
+    one frontier).  k_raw / v
     [n_tot, Hkv, d]: raw values of every token of every node in (node, token) order, a node's new tokens last inside
     it.  q_raw [n_new, Hq, d]: one raw query per new token, (node, token) order.  New token j of node w sees every
     token of every other node of vis(w), and tokens 0 .. node_len(w) + j of w itself (causal inside the own node,
@@ -333,10 +334,11 @@ def append_request(batch, r, q_raw, k_raw, v, base=10000.0, scale=None, rows=Non
     lo, hi, parents, layer, vis, tot, start = _request_layout(batch, r)
     tok_off = np.concatenate([[0], np.cumsum(tot)]).astype(np.int64)
     fresh = [vl for vl in range(hi - lo) if int(batch["node_new"][lo + vl]) > 0]
-    for w in fresh:
-        for u in vis[w]:
-            if u != w and u in fresh:
-                raise ValueError("nodes that receive tokens in one call must not see one another")
+    if any(int(batch["node_new"][lo + w]) > 1 for w in fresh):
+        for w in fresh:
+            for u in vis[w]:
+                if u != w and u in fresh:
+                    raise ValueError("nodes that receive several tokens in one call must not see one another")
     q_raw = np.asarray(q_raw)
     out = np.full(q_raw.shape, np.nan, np.float64)
     ri = 0

@@ -243,8 +243,12 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     for (int u = 0; u < n; ++u)
       if (seen_by_frontier[u]) unique_tokens += b->node_len[lo + u] + b->node_new[lo + u];
 
-    // the decode path applies when the nodes that receive tokens form one frontier: none of them sees another
-    for (int v = 0; v < n && decode_ready; ++v) {
+    // a request in which some node receives several tokens takes the decode path only if the nodes that receive
+    // tokens form one frontier: none of them sees another (single-token steps have no such condition: a row sees
+    // the token another row of the step has just written whenever it sees that row's node)
+    bool multi = false;
+    for (int v = 0; v < n; ++v) multi |= b->node_new[lo + v] > 1;
+    for (int v = 0; v < n && decode_ready && multi; ++v) {
       if (b->node_new[lo + v] == 0) continue;
       for (int u = 0; u < n; ++u)
         if (u != v && b->node_new[lo + u] > 0 && vis.get(v, u)) decode_ready = false;
