@@ -216,6 +216,20 @@ def test_prefill_config4_sampled():
     assert stats["visible_pairs"] < stats["tile_pairs"] < 17083 * 17084 // 2 * 1.05
 
 
+def test_prefill_config4_paper_literal_modes():
+    rt = _rt()
+    wl = synth.config4()
+    wl.batch.vis_mode, wl.batch.pos_mode = 1, 1
+    st = rt.PrefillState(wl, with_pool=False)
+    out = _np(st.step())
+    torch.cuda.synchronize()
+    assert np.isfinite(out).all()
+    rows = _config4_rows(wl, n_random=24)
+    _check(out[rows], _oracle_prefill(wl, {0: rows}), "bf16")
+    # the literal mask is denser than the ancestor mask
+    assert st.plan.stats()["visible_pairs"] > 91435434
+
+
 # ------------------------------------------------------------------ mv_dag_decode_attn
 
 @pytest.mark.parametrize("chunk", [0, 16, 64])
@@ -314,6 +328,20 @@ def test_decode_config3(frontier_layer):
     got = _np(st.step())
     torch.cuda.synchronize()
     assert np.isfinite(got).all()
+    check_decode(wl, got, requests=[0, 13, 31])
+
+
+@pytest.mark.parametrize("vis_mode,pos_mode", [(1, 1), (1, 0), (0, 1)])
+def test_decode_config3_paper_literal_modes(vis_mode, pos_mode):
+    # the mask of Eq. 3 read literally (every node of an earlier frontier layer is visible) and positions aligned per
+    # frontier, at full size
+    rt = _rt()
+    wl = synth.config3()
+    wl.batch.vis_mode, wl.batch.pos_mode = vis_mode, pos_mode
+    st = rt.DecodeState(wl)
+    got = _np(st.step())
+    torch.cuda.synchronize()
+    assert np.isfinite(got).all() and st.plan.read_status() == 0
     check_decode(wl, got, requests=[0, 13, 31])
 
 
