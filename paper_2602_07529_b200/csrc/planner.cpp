@@ -36,8 +36,6 @@ struct Bits {  // dense bitset rows, n_words per node
 
 // a decode stream: one per (request, row group): a run of stages and the rows of the group
 struct Seg { int32_t stage_begin, n_stages, rows_begin, n_rows; };
-// a partial slot to be numbered: (row, KV head), unit, row of the unit
-struct PartKey { int32_t rowkv, unit, k; };
 
 size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
@@ -131,7 +129,6 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     std::vector<int64_t> node_tok_start, cost_prefix;
     std::vector<char> seen_by_frontier, stage_plain;
     std::vector<Seg> segs;
-    std::vector<PartKey> keys;
   };
   static thread_local Scratch scratch;
   Scratch& sc = scratch;
@@ -141,7 +138,6 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   std::vector<int64_t>&node_tok_start = sc.node_tok_start, &cost_prefix = sc.cost_prefix;
   std::vector<char>&seen_by_frontier = sc.seen_by_frontier, &stage_plain = sc.stage_plain;
   std::vector<Seg>& segs = sc.segs;
-  std::vector<PartKey>& keys = sc.keys;
   node_tok_start.assign(size_t(n_nodes), 0);  // flattened index of a node's first NEW token
   int64_t unique_tokens = 0, per_row_tokens = 0, visible_pairs = 0, tile_pairs = 0;
   const int sched_kv_heads = b->n_kv_heads > 0 ? b->n_kv_heads : 8;
@@ -431,7 +427,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       return std::max<int64_t>((remaining + left * kUnitOverhead + left - 1) / left, 2 * kStage + kUnitOverhead);
     };
     P->cta_unit_off.assign(size_t(n_ctas) + 1, 0);
-    keys.clear();
+    P->rowkv_part_off.assign(size_t(n_rows) * sched_kv_heads + 1, 0);  // first counts, then offsets
     int cta = 0;
     int64_t acc = 0, target = share(0), max_acc = 0;
     const int64_t first_share = target;
@@ -451,8 +447,8 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       for (int32_t k = 0; k < sg.n_rows; ++k) {
         const int32_t row = seg_rows[size_t(sg.rows_begin + k)];
         const bool has = (seen >> k) & 1;
-        if (has) keys.push_back(PartKey{row * sched_kv_heads + kvh, int32_t(P->units.size()), k});
-        P->item_rows.push_back(ItemRow{row, -1});
+        if (has) P->rowkv_part_off[size_t(row) * sched_kv_heads + kvh + 1]++;
+        P->item_rows.push_back(ItemRow{row, has ? 0 : -1});  // 0: a slot is numbered below
       }
       P->units.push_back(wu);
       P->cta_unit_off[size_t(cta) + 1] = int32_t(P->units.size());
@@ -503,13 +499,15 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       P->cta_head[size_t(c)].pad[1] = ue;
     }
     // partial slots: contiguous per (row, KV head), in unit order
-    P->rowkv_part_off.assign(size_t(n_rows) * sched_kv_heads + 1, 0);
-    for (const PartKey& k : keys) P->rowkv_part_off[size_t(k.rowkv) + 1]++;
     for (size_t i = 1; i < P->rowkv_part_off.size(); ++i) P->rowkv_part_off[i] += P->rowkv_part_off[i - 1];
     next_part.assign(P->rowkv_part_off.begin(), P->rowkv_part_off.end() - 1);
-    for (const PartKey& k : keys) P->item_rows[size_t(P->units[k.unit].row_begin + k.k)].part = next_part[k.rowkv]++;
+    for (const WorkUnit& wu : P->units) {
+      ItemRow* ir = P->item_rows.data() + wu.row_begin;
+      for (int32_t k = 0; k < wu.n_rows; ++k)
+        if (ir[k].part == 0) ir[k].part = next_part[size_t(ir[k].row) * sched_kv_heads + wu.kvh]++;
+    }
     S.n_items = int64_t(P->units.size());
-    S.n_partials = int64_t(keys.size());
+    S.n_partials = int64_t(P->rowkv_part_off.back());
     S.n_ctas = n_ctas;
     S.chunk_tokens = chunk > 0 ? chunk : first_share;
   }
