@@ -116,7 +116,15 @@ typedef enum {
   MV_TAB_SEG_OFF = 6,       /* int32 [n_qnodes+1]   CSR over the q-node's visible segments                       */
   MV_TAB_SEG_NODE = 7,      /* int32 [n_segs]       global node index of the segment (ascending in a q-node)     */
   MV_TAB_SEG_LEN = 8,       /* int32 [n_segs]       node_len + node_new of that node                             */
-  MV_TAB_KV_LEN = 9         /* int64 [n_qnodes]     tokens visible to the last new token of the q-node           */
+  MV_TAB_KV_LEN = 9,        /* int64 [n_qnodes]     tokens visible to the last new token of the q-node           */
+  /* The decode kernels' work lists, as int32 words, for tests that replay them on the host (the layout is the
+   * kernels' own and may change): */
+  MV_TAB_WORK_STAGES = 10,        /* 16 words per stage: page[4], valid tokens (a byte per page slot), page slots
+                                     in use, row mask low word [4], row mask high word [4], 2 unused              */
+  MV_TAB_WORK_UNITS = 11,         /* 8 words per unit: first stage, stages, first item row, rows, KV head, 3 unused */
+  MV_TAB_WORK_ITEM_ROWS = 12,     /* 2 words per (unit, row): row, first partial slot or -1                       */
+  MV_TAB_WORK_CTA_UNIT_OFF = 13,  /* [n_ctas + 1] CSR over the units of every share                               */
+  MV_TAB_WORK_ROWKV_PART_OFF = 14 /* [n_rows * n_kv_heads + 1] CSR over the partial slots of a (row, KV head)     */
 } mv_plan_table_id;
 
 typedef struct {

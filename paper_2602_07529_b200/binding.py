@@ -22,6 +22,8 @@ OP_ROPE_WRITE_KV, OP_DECODE_ATTN, OP_PREFILL_ATTN = 0, 1, 2
 TABLES = {"layer": (0, np.int32), "pos_start": (1, np.int32), "pos_id": (2, np.int32), "slot": (3, np.int64),
           "qnode": (4, np.int32), "qnode_tok_off": (5, np.int32), "seg_off": (6, np.int32),
           "seg_node": (7, np.int32), "seg_len": (8, np.int32), "kv_len": (9, np.int64)}
+# the decode kernels' work lists as int32 words (read by tests that replay them on the host)
+WORK_TABLES = {"stages": 10, "units": 11, "item_rows": 12, "cta_unit_off": 13, "rowkv_part_off": 14}
 
 EXPORTS = ["mv_plan_dag", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_bytes", "mv_plan_upload",
            "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
@@ -181,6 +183,14 @@ class Plan:
             return np.zeros(0, dt)
         buf = (C.c_char * (n.value * np.dtype(dt).itemsize)).from_address(p.value)
         return np.frombuffer(buf, dtype=dt).copy()
+
+    def work_table(self, name: str) -> np.ndarray:
+        p, n = C.c_void_p(), C.c_int64()
+        _check(lib.mv_plan_table(self._h, WORK_TABLES[name], C.byref(p), C.byref(n)), "mv_plan_table")
+        if n.value == 0:
+            return np.zeros(0, np.int32)
+        buf = (C.c_char * (n.value * 4)).from_address(p.value)
+        return np.frombuffer(buf, dtype=np.int32).copy()
 
     def stats(self) -> dict:
         s = _Stats()

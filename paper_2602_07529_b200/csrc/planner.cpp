@@ -576,6 +576,14 @@ extern "C" mv_status mv_plan_table(const mv_plan* P, int which, const void** hos
     case MV_TAB_SEG_NODE: return give32(P->seg_node);
     case MV_TAB_SEG_LEN: return give32(P->seg_len);
     case MV_TAB_KV_LEN: return give64(P->kv_len);
+    case MV_TAB_WORK_STAGES:
+      *host_ptr = P->stages.data(); *count = int64_t(P->stages.size()) * int64_t(sizeof(StageDesc) / 4); return MV_OK;
+    case MV_TAB_WORK_UNITS:
+      *host_ptr = P->units.data(); *count = int64_t(P->units.size()) * int64_t(sizeof(WorkUnit) / 4); return MV_OK;
+    case MV_TAB_WORK_ITEM_ROWS:
+      *host_ptr = P->item_rows.data(); *count = int64_t(P->item_rows.size()) * 2; return MV_OK;
+    case MV_TAB_WORK_CTA_UNIT_OFF: return give32(P->cta_unit_off);
+    case MV_TAB_WORK_ROWKV_PART_OFF: return give32(P->rowkv_part_off);
     default: return MV_ERR_INVALID_ARG;
   }
 }
