@@ -147,6 +147,9 @@ typedef struct {
   int64_t n_ctas;              /* decode: CTAs the step was cut for                                         */
   int64_t max_cta_cost;        /* decode: largest share handed to one CTA, in tokens of one KV head (a unit
                                   counts as its tokens + 48)                                                */
+  int64_t append_tiles;        /* node append: 128-row query tiles over the paged cache (0 when no node of a
+                                  decode_ready batch receives several tokens)                               */
+  int64_t max_node_new;        /* most new tokens any node receives                                         */
 } mv_plan_stats;
 
 enum { MV_OP_ROPE_WRITE_KV = 0, MV_OP_DECODE_ATTN = 1, MV_OP_PREFILL_ATTN = 2 };
@@ -208,7 +211,9 @@ mv_status mv_rope_write_kv(const mv_plan* plan, const mv_attn_geom* geom, const 
  * written to a node at once): a node may receive up to 256 new tokens, one row each in (node, token) order; new
  * token j of v then sees v's tokens 0 .. node_len(v) + j and every other visible node in full.  In a request
  * where some node receives several tokens, the nodes that receive tokens must not see one another, else the
- * plan is not decode_ready.
+ * plan is not decode_ready.  With head_dim 128, an even group size, 16-byte aligned q_rot and out, and some
+ * node receiving at least 48 tokens, the step runs as 128-row query tiles over the paged cache (a node's
+ * history is then read once per 128 new tokens); the workspace is still required but left untouched.
  *   q_rot   device [n_rows][n_q_heads][head_dim]  bf16
  *   k_pages, v_pages  device pools, bf16
  *   out     device [n_rows][n_q_heads][head_dim]  bf16

@@ -57,7 +57,8 @@ class _Stats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "n_nodes", "n_new_tokens", "n_qnodes", "n_segs", "decode_ready", "prefill_ready", "n_items", "n_partials",
         "chunk_tokens", "unique_kv_tokens", "per_row_kv_tokens", "n_q_tiles", "visible_pairs", "tile_pairs",
-        "max_page_id", "max_item_rows", "sched_kv_heads", "sched_group", "n_ctas", "max_cta_cost")]
+        "max_page_id", "max_item_rows", "sched_kv_heads", "sched_group", "n_ctas", "max_cta_cost", "append_tiles",
+        "max_node_new")]
 
 
 class _SchedStats(C.Structure):

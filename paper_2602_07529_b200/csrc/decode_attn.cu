@@ -27,6 +27,8 @@
 #include "common.cuh"
 
 namespace mv {
+mv_status append_tc(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_pages, const void* v_pages, void* out,
+                    cudaStream_t st);
 mv_status decode_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* kp, const void* vp, void* ws,
                     cudaStream_t st);
 }
@@ -694,6 +696,11 @@ extern "C" mv_status mv_dag_decode_attn(const mv_plan* P, const mv_attn_geom* g,
   const size_t need = mv_workspace_bytes(P, g, MV_OP_DECODE_ATTN);
   if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return MV_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  // Node append with long runs of new tokens: 128-row query tiles over the paged cache read a node's history once per
+  // 128 rows, where the decode kernels' row groups read it once per 64 / group_size rows.
+  if (P->stats.append_tiles > 0 && P->stats.max_node_new >= mv::kAppendTileTokens && g->head_dim == 128 &&
+      (g->n_q_heads / g->n_kv_heads) % 2 == 0 && (reinterpret_cast<uintptr_t>(q_rot) & 15) == 0 && (reinterpret_cast<uintptr_t>(out) & 15) == 0)
+    return mv::append_tc(P, g, q_rot, k_pages, v_pages, out, s);
   return g->head_dim == 128 ? launch<128>(P, g, q_rot, k_pages, v_pages, out, workspace, s)
                             : launch<64>(P, g, q_rot, k_pages, v_pages, out, workspace, s);
 }

@@ -10,6 +10,8 @@
 namespace mv {
 
 constexpr int kPrefillQTile = 128;   // query rows per prefill tile (tiles never straddle a node)
+constexpr int kAppendTileTokens = 48;  // a node that receives at least this many tokens sends the step to the tiled kernel
+                                       // (measured break-even against the row-group kernels: about 44 tokens per node)
 constexpr int kMaxAppendTokens = 256;  // most new tokens per node that the decode path takes (beyond that: prefill only)
 constexpr int kPrefillKvTile = 64;   // granularity used only for the executed-pairs statistic
 
@@ -39,18 +41,24 @@ struct ItemRow {
                  // or -1 if the row sees none of the unit's stages
 };
 // One prefill query tile: rows [q_start, q_start+q_len) of one node and the KV ranges they may see.
+// Two forms.  Flat (prefill: every token is new, K / V come as token-ordered arrays): q and key indices are flattened
+// token indices.  Paged (node append: the tile's rows are new tokens of one node, K / V come from the page pool): a
+// range is one whole node, keys are counted inside the node (kv_start = 0) and `pages` is the index of the node's
+// first page in the plan's page table; the causal range is the tile's own node.
 struct QTile {
   int32_t q_start, q_len, range_begin, range_count;
+  int32_t causal_base;  // index, in the causal range's key numbering, of the tile's first query (flat: = q_start)
+  int32_t pad[3];
 };
 struct KvRange {
   int32_t kv_start, kv_len;
-  int32_t causal;  // 1: key j is visible to query i only if j <= i (flattened token indices)
-  int32_t pad;
+  int32_t causal;  // 1: key j is visible to query i only if j <= causal_base + i
+  int32_t pages;   // paged form: index of the node's first page in the page table; flat form: 0
 };
 
 struct DeviceLayout {  // byte offsets into the device table buffer (all multiples of 256)
   size_t pos_id = 0, slot = 0, stages = 0, units = 0, cta_unit_off = 0, cta_head = 0, item_rows = 0, rowkv_part_off = 0, sched = 0,
-         q_tiles = 0, kv_ranges = 0, total = 0;
+         q_tiles = 0, kv_ranges = 0, page_tab = 0, total = 0;
 };
 
 }  // namespace mv
@@ -69,6 +77,7 @@ struct mv_plan {
   int32_t sched_zero[64] = {};  // device-side status words ([2] = status of bounded waits), uploaded as zeros
   std::vector<mv::QTile> q_tiles;
   std::vector<mv::KvRange> kv_ranges;
+  std::vector<int32_t> page_tab;         // paged tiles only: the batch's page ids
   mv_plan_stats stats{};
   int32_t page_size = 16;
   bool valid = false;

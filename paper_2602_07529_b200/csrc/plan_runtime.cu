@@ -56,6 +56,7 @@ extern "C" mv_status mv_plan_upload(mv_plan* P, void* device_buf, size_t device_
   std::memcpy(h + L.sched, P->sched_zero, sizeof(P->sched_zero));
   put(h, L.q_tiles, P->q_tiles);
   put(h, L.kv_ranges, P->kv_ranges);
+  put(h, L.page_tab, P->page_tab);
   // only the bytes in use travel (the tail of the last table)
   if (cudaMemcpyAsync(device_buf, h, need, cudaMemcpyHostToDevice, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
     (void)cudaGetLastError();

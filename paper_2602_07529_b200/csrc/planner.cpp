@@ -108,14 +108,18 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   P->seg_off.assign(1, 0);
   P->seg_node.clear(); P->seg_len.clear(); P->kv_len.clear();
   P->units.clear(); P->cta_unit_off.clear(); P->cta_head.clear(); P->item_rows.clear(); P->rowkv_part_off.clear();
-  P->q_tiles.clear(); P->kv_ranges.clear();
+  P->q_tiles.clear(); P->kv_ranges.clear(); P->page_tab.clear();
   P->stages.clear();
   mv_plan_stats S{};
   S.n_nodes = n_nodes;
   S.max_page_id = max_page;
 
-  bool decode_ready = true, prefill_ready = true;
+  bool decode_ready = true, prefill_ready = true, any_multi = false;
+  int32_t max_new = 0;
+  int64_t append_tiles = 0;
   for (int g = 0; g < n_nodes; ++g) {
+    any_multi |= b->node_new[g] > 1;
+    max_new = std::max(max_new, b->node_new[g]);
     if (b->node_new[g] > mv::kMaxAppendTokens) decode_ready = false;
     if (b->node_len[g] != 0) prefill_ready = false;
   }
@@ -352,6 +356,35 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
       }
     }
 
+    // ---- node append: paged query tiles of this request (128 new tokens of one node; one range per visible node,
+    // the node's own range causal).  Built whenever some node of the batch receives several tokens; which kernel
+    // runs the step is the launcher's choice.
+    if (decode_ready && !prefill_ready && any_multi) {
+      for (int v = 0; v < n; ++v) {
+        const int g = lo + v;
+        const int32_t nn = b->node_new[g], old_len = b->node_len[g];
+        for (int32_t q0 = 0; q0 < nn; q0 += mv::kPrefillQTile) {
+          const int32_t ql = std::min<int32_t>(mv::kPrefillQTile, nn - q0);
+          QTile qt{};
+          qt.q_start = int32_t(node_tok_start[g]) + q0;
+          qt.q_len = ql;
+          qt.range_begin = int32_t(P->kv_ranges.size());
+          qt.causal_base = old_len + q0;
+          for (int u = 0; u < n; ++u) {
+            if (u == v) {
+              P->kv_ranges.push_back(KvRange{0, old_len + q0 + ql, 1, b->page_off[g]});
+            } else if (vis.get(v, u)) {
+              const int32_t lu = b->node_len[lo + u] + b->node_new[lo + u];
+              if (lu > 0) P->kv_ranges.push_back(KvRange{0, lu, 0, b->page_off[lo + u]});
+            }
+          }
+          qt.range_count = int32_t(P->kv_ranges.size()) - qt.range_begin;
+          P->q_tiles.push_back(qt);
+          ++append_tiles;
+        }
+      }
+    }
+
     // ---- prefill tiles of this request
     if (prefill_ready) {
       // flattened start of every node of the request
@@ -374,8 +407,9 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
         visible_pairs += vis_before * len_v + int64_t(len_v) * (len_v + 1) / 2;
         for (int32_t q0 = 0; q0 < len_v; q0 += mv::kPrefillQTile) {
           const int32_t ql = std::min<int32_t>(mv::kPrefillQTile, len_v - q0);
-          QTile qt;
+          QTile qt{};
           qt.q_start = int32_t(v_start + q0);
+          qt.causal_base = qt.q_start;
           qt.q_len = ql;
           qt.range_begin = int32_t(P->kv_ranges.size());
           // own causal range [v_start, q_start + q_len), placed in flattened order.  A fully visible
@@ -511,8 +545,10 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     S.n_ctas = n_ctas;
     S.chunk_tokens = chunk > 0 ? chunk : first_share;
   }
-  // ---- prefill: heaviest query tiles first
-  if (prefill_ready) {
+  if (!(decode_ready && !prefill_ready && any_multi)) append_tiles = 0;  // a later request took the batch off the decode path
+  if (append_tiles > 0) P->page_tab.assign(b->page_idx, b->page_idx + b->page_off[n_nodes]);
+  // ---- prefill and node append: heaviest query tiles first
+  if (prefill_ready || append_tiles > 0) {
     std::vector<int64_t> cost(P->q_tiles.size(), 0);
     for (size_t i = 0; i < P->q_tiles.size(); ++i)
       for (int k = 0; k < P->q_tiles[i].range_count; ++k) cost[i] += P->kv_ranges[P->q_tiles[i].range_begin + k].kv_len;
@@ -523,9 +559,13 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     sorted.reserve(order.size());
     for (int32_t i : order) sorted.push_back(P->q_tiles[i]);
     P->q_tiles.swap(sorted);
-    S.n_q_tiles = int64_t(P->q_tiles.size());
-    S.visible_pairs = visible_pairs;
-    S.tile_pairs = tile_pairs;
+    if (prefill_ready) {
+      S.n_q_tiles = int64_t(P->q_tiles.size());
+      S.visible_pairs = visible_pairs;
+      S.tile_pairs = tile_pairs;
+    } else {
+      S.append_tiles = int64_t(P->q_tiles.size());
+    }
   }
 
   S.n_new_tokens = new_tok_count;
@@ -537,6 +577,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   S.sched_group = sched_group;
   S.unique_kv_tokens = unique_tokens;
   S.per_row_kv_tokens = per_row_tokens;
+  S.max_node_new = max_new;
   P->stats = S;
 
   // ---- device table layout
@@ -554,6 +595,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   L.sched = place(sizeof(P->sched_zero));
   L.q_tiles = place(P->q_tiles.size() * sizeof(QTile));
   L.kv_ranges = place(P->kv_ranges.size() * sizeof(KvRange));
+  L.page_tab = place(P->page_tab.size() * sizeof(int32_t));
   L.total = std::max<size_t>(off, 256);
   P->layout = L;
   P->valid = true;

@@ -13,6 +13,11 @@
 // log2 units, P written back over S as packed bf16, O rescaled in tensor memory only when the row maximum
 // moved by more than 2^8, final normalisation and store).  The issuer alternates the two heads, so one
 // group's softmax overlaps the other head's products.  Every mbarrier wait is bounded (status word).
+//
+// The same kernel in its PAGED form serves node append (several new tokens of a node against the page pool, Sec. 4.3):
+// a KV range is then one whole visible node, its 128-key tiles are gathered page by page (one 2 KB box per page and
+// column block, the pool layout of the decode kernels), keys are counted inside the node, and the causal range is the
+// tile's own node with the first query sitting at key index causal_base.
 #include "common.cuh"
 #include "umma.cuh"
 
@@ -38,18 +43,20 @@ struct Bars {  // shared-memory addresses
 struct PrefillArgs {
   const mv::QTile* q_tiles;
   const mv::KvRange* ranges;
+  const int32_t* page_tab;  // paged form: page ids, indexed by KvRange::pages + key / 16
   bf16* out;
   int32_t* status;
-  int Hq, G;
+  int Hq, Hkv, G;
   float scale_log2;
 };
 
 // The KV tiles of a query tile, in the order every role walks them: ranges in table order, 128 keys at a time;
-// a causal range stops after the tile's last query.
+// a causal range stops after the tile's last query (q_last: its index in the causal range's key numbering).
 struct TileIter {
   const mv::KvRange* rg;
   int n_ranges, q_last;
   int ri = 0, pos = 0, end = 0, causal = 0;
+  int pages = 0;    // paged form: first page-table index of the current range
   mv::KvRange nxt;  // the range after the current one, read one range ahead so that no load sits on the walk
   __device__ TileIter(const mv::KvRange* r, int n, int ql) : rg(r), n_ranges(n), q_last(ql) {
     nxt = n > 0 ? r[0] : mv::KvRange{0, 0, 0, 0};
@@ -63,6 +70,7 @@ struct TileIter {
       pos = r.kv_start;
       end = r.kv_start + r.kv_len;
       causal = r.causal;
+      pages = r.pages;
       if (causal) end = min(end, q_last + 1);
     }
     start = pos;
@@ -85,16 +93,50 @@ struct Waiter {  // bounded waits: after one ran out every later wait returns at
   }
 };
 
+template <bool PAGED>
 __device__ __forceinline__ void producer_warp(const mv::QTile& qt, const PrefillArgs& a, int h0, int kvh, uint32_t smem_base,
                                               const Bars& br, const Waiter& w, const CUtensorMap* tm_q, const CUtensorMap* tm_k,
                                               const CUtensorMap* tm_v) {
-  if ((threadIdx.x & 31) != 0) return;
-  mv::mbar_arrive_expect_tx(br.q_full, 2 * TILE_BYTES);
-  for (int i = 0; i < 2; ++i)
-    for (int h = 0; h < 2; ++h)
-      mv::tma_load_2d(smem_base + OFF_Q + i * TILE_BYTES + h * (TILE_BYTES / 2), tm_q, (h0 + i) * D + h * 64, qt.q_start, br.q_full);
-  TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.q_start + qt.q_len - 1);
+  const int lane = threadIdx.x & 31;
+  if (!PAGED && lane != 0) return;  // flat form: one thread issues the few large boxes of a tile
+  if (lane == 0) {
+    mv::mbar_arrive_expect_tx(br.q_full, 2 * TILE_BYTES);
+    for (int i = 0; i < 2; ++i)
+      for (int h = 0; h < 2; ++h)
+        mv::tma_load_2d(smem_base + OFF_Q + i * TILE_BYTES + h * (TILE_BYTES / 2), tm_q, (h0 + i) * D + h * 64, qt.q_start, br.q_full);
+  }
+  TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.causal_base + qt.q_len - 1);
   int start, n, c, e = 0;  // e: ring entries issued so far
+  if (PAGED) {
+    // Paged form: a tile is gathered page by page, one 2 KB box per (page, column block).  Lane l < 16 owns page l / 2,
+    // column block l % 2 of every tile; it reads its page id one tile ahead, so no load sits between two tiles.
+    const int p = lane >> 1, h = lane & 1;
+    auto page_of = [&](bool valid, int st_, int n_) {
+      return (valid && lane < 16 && p < ((n_ + 15) >> 4)) ? __ldg(a.page_tab + it.pages + (st_ >> 4) + p) : -1;
+    };
+    bool more = it.next(start, n, c);
+    int page = page_of(more, start, n);
+    while (more) {
+      int start2 = 0, n2 = 0, c2 = 0;
+      const int n_pg = (n + 15) >> 4;
+      const bool more2 = it.next(start2, n2, c2);
+      const int page2 = page_of(more2, start2, n2);
+      for (int kv = 0; kv < 2; ++kv, ++e) {
+        const int slot = e % RING;
+        const uint32_t bar = br.kv_full + 8 * slot;
+        if (lane == 0) {
+          w.wait(br.kv_empty + 8 * slot, ((e / RING) & 1) ^ 1);
+          mv::mbar_arrive_expect_tx(bar, uint32_t(n_pg) * 4096u);
+        }
+        __syncwarp();
+        if (page >= 0)
+          mv::tma_load_2d(smem_base + OFF_RING + slot * TILE_BYTES + h * (TILE_BYTES / 2) + p * 2048, kv ? tm_v : tm_k, 0,
+                          ((page * a.Hkv + kvh) * 2 + h) * 16, bar);
+      }
+      more = more2; start = start2; n = n2; c = c2; page = page2;
+    }
+    return;
+  }
   while (it.next(start, n, c)) {
     for (int kv = 0; kv < 2; ++kv, ++e) {
       const int slot = e % RING;
@@ -128,10 +170,11 @@ __device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint6
     if (k < k_steps) mv::um::mma_ts<true>(o_tmem, p_tmem + k * 8, v_desc + uint32_t((k * 2048) >> 4), idesc);
 }
 
-__device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs& a, uint32_t smem_base, uint32_t tmem, const Bars& br,
-                                         const Waiter& w) {
+template <bool PAGED>
+__device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs& a, unsigned char* smem, uint32_t smem_base, uint32_t tmem,
+                                         const Bars& br, const Waiter& w) {
   if ((threadIdx.x & 31) != 0) return;
-  TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.q_start + qt.q_len - 1);
+  TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.causal_base + qt.q_len - 1);
   int start, n_cur, n_next = 0, c;
   if (!it.next(start, n_cur, c)) return;
   bool more = it.next(start, n_next, c);
@@ -154,6 +197,15 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
     const int ev = 2 * j + 1, ek = 2 * j + 2;  // ring entries of V_j and K_{j+1}
     const int k_steps = (n_cur + 15) >> 4;
     wait_full(ev);
+    if (PAGED && (n_cur & 15)) {
+      // the last page of a node is not full: its rows past the last key hold whatever the pool held; V must be zero
+      // where P is zero, or 0 * NaN would poison O
+      unsigned char* vt = smem + OFF_RING + (ev % RING) * TILE_BYTES;
+      for (int rr = n_cur; rr < k_steps * 16; ++rr)
+        for (int i = 0; i < 16; ++i)
+          *reinterpret_cast<uint4*>(vt + (i >> 3) * (TILE_BYTES / 2) + rr * 128 + ((i & 7) << 4)) = make_uint4(0, 0, 0, 0);
+      mv::fence_proxy_async();  // ordinary stores, read next by the tensor core
+    }
     w.wait(br.p_full, j & 1);
     mv::um::fence_after();
     issue_pv(o0, s0, v_desc(ev), j > 0, k_steps);
@@ -183,11 +235,12 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
                                               const Waiter& w) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = (warp & 3) * 32 + lane;                   // query row of the tile = tensor-memory lane
-  const int qi = qt.q_start + r;                          // flattened index of the query
+  const int qi = qt.q_start + r;                          // row of q and out
+  const int qc = qt.causal_base + r;                      // the query's index in the causal range's key numbering
   const uint32_t lane_base = tmem + (uint32_t((warp & 3) * 32) << 16);
   const uint32_t s_t = lane_base + i * 128, o_t = lane_base + 256 + i * 128;
   const uint32_t s_full = br.s_full + 8 * i, p_full = br.p_full + 8 * i, o_done = br.o_done + 8 * i;
-  TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.q_start + qt.q_len - 1);
+  TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.causal_base + qt.q_len - 1);
   float m = -INFINITY, l = 0.f;  // running maximum (log2 units) and sum of this row
   int start, n, causal, j = 0;
   while (it.next(start, n, causal)) {
@@ -201,13 +254,13 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
     mv::um::wait_ld();
     // mask the ragged end of the range and, on diagonal tiles, keys after the query; row maximum of the raw
     // scores with four independent chains (the softmax scale is positive, so it commutes with the maximum)
-    const bool need_mask = n < BK || (causal && start + BK - 1 > qt.q_start);
+    const bool need_mask = n < BK || (causal && start + BK - 1 > qt.causal_base);
     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
     if (!need_mask) {
 #pragma unroll
       for (int c = 0; c < BK; c += 2) mx4[(c >> 1) & 3] = mv::max3(mx4[(c >> 1) & 3], __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
     } else {
-      const int lim = causal ? min(n, qi - start + 1) : n;  // keys [0, lim) of the tile are visible to this row
+      const int lim = causal ? min(n, qc - start + 1) : n;  // keys [0, lim) of the tile are visible to this row
 #pragma unroll
       for (int c = 0; c < BK; ++c) {
         if (c >= lim) s[c] = __float_as_uint(-INFINITY);
@@ -281,6 +334,7 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
   }
 }
 
+template <bool PAGED>
 __global__ void __launch_bounds__(NTHREADS, 1) prefill_tc_kernel(const PrefillArgs a, const __grid_constant__ CUtensorMap tm_q,
                                                                  const __grid_constant__ CUtensorMap tm_k,
                                                                  const __grid_constant__ CUtensorMap tm_v) {
@@ -328,9 +382,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) prefill_tc_kernel(const PrefillAr
   const int h0 = blockIdx.y * 2, kvh = h0 / a.G;
   Waiter w{abort_flag, a.status};
   if (warp < 4) {
-    mv::um::reg_dec<48>();
-    if (warp == 0) producer_warp(qt, a, h0, kvh, smem_base, br, w, &tm_q, &tm_k, &tm_v);
-    else if (warp == 1) mma_warp(qt, a, smem_base, tmem, br, w);
+    mv::um::reg_dec<PAGED ? 56 : 48>();
+    if (warp == 0) producer_warp<PAGED>(qt, a, h0, kvh, smem_base, br, w, &tm_q, &tm_k, &tm_v);
+    else if (warp == 1) mma_warp<PAGED>(qt, a, smem, smem_base, tmem, br, w);
   } else {
     mv::um::reg_inc<224>();
     const int i = (warp - 4) >> 2;
@@ -343,7 +397,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) prefill_tc_kernel(const PrefillAr
 
 struct TcMaps {  // the last problem's tensor maps (pointers and token count rarely change between calls)
   const void *q = nullptr, *k = nullptr, *v = nullptr;
-  int64_t T = 0;
+  int64_t T = 0, pool_rows = 0;
   int Hq = 0, Hkv = 0;
   CUtensorMap tm_q, tm_k, tm_v;
 };
@@ -355,7 +409,7 @@ namespace mv {
 mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+    if (cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
       (void)cudaGetLastError();
       return MV_ERR_CUDA;
     }
@@ -376,11 +430,54 @@ mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, con
   a.ranges = mv::table<mv::KvRange>(P, P->layout.kv_ranges);
   a.out = static_cast<bf16*>(out);
   a.status = const_cast<int32_t*>(mv::table<int32_t>(P, P->layout.sched)) + 2;
+  a.page_tab = nullptr;
   a.Hq = g->n_q_heads;
+  a.Hkv = g->n_kv_heads;
   a.G = g->n_q_heads / g->n_kv_heads;
   a.scale_log2 = mv::softmax_scale(g) * 1.4426950408889634f;
   dim3 grid(unsigned(P->stats.n_q_tiles), unsigned(g->n_q_heads / 2));
-  prefill_tc_kernel<<<grid, NTHREADS, SMEM_BYTES, st>>>(a, tc.tm_q, tc.tm_k, tc.tm_v);
+  prefill_tc_kernel<false><<<grid, NTHREADS, SMEM_BYTES, st>>>(a, tc.tm_q, tc.tm_k, tc.tm_v);
+  mv::g_launches++;
+  return cudaGetLastError() == cudaSuccess ? MV_OK : MV_ERR_CUDA;
+}
+
+// Node append for head_dim 128 and an even group size: the paged form of the kernel over the plan's append tiles.
+// q_rot [n_rows][n_q_heads][128]; k_pages / v_pages the page pools (the new tokens' K / V already written).  Writes
+// the normalised output directly: no partials, no merge.  The caller has validated the arguments.
+mv_status append_tc(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_pages, const void* v_pages, void* out,
+                    cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return MV_ERR_CUDA;
+    }
+    attr_set = true;
+  }
+  const int64_t T = P->stats.n_new_tokens;
+  const int64_t pool_rows = g->num_pages * g->n_kv_heads * 2 * 16;  // 128-byte rows of a pool
+  static thread_local TcMaps tc;
+  if (!(tc.q == q_rot && tc.k == k_pages && tc.v == v_pages && tc.T == T && tc.Hq == g->n_q_heads && tc.Hkv == g->n_kv_heads &&
+        tc.pool_rows == pool_rows)) {
+    tc.q = nullptr;
+    if (!mv::make_tmap_bf16_2d(&tc.tm_q, q_rot, uint64_t(T), uint64_t(g->n_q_heads) * D, BQ) ||
+        !mv::make_tmap_bf16_2d(&tc.tm_k, k_pages, uint64_t(pool_rows), 64, 16) ||
+        !mv::make_tmap_bf16_2d(&tc.tm_v, v_pages, uint64_t(pool_rows), 64, 16))
+      return MV_ERR_CUDA;
+    tc.q = q_rot; tc.k = k_pages; tc.v = v_pages; tc.T = T; tc.Hq = g->n_q_heads; tc.Hkv = g->n_kv_heads; tc.pool_rows = pool_rows;
+  }
+  PrefillArgs a;
+  a.q_tiles = mv::table<mv::QTile>(P, P->layout.q_tiles);
+  a.ranges = mv::table<mv::KvRange>(P, P->layout.kv_ranges);
+  a.page_tab = mv::table<int32_t>(P, P->layout.page_tab);
+  a.out = static_cast<bf16*>(out);
+  a.status = const_cast<int32_t*>(mv::table<int32_t>(P, P->layout.sched)) + 2;
+  a.Hq = g->n_q_heads;
+  a.Hkv = g->n_kv_heads;
+  a.G = g->n_q_heads / g->n_kv_heads;
+  a.scale_log2 = mv::softmax_scale(g) * 1.4426950408889634f;
+  dim3 grid(unsigned(P->stats.append_tiles), unsigned(g->n_q_heads / 2));
+  prefill_tc_kernel<true><<<grid, NTHREADS, SMEM_BYTES, st>>>(a, tc.tm_q, tc.tm_k, tc.tm_v);
   mv::g_launches++;
   return cudaGetLastError() == cudaSuccess ? MV_OK : MV_ERR_CUDA;
 }

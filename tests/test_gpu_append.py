@@ -75,3 +75,37 @@ def test_append_of_256_tokens_and_refusal_beyond():
     # nodes that receive tokens and see one another are a prefill, not an append
     chain = synth.build_batch([[([], 10, 3), ([0], 0, 2)]])
     assert B.Plan(chain, 0, 2, 4).stats()["decode_ready"] == 0
+
+
+def test_long_runs_take_the_tiled_kernel_and_short_ones_the_row_group_kernel():
+    from paper_2602_07529_b200 import binding as B, runtime
+    # 150 new tokens per branch: two query tiles per branch, the second ragged; histories that end inside a page
+    wl = synth.config2(n_req=2, prefix=500, branches=3, branch_len=70, new_tokens=150)
+    st = _run_and_check(wl)
+    assert st.plan.stats()["append_tiles"] == 2 * 3 * 2
+    n0 = B.mv_launch_count()
+    st.step()
+    assert B.mv_launch_count() - n0 == 2      # RoPE + cache write, then the tiled kernel (no partials, no merge)
+    wl = synth.config2(n_req=2, prefix=500, branches=3, branch_len=70, new_tokens=8)
+    st = _run_and_check(wl)
+    n0 = B.mv_launch_count()
+    st.step()
+    assert B.mv_launch_count() - n0 == 3      # RoPE + cache write, row-group attention, merge
+    # an odd group size keeps the row-group kernels whatever the run length
+    wl = synth.Workload("append_odd_group", "decode", synth.Geometry(6, 2, 128, 16, "bf16"),
+                        synth.build_batch([[([], 200, 0), ([0], 30, 100)]], rng=np.random.default_rng(9)), 79)
+    st = _run_and_check(wl)
+    n0 = B.mv_launch_count()
+    st.step()
+    assert B.mv_launch_count() - n0 == 3
+
+
+def test_tiled_append_joins_empty_nodes_and_many_small_ranges():
+    # a join that starts with 64 tokens and sees five finished branches of odd lengths (every range ends inside a page),
+    # next to a branch that receives 33 tokens on top of 130
+    reqs = [[([], 100, 0), ([0], 17, 0), ([0], 1, 0), ([0], 31, 0), ([0], 16, 0), ([0], 129, 0), ([1, 2, 3, 4, 5], 0, 64),
+             ([0], 130, 33)]]
+    wl = synth.Workload("append_join", "decode", synth.Geometry(32, 8, 128, 16, "bf16"),
+                        synth.build_batch(reqs, rng=np.random.default_rng(11)), 80)
+    st = _run_and_check(wl)
+    assert st.plan.stats()["append_tiles"] == 2
