@@ -277,6 +277,18 @@ mv_status mv_decode_step_host(mv_plan* plan, const mv_attn_geom* geom, const voi
                               const void* v_host, void* out_host, void* k_pages, void* v_pages, void* staging,
                               size_t staging_bytes, void* cuda_stream);
 
+/* The same step starting from the batch description instead of a finished plan: the copies of q, k, v are
+ * enqueued first and travel while the host plans the step (mv_plan_dag into *plan, which is created when NULL
+ * and reused otherwise), then the step runs as in mv_decode_step_host.  The staging layout depends on the plan
+ * only behind the q / k / v / out copies; size the buffer with mv_decode_step_staging_bytes on a plan of a batch
+ * of the same shape (a too small buffer is refused with MV_ERR_WORKSPACE, possibly after the input copies were
+ * enqueued).  *plan must not have an upload in flight (synchronise the stream between steps that share a plan).
+ * Errors: those of mv_plan_dag and of mv_decode_step_host. */
+mv_status mv_decode_step_host_batch(const mv_dag_batch* batch, mv_plan** plan, const mv_attn_geom* geom,
+                                    const void* q_host, const void* k_host, const void* v_host, void* out_host,
+                                    void* k_pages, void* v_pages, void* staging, size_t staging_bytes,
+                                    void* cuda_stream);
+
 /* Reads the device-side status word of the kernels that last ran with this plan's uploaded tables: MV_OK, or
  * MV_ERR_TIMEOUT if a bounded wait inside a kernel ran out (the kernel then still terminated, with an
  * undefined result).  Copies 4 bytes device->host on `cuda_stream` and synchronises that stream.

@@ -27,7 +27,7 @@ WORK_TABLES = {"stages": 10, "units": 11, "item_rows": 12, "cta_unit_off": 13, "
 
 EXPORTS = ["mv_plan_dag", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_bytes", "mv_plan_upload",
            "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
-           "mv_dag_prefill_attn", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_status_string",
+           "mv_dag_prefill_attn", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_decode_step_host_batch", "mv_status_string",
            "mv_launch_count", "mv_plan_read_status", "mv_dag_decode_attn_static",
            "mv_static_workspace_bytes",
            "mv_sched_create", "mv_sched_destroy", "mv_sched_add_request", "mv_sched_step", "mv_sched_rows",
@@ -92,6 +92,7 @@ def _load():
     lib.mv_decode_step_staging_bytes.argtypes = [vp, C.POINTER(_Geom)]
     lib.mv_decode_step_staging_bytes.restype = sz
     lib.mv_decode_step_host.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 7 + [sz, vp]
+    lib.mv_decode_step_host_batch.argtypes = [C.POINTER(_DagBatch), C.POINTER(vp), C.POINTER(_Geom)] + [vp] * 7 + [sz, vp]
     lib.mv_status_string.argtypes = [C.c_int]
     lib.mv_status_string.restype = C.c_char_p
     lib.mv_plan_read_status.argtypes = [vp, vp, C.POINTER(i32)]
@@ -267,6 +268,13 @@ def mv_decode_step_host(plan: Plan, geom: _Geom, q_host, k_host, v_host, out_hos
     _check(lib.mv_decode_step_host(plan.handle, C.byref(geom), _ptr(q_host), _ptr(k_host), _ptr(v_host), _ptr(out_host),
                                    _ptr(k_pages), _ptr(v_pages), _ptr(staging),
                                    staging.numel() * staging.element_size(), _stream_ptr(stream)), "mv_decode_step_host")
+
+
+def mv_decode_step_host_batch(plan: Plan, geom: _Geom, q_host, k_host, v_host, out_host, k_pages, v_pages, staging, stream=None):
+    """Plans ``plan``'s batch again inside the call (the input copies travel meanwhile) and runs the step."""
+    _check(lib.mv_decode_step_host_batch(C.byref(plan.c_batch), C.byref(plan._h), C.byref(geom), _ptr(q_host), _ptr(k_host),
+                                         _ptr(v_host), _ptr(out_host), _ptr(k_pages), _ptr(v_pages), _ptr(staging),
+                                         staging.numel() * staging.element_size(), _stream_ptr(stream)), "mv_decode_step_host_batch")
 
 
 def mv_launch_count() -> int:

@@ -396,6 +396,14 @@ def test_decode_step_host_matches_device_calls():
     B.mv_decode_step_host(st.plan, st.geom, qh, kh, vh, oh, kp, vp, staging)
     torch.cuda.synchronize()
     assert torch.equal(oh, want.cpu())
+    # the form that plans inside the call (the input copies travel meanwhile): same bits, twice in a row
+    for _ in range(2):
+        oh.zero_()
+        B.mv_decode_step_host_batch(st.plan, st.geom, qh, kh, vh, oh, kp, vp, staging)
+        torch.cuda.synchronize()
+        assert torch.equal(oh, want.cpu())
+    with pytest.raises(B.MvError):   # a staging buffer that cannot even hold q, k, v and out
+        B.mv_decode_step_host_batch(st.plan, st.geom, qh, kh, vh, oh, kp, vp, staging[:256])
     # the plan now points at the staging buffer; restore it for later use of st
     st.plan.upload(st.pod.tables)
 
