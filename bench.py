@@ -298,6 +298,7 @@ def run_ours(args):
     extra = {}
     if rank == 0 and not args.no_prefill:
         extra["prefill"] = _prefill_leg(torch, B, runtime, synth, dev, peaks)
+        extra["append"] = _append_leg(torch, B, runtime, synth, dev, peaks)
     sampler.stop()
 
     if rank != 0:
@@ -367,6 +368,40 @@ def _prefill_leg(torch, B, runtime, synth, dev, peaks):
             "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"], "frac_of_nominal_2250": tf / 2250.0,
             "visible_pairs": stats["visible_pairs"], "tile_pairs": stats["tile_pairs"],
             "executed_tflops": 4.0 * g.head_dim * g.n_q_heads * stats["tile_pairs"] / (ms * 1e-3) / 1e12}
+
+
+def _append_leg(torch, B, runtime, synth, dev, peaks, new_tokens=128):
+    """Node append on the multi-branch workload: every branch receives ``new_tokens`` tokens at once against the paged
+    cache (the tiled form of mv_dag_decode_attn).  Useful flops count every (new token, visible key) pair once."""
+    wl = synth.config2(new_tokens=new_tokens)
+    st = runtime.DecodeState(wl, dev, n_pool_copies=2)
+    stats = st.plan.stats()
+    g, b = wl.geom, wl.batch
+    pairs = 0
+    for r in range(b.n_req):
+        lo, hi = int(b.node_off[r]), int(b.node_off[r + 1])
+        ln, nw = b.node_len[lo:hi].astype(np.int64), b.node_new[lo:hi].astype(np.int64)
+        # every workload of this shape is prefix + branches: a branch sees the prefix and itself
+        for v in range(1, hi - lo):
+            pairs += int(nw[v] * (ln[0] + ln[v]) + nw[v] * (nw[v] + 1) // 2)
+    flops = 4.0 * g.head_dim * g.n_q_heads * pairs
+    for i in range(3):
+        st.step(i % 2)
+    torch.cuda.synchronize()
+    evs = []
+    for i in range(10):
+        kp, vp = st.pools[i % 2]
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        B.mv_dag_decode_attn(st.plan, st.geom, st.q_rot, kp, vp, st.out, st.workspace)
+        c.record()
+        evs.append((a, c))
+    torch.cuda.synchronize()
+    ms = float(np.median([a.elapsed_time(c) for a, c in evs]))
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"workload": f"{wl.name}, {new_tokens} new tokens per branch", "rows": stats["n_new_tokens"],
+            "query_tiles": stats["append_tiles"], "ms": ms, "query_tokens_per_s": stats["n_new_tokens"] / (ms * 1e-3),
+            "visible_pairs": pairs, "useful_tflops": tf, "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"]}
 
 
 def main():
