@@ -173,7 +173,9 @@ __device__ __forceinline__ void issue_pv(uint32_t o_tmem, uint32_t p_tmem, uint6
 template <bool PAGED>
 __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs& a, unsigned char* smem, uint32_t smem_base, uint32_t tmem,
                                          const Bars& br, const Waiter& w) {
-  if ((threadIdx.x & 31) != 0) return;
+  // The whole warp walks the tiles and waits on the barriers; one elected lane issues the products and the commits.
+  // Descriptors and tensor-memory addresses are then computed in warp-uniform code.
+  const bool lead = mv::um::elect_one();
   TileIter it(a.ranges + qt.range_begin, qt.range_count, qt.causal_base + qt.q_len - 1);
   int start, n_cur, n_next = 0, c;
   if (!it.next(start, n_cur, c)) return;
@@ -183,21 +185,23 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
   auto k_desc = [&](int e) { return mv::um::smem_desc(smem_base + OFF_RING + (e % RING) * TILE_BYTES, 16, 1024); };
   auto v_desc = [&](int e) { return mv::um::smem_desc(smem_base + OFF_RING + (e % RING) * TILE_BYTES, TILE_BYTES / 2, 1024); };
   auto wait_full = [&](int e) { w.wait(br.kv_full + 8 * (e % RING), (e / RING) & 1); };
-  auto release = [&](int e) { mv::um::commit(br.kv_empty + 8 * (e % RING)); };
+  auto release = [&](int e) { if (lead) mv::um::commit(br.kv_empty + 8 * (e % RING)); };
   auto cols = [](int n) { return ((n + 15) >> 4) << 4; };  // score columns computed; the softmax groups mask the rest
   w.wait(br.q_full, 0);
   wait_full(0);
   mv::um::fence_after();
-  issue_qk(s0, q0, k_desc(0), cols(n_cur));
-  mv::um::commit(br.s_full);
-  issue_qk(s1, q1, k_desc(0), cols(n_cur));
-  mv::um::commit(br.s_full + 8);
+  if (lead) {
+    issue_qk(s0, q0, k_desc(0), cols(n_cur));
+    mv::um::commit(br.s_full);
+    issue_qk(s1, q1, k_desc(0), cols(n_cur));
+    mv::um::commit(br.s_full + 8);
+  }
   release(0);
   for (int j = 0;; ++j) {
     const int ev = 2 * j + 1, ek = 2 * j + 2;  // ring entries of V_j and K_{j+1}
     const int k_steps = (n_cur + 15) >> 4;
     wait_full(ev);
-    if (PAGED && (n_cur & 15)) {
+    if (PAGED && (n_cur & 15) && lead) {
       // the last page of a node is not full: its rows past the last key hold whatever the pool held; V must be zero
       // where P is zero, or 0 * NaN would poison O
       unsigned char* vt = smem + OFF_RING + (ev % RING) * TILE_BYTES;
@@ -206,24 +210,33 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
           *reinterpret_cast<uint4*>(vt + (i >> 3) * (TILE_BYTES / 2) + rr * 128 + ((i & 7) << 4)) = make_uint4(0, 0, 0, 0);
       mv::fence_proxy_async();  // ordinary stores, read next by the tensor core
     }
+    __syncwarp();  // the patch above is one lane's
     w.wait(br.p_full, j & 1);
     mv::um::fence_after();
-    issue_pv(o0, s0, v_desc(ev), j > 0, k_steps);
-    mv::um::commit(br.o_done);
+    if (lead) {
+      issue_pv(o0, s0, v_desc(ev), j > 0, k_steps);
+      mv::um::commit(br.o_done);
+    }
     if (more) {
       wait_full(ek);
       mv::um::fence_after();
-      issue_qk(s0, q0, k_desc(ek), cols(n_next));
-      mv::um::commit(br.s_full);
+      if (lead) {
+        issue_qk(s0, q0, k_desc(ek), cols(n_next));
+        mv::um::commit(br.s_full);
+      }
     }
     w.wait(br.p_full + 8, j & 1);
     mv::um::fence_after();
-    issue_pv(o1, s1, v_desc(ev), j > 0, k_steps);
-    mv::um::commit(br.o_done + 8);
+    if (lead) {
+      issue_pv(o1, s1, v_desc(ev), j > 0, k_steps);
+      mv::um::commit(br.o_done + 8);
+    }
     release(ev);
     if (!more) break;
-    issue_qk(s1, q1, k_desc(ek), cols(n_next));
-    mv::um::commit(br.s_full + 8);
+    if (lead) {
+      issue_qk(s1, q1, k_desc(ek), cols(n_next));
+      mv::um::commit(br.s_full + 8);
+    }
     release(ek);
     n_cur = n_next;
     more = it.next(start, n_next, c);
