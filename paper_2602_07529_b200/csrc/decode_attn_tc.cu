@@ -215,7 +215,9 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
 
 // ---- issuer warp of one half (one thread) ----------------------------------------------------------------
 __device__ __forceinline__ void issuer(const TcArgs& a, const Half& h) {
-  if ((threadIdx.x & 31) != 0) return;
+  // The whole warp walks the units and waits on the barriers; one elected lane issues the products and the commits, so
+  // that descriptors and tensor-memory addresses are computed in warp-uniform code.
+  const bool lead = mv::um::elect_one();
   Meta* meta = h.meta;
   int u_begin, u_end;
   {
@@ -235,13 +237,15 @@ __device__ __forceinline__ void issuer(const TcArgs& a, const Half& h) {
     mv::um::fence_after();
     const uint64_t k_desc = mv::um::smem_desc(h.stage_smem + sb * STAGE_BYTES, 16, 1024);
     const uint32_t s_t = h.tmem + (t & 1) * 64;
-    mv::um::mma_ss<false>(s_t, q_desc, k_desc, idesc_qk);
+    if (lead) {
+      mv::um::mma_ss<false>(s_t, q_desc, k_desc, idesc_qk);
 #pragma unroll
-    for (int k = 1; k < D / 16; ++k) {
-      const uint32_t qo = ((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4, ko = ((k >> 2) * (KV_BYTES / 2) + (k & 3) * 32) >> 4;
-      mv::um::mma_ss<true>(s_t, q_desc + qo, k_desc + ko, idesc_qk);
+      for (int k = 1; k < D / 16; ++k) {
+        const uint32_t qo = ((k >> 2) * (Q_BYTES / 2) + (k & 3) * 32) >> 4, ko = ((k >> 2) * (KV_BYTES / 2) + (k & 3) * 32) >> 4;
+        mv::um::mma_ss<true>(s_t, q_desc + qo, k_desc + ko, idesc_qk);
+      }
+      mv::um::commit(bar(&meta->s_full[t & 1]));
     }
-    mv::um::commit(bar(&meta->s_full[t & 1]));
     ++t;
   };
   for (int u = u_begin; u < u_end; ++u) {
@@ -251,11 +255,11 @@ __device__ __forceinline__ void issuer(const TcArgs& a, const Half& h) {
     const int n = meta->n_stages;
     const int t0 = t;  // stage s of this unit is score tile t0 + s: S / P buffer (t0 + s) & 1
     scores(g);
-    if (n == 1) mv::um::commit(bar(&meta->q_empty));  // the unit's last scores are queued: q tile free once they ran
+    if (n == 1 && lead) mv::um::commit(bar(&meta->q_empty));  // the unit's last scores are queued: q tile free once they ran
     for (int s = 0; s < n; ++s) {
       if (s + 1 < n) {
         scores(g + 1);
-        if (s + 2 == n) mv::um::commit(bar(&meta->q_empty));
+        if (s + 2 == n && lead) mv::um::commit(bar(&meta->q_empty));
       }
       if (s == 0 && ui > 0) wait_or_flag(h, bar(&meta->o_free), (ui - 1) & 1);  // the previous unit's O has been read
       const int sb = g % NSTAGES, T = t0 + s, pb = T & 1;
@@ -264,13 +268,15 @@ __device__ __forceinline__ void issuer(const TcArgs& a, const Half& h) {
       mv::um::fence_after();
       const uint64_t v_desc = mv::um::smem_desc(h.stage_smem + sb * STAGE_BYTES + KV_BYTES, KV_BYTES / 2, 1024);
       const uint32_t o_t = h.tmem + 128, p_t = h.tmem + pb * 64;
-      if (s == 0) mv::um::mma_ts<false>(o_t, p_t, v_desc, idesc_pv);
-      else mv::um::mma_ts<true>(o_t, p_t, v_desc, idesc_pv);
+      if (lead) {
+        if (s == 0) mv::um::mma_ts<false>(o_t, p_t, v_desc, idesc_pv);
+        else mv::um::mma_ts<true>(o_t, p_t, v_desc, idesc_pv);
 #pragma unroll
-      for (int k = 1; k < ST / 16; ++k)
-        if (uint32_t(k) < n_pages) mv::um::mma_ts<true>(o_t, p_t + k * 8, v_desc + uint32_t((k * 2048) >> 4), idesc_pv);
-      mv::um::commit(bar(&meta->o_done));
-      mv::um::commit(bar(&meta->empty[sb]));
+        for (int k = 1; k < ST / 16; ++k)
+          if (uint32_t(k) < n_pages) mv::um::mma_ts<true>(o_t, p_t + k * 8, v_desc + uint32_t((k * 2048) >> 4), idesc_pv);
+        mv::um::commit(bar(&meta->o_done));
+        mv::um::commit(bar(&meta->empty[sb]));
+      }
       ++g;
     }
   }
