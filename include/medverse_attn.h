@@ -212,7 +212,7 @@ mv_status mv_rope_write_kv(const mv_plan* plan, const mv_attn_geom* geom, const 
  * token j of v then sees v's tokens 0 .. node_len(v) + j and every other visible node in full.  In a request
  * where some node receives several tokens, the nodes that receive tokens must not see one another, else the
  * plan is not decode_ready.  With head_dim 128, an even group size, 16-byte aligned q_rot and out, and some
- * node receiving at least 48 tokens, the step runs as 128-row query tiles over the paged cache (a node's
+ * node receiving at least 40 tokens, the step runs as 128-row query tiles over the paged cache (a node's
  * history is then read once per 128 new tokens); the workspace is still required but left untouched.
  *   q_rot   device [n_rows][n_q_heads][head_dim]  bf16
  *   k_pages, v_pages  device pools, bf16

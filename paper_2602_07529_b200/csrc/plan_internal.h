@@ -10,8 +10,8 @@
 namespace mv {
 
 constexpr int kPrefillQTile = 128;   // query rows per prefill tile (tiles never straddle a node)
-constexpr int kAppendTileTokens = 48;  // a node that receives at least this many tokens sends the step to the tiled kernel
-                                       // (measured break-even against the row-group kernels: about 44 tokens per node)
+constexpr int kAppendTileTokens = 40;  // a node that receives at least this many tokens sends the step to the tiled kernel
+                                       // (measured break-even against the row-group kernels: about 37 tokens per node)
 constexpr int kMaxAppendTokens = 256;  // most new tokens per node that the decode path takes (beyond that: prefill only)
 constexpr int kPrefillKvTile = 64;   // granularity used only for the executed-pairs statistic
 
