@@ -211,16 +211,15 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
       mv::fence_proxy_async();  // ordinary stores, read next by the tensor core
     }
     __syncwarp();  // the patch above is one lane's
+    // the next K tile is waited for here, while P of head 0 is still being computed, not between the two products below:
+    // that wait sat on head 0's chain (softmax -> P V -> next Q K^T -> softmax) in every step
+    if (more) wait_full(ek);
     w.wait(br.p_full, j & 1);
     mv::um::fence_after();
     if (lead) {
       issue_pv(o0, s0, v_desc(ev), j > 0, k_steps);
       mv::um::commit(br.o_done);
-    }
-    if (more) {
-      wait_full(ek);
-      mv::um::fence_after();
-      if (lead) {
+      if (more) {
         issue_qk(s0, q0, k_desc(ek), cols(n_next));
         mv::um::commit(br.s_full);
       }
