@@ -109,3 +109,15 @@ def test_tiled_append_joins_empty_nodes_and_many_small_ranges():
                         synth.build_batch(reqs, rng=np.random.default_rng(11)), 80)
     st = _run_and_check(wl)
     assert st.plan.stats()["append_tiles"] == 2
+
+
+def test_kernel_choice_at_the_run_length_threshold():
+    from paper_2602_07529_b200 import binding as B
+    # 40 new tokens on one node send the step to the tiled kernel (two launches per step), 39 keep the row groups (three)
+    for new, launches in ((40, 2), (39, 3)):
+        wl = synth.Workload("append_threshold", "decode", synth.Geometry(32, 8, 128, 16, "bf16"),
+                            synth.build_batch([[([], 150, 0), ([0], 21, new), ([0], 64, 3)]], rng=np.random.default_rng(new)), 81)
+        st = _run_and_check(wl)
+        n0 = B.mv_launch_count()
+        st.step()
+        assert B.mv_launch_count() - n0 == launches

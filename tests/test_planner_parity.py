@@ -119,3 +119,20 @@ def test_error_statuses():
     empty = synth.build_batch([])
     assert B.Plan(empty).stats()["n_new_tokens"] == 0
     assert B.Plan(synth.build_batch([[], [([], 3, 1)]])).stats()["n_new_tokens"] == 1
+
+
+def test_append_tiles_in_the_plan_statistics():
+    # node append: one 128-row query tile per 128 new tokens of a node, counted only when some node of a decode-ready
+    # batch receives several tokens
+    batch = synth.build_batch([[([], 300, 0), ([0], 70, 130), ([0], 5, 128), ([0], 40, 1)],
+                               [([], 50, 0), ([0], 0, 256)]], rng=np.random.default_rng(3))
+    st = B.Plan(batch, 0, 8, 4).stats()
+    assert st["decode_ready"] == 1 and st["prefill_ready"] == 0
+    assert st["max_node_new"] == 256
+    assert st["append_tiles"] == 2 + 1 + 1 + 2
+    single = synth.build_batch([[([], 300, 0), ([0], 70, 1), ([0], 5, 1)]], rng=np.random.default_rng(4))
+    st = B.Plan(single, 0, 8, 4).stats()
+    assert st["decode_ready"] == 1 and st["append_tiles"] == 0 and st["max_node_new"] == 1
+    fresh = synth.build_batch([[([], 0, 300), ([0], 0, 70)]], rng=np.random.default_rng(5))
+    st = B.Plan(fresh, 0, 8, 4).stats()
+    assert st["prefill_ready"] == 1 and st["append_tiles"] == 0 and st["n_q_tiles"] == 3 + 1
