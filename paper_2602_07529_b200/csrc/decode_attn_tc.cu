@@ -471,6 +471,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) decode_tc_kernel(const TcArgs a, 
   mv::um::fence_before();
   __syncthreads();
   mv::um::fence_after();
+  // launched with programmatic stream serialisation: everything above may overlap the tail of the kernel before (the
+  // RoPE + cache write of the step); nothing of q or of the pools is read before that grid has completed
+  mv::grid_dependency_wait();
   const int hi = warp < 4 ? (warp >> 1) : ((warp - 4) >> 2);  // which half this warp serves
   Half h;
   h.smem_base = smem_base;
@@ -548,8 +551,22 @@ mv_status decode_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, cons
   a.G = G;
   a.scale_log2 = mv::softmax_scale(g) * 1.4426950408889634f;
   const int n_shares = int(P->stats.n_ctas);
-  decode_tc_kernel<<<unsigned((n_shares + 1) / 2), NTHREADS, SMEM_BYTES, st>>>(a, hit->tm_k, hit->tm_v, n_shares);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(unsigned((n_shares + 1) / 2), 1, 1);
+  cfg.blockDim = dim3(NTHREADS, 1, 1);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, decode_tc_kernel, a, hit->tm_k, hit->tm_v, n_shares);
   mv::g_launches++;
-  return cudaGetLastError() == cudaSuccess ? MV_OK : MV_ERR_CUDA;
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return MV_ERR_CUDA;
+  }
+  return MV_OK;
 }
 }  // namespace mv

@@ -61,6 +61,9 @@ __global__ void __launch_bounds__(128) rope_write_kv_kernel(const T* q, const T*
   constexpr int CH = HALF / N;  // 16-byte chunks per half head
   __shared__ float cs[HALF], sn[HALF];
   const int t = blockIdx.x;
+  // a kernel launched behind this one with programmatic stream serialisation (the decode attention kernel) may become
+  // resident and run its set-up now; it waits for this grid's completion before it reads what is written here
+  mv::grid_dependency_launch_dependents();
   if (t >= n_tok) return;
   const int pos = pos_id[t];
   const int64_t sl = slot[t];
