@@ -16,7 +16,9 @@
  *   - Streams: `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *     The three kernel calls and mv_plan_upload are asynchronous; they return the launch status only.
  *   - Errors: an mv_status is returned; argument errors are found on the host before any launch.
- *     Kernels never trap.  mv_status_string() names a status.
+ *     Kernels never trap: every device-side wait is bounded; when one runs out the CTA issues nothing further, waits
+ *     (again bounded) for its copies and products in flight, frees its tensor memory and returns, and
+ *     mv_plan_read_status() then gives MV_ERR_TIMEOUT.  mv_status_string() names a status.
  *   - Layouts: q, k, v, q_rot, out are [tokens][heads][head_dim], row-major, element type
  *     mv_attn_geom.dtype.  The K and V page pools are separate buffers of the same element type, each
  *     [num_pages][n_kv_heads][head_dim / 64][page_size][64]: the block of one (page, KV head) is contiguous
@@ -46,7 +48,7 @@ typedef enum {
   MV_ERR_UNSUPPORTED = 4,      /* head_dim / dtype / group size / batch shape the kernel does not take  */
   MV_ERR_WORKSPACE = 5,        /* workspace or table buffer missing, too small or misaligned            */
   MV_ERR_CUDA = 6,             /* a CUDA runtime call failed (launch error, copy error)                 */
-  MV_ERR_TIMEOUT = 7           /* reserved for bounded device-side waits                                */
+  MV_ERR_TIMEOUT = 7           /* a bounded device-side wait ran out (read with mv_plan_read_status)    */
 } mv_status;
 
 /* Which nodes a token may attend to.  The paper states the mask twice, differently (Eq. 3 masks only
@@ -187,8 +189,9 @@ size_t mv_workspace_bytes(const mv_plan* plan, const mv_attn_geom* geom, int op)
 /* RoPE with adaptive positions fused into the KV-cache write (P(i) of Eq. 2 at the indices of Sec. 4.2).
  * For new token t (n = n_new_tokens of the plan):
  *   q_rot[t] = RoPE(q[t], pos_id[t]);  k_pages[slot[t]] = k_rot[t] = RoPE(k[t], pos_id[t]);  v_pages[slot[t]] = v[t].
- * RoPE pairs element i with i + head_dim/2; the angle pos * rope_base^(-2i/head_dim) and its cos / sin are
- * evaluated in double precision and rounded to float; the rotation is float; results are stored in `dtype`.
+ * RoPE pairs element i with i + head_dim/2; the angle pos * rope_base^(-2i/head_dim) and its reduction modulo
+ * pi/2 are evaluated in double precision, cos / sin of the reduced angle in float (within two float ulps of the
+ * double-precision values at any position); the rotation is float; results are stored in `dtype`.
  *   q       device [n][n_q_heads][head_dim]   raw queries, or NULL (then q_rot is not written)
  *   k, v    device [n][n_kv_heads][head_dim]  raw keys / values
  *   q_rot   device [n][n_q_heads][head_dim]   out (may alias q); NULL exactly when q is NULL
@@ -299,6 +302,23 @@ const char* mv_status_string(mv_status s);
 
 /* Number of kernel launches the library has issued in this process since load (diagnostic counter). */
 int64_t mv_launch_count(void);
+
+/* Self-tests (diagnostics; no counterpart in the paper, nothing of the attention path runs).
+ *
+ * mv_selftest_bounded_wait: every wait inside the kernels is bounded and reports through the plan's status word
+ * (mv_plan_read_status).  This call exercises that mechanism alone: one thread of a one-CTA kernel waits, with the
+ * same bounded wait and a limit of `limit_ns` nanoseconds (1 .. 100 000 000), on a barrier that nothing ever
+ * completes; when the limit has passed it records MV_ERR_TIMEOUT in the status word of `plan` (which must have been
+ * uploaded) and returns.  No copy or product is in flight, the context stays usable; upload the plan again to clear
+ * the word.  Asynchronous on `cuda_stream`.  Errors: MV_ERR_INVALID_ARG, MV_ERR_WORKSPACE, MV_ERR_CUDA.
+ *
+ * mv_selftest_tmap_cache: the launchers keep the tensor maps of recent calls in a small cache keyed by (device index,
+ * up to three base pointers, row count, one more word).  This call runs the same lookup on a private instance with
+ * four entries: returns 1 if the key is cached, else 0 after caching it (the oldest entry is replaced); reset != 0
+ * empties the instance first.  Host only. */
+mv_status mv_selftest_bounded_wait(const mv_plan* plan, uint64_t limit_ns, void* cuda_stream);
+int32_t mv_selftest_tmap_cache(int32_t device, const void* a, const void* b, const void* c, int64_t rows, int64_t aux,
+                               int32_t reset);
 
 #ifdef __cplusplus
 }

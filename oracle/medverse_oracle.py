@@ -321,7 +321,7 @@ def decode_request(batch, r, q_raw, k_raw, v, base=10000.0, scale=None, rows=Non
 
 def append_request(batch, r, q_raw, k_raw, v, base=10000.0, scale=None, rows=None):
     """Several new tokens per node against the existing cache (Sec. 4.3: what follows a Join or the Phase I -> II
-    hand-over, where generation "proceeds from the merged KV state" with more than one token to write at once).
+    hand-over, where generation continues on the joined KV state with more than one token to write at once).
 
     When some node receives more than one token, the nodes that receive tokens must not see one another (they are
     one frontier).  k_raw / v

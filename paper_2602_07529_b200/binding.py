@@ -29,7 +29,7 @@ EXPORTS = ["mv_plan_dag", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_
            "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
            "mv_dag_prefill_attn", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_decode_step_host_batch", "mv_status_string",
            "mv_launch_count", "mv_plan_read_status", "mv_dag_decode_attn_static",
-           "mv_static_workspace_bytes",
+           "mv_static_workspace_bytes", "mv_selftest_bounded_wait", "mv_selftest_tmap_cache",
            "mv_sched_create", "mv_sched_destroy", "mv_sched_add_request", "mv_sched_step", "mv_sched_rows",
            "mv_sched_commit", "mv_sched_page_refs", "mv_sched_get_stats"]
 
@@ -96,6 +96,9 @@ def _load():
     lib.mv_status_string.argtypes = [C.c_int]
     lib.mv_status_string.restype = C.c_char_p
     lib.mv_plan_read_status.argtypes = [vp, vp, C.POINTER(i32)]
+    lib.mv_selftest_bounded_wait.argtypes = [vp, C.c_uint64, vp]
+    lib.mv_selftest_tmap_cache.argtypes = [i32, vp, vp, vp, i64, i64, i32]
+    lib.mv_selftest_tmap_cache.restype = i32
     lib.mv_launch_count.argtypes = []
     lib.mv_launch_count.restype = i64
     lib.mv_sched_create.argtypes = [i32, i32, C.POINTER(vp)]
@@ -275,6 +278,17 @@ def mv_decode_step_host_batch(plan: Plan, geom: _Geom, q_host, k_host, v_host, o
     _check(lib.mv_decode_step_host_batch(C.byref(plan.c_batch), C.byref(plan._h), C.byref(geom), _ptr(q_host), _ptr(k_host),
                                          _ptr(v_host), _ptr(out_host), _ptr(k_pages), _ptr(v_pages), _ptr(staging),
                                          staging.numel() * staging.element_size(), _stream_ptr(stream)), "mv_decode_step_host_batch")
+
+
+def mv_selftest_bounded_wait(plan: Plan, limit_ns: int, stream=None):
+    """Lets one bounded device-side wait run out (nothing arrives at its barrier): the plan's status word then reads
+    MV_ERR_TIMEOUT.  Upload the plan again to clear it."""
+    _check(lib.mv_selftest_bounded_wait(plan.handle, int(limit_ns), _stream_ptr(stream)), "mv_selftest_bounded_wait")
+
+
+def mv_selftest_tmap_cache(device: int, a: int, b: int, c: int, rows: int, aux: int, reset: bool = False) -> bool:
+    """True if the key was already in the self-test instance of the launchers' tensor-map cache (else it is now)."""
+    return bool(lib.mv_selftest_tmap_cache(int(device), a, b, c, int(rows), int(aux), 1 if reset else 0))
 
 
 def mv_launch_count() -> int:

@@ -26,6 +26,31 @@ inline float softmax_scale(const mv_attn_geom* g) {
   return g->sm_scale != 0.f ? g->sm_scale : 1.0f / sqrtf(float(g->head_dim));
 }
 
+// Opt-in to more than 48 KB of dynamic shared memory.  cudaFuncSetAttribute applies to the CURRENT device only, so the
+// "already done" record is a bit per device (bit d of `done`; devices past 63 set the attribute on every call).
+template <typename Kernel>
+inline bool opt_in_smem(Kernel kernel, int bytes, std::atomic<uint64_t>& done) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return false;
+  }
+  const uint64_t bit = (dev >= 0 && dev < 64) ? (uint64_t(1) << dev) : 0;
+  if (bit && (done.load(std::memory_order_acquire) & bit)) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return false;
+  }
+  if (bit) done.fetch_or(bit, std::memory_order_release);
+  return true;
+}
+
+inline int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) (void)cudaGetLastError();
+  return dev;
+}
+
 template <typename T>
 inline const T* table(const mv_plan* p, size_t off) {
   return reinterpret_cast<const T*>(static_cast<const char*>(p->device_buf) + off);
@@ -44,6 +69,7 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
 }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -159,14 +185,17 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 // Bounded wait: polls until the phase completes or about `limit_ns` (default two seconds) have passed, then
-// returns false; the caller records the failure and carries on so that every barrier still completes.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint64_t limit_ns = 2000000000ull) {
+// returns false.  `abort` (optional, shared memory) is the CTA's "a wait ran out" flag: once another role has set
+// it, a wait on the slow path gives up as well instead of running out on its own.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint64_t limit_ns = 2000000000ull,
+                                                  const volatile int* abort = nullptr) {
   for (int i = 0; i < 64; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (;;) {
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
+    if (abort && *abort) return false;
     if (global_timer_ns() - t0 > limit_ns) return false;
   }
 }
@@ -198,6 +227,13 @@ __device__ __forceinline__ void cp_async_mbar_arrive_noinc(uint32_t bar) {
 // kernel of the stream to complete with its memory visible.
 __device__ __forceinline__ void grid_dependency_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+// Arrival on a device-wide counter: one atomic add that releases everything that happened before it in this thread
+// (including, through a CTA-level barrier, what other threads of the CTA stored) and acquires what earlier arrivals released.
+__device__ __forceinline__ int atomic_add_acq_rel_gpu(int32_t* p, int v) {
+  int old;
+  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;\n" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
 __device__ __forceinline__ void named_bar_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;\n" ::"r"(id), "r"(threads) : "memory");
 }

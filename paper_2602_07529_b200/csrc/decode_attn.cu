@@ -25,6 +25,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "tmap_cache.h"
 
 namespace mv {
 mv_status append_tc(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_pages, const void* v_pages, void* out,
@@ -101,12 +102,16 @@ struct Sync {
   int32_t* status;                        // global status word
 };
 
-__device__ __forceinline__ void wait_or_flag(const Sync& sy, uint32_t bar, uint32_t parity) {
-  if (*sy.abort) return;
-  if (!mv::mbar_wait_bounded(bar, parity)) {
+// Bounded wait.  False once a wait of this CTA has run out (this one or an earlier one): the producer then issues no
+// further copy and waits for those in flight; the consumers only read shared memory and finish their lists.
+__device__ __forceinline__ bool wait_or_flag(const Sync& sy, uint32_t bar, uint32_t parity) {
+  if (*sy.abort) return false;
+  if (!mv::mbar_wait_bounded(bar, parity, 2000000000ull, sy.abort)) {
+    if (!*sy.abort) atomicExch(sy.status, int(MV_ERR_TIMEOUT));
     *sy.abort = 1;
-    atomicExch(sy.status, int(MV_ERR_TIMEOUT));
+    return false;
   }
+  return true;
 }
 
 // ---- producer warp: walks the CTA's units; per unit the q-vectors + slot ids, then the KV stages -----------------
@@ -161,7 +166,8 @@ __device__ __forceinline__ void producer(const DecodeArgs& a, uint32_t smem_base
   UnitRegs wu1 = load_unit(u_begin + 1);
   mv::ItemRow ir0 = load_rows(wu, 0), ir1 = load_rows(wu, 32);
   StageRegs win = load_window(wu, 0);
-  for (int u = u_begin; u < u_end; ++u) {
+  bool ok = true;  // warp-uniform: no wait of this CTA has run out
+  for (int u = u_begin; u < u_end && ok; ++u) {
     const int ui = u - u_begin;
     const UnitRegs wu2 = load_unit(u + 2);
     const mv::ItemRow nir0 = load_rows(wu1, 0), nir1 = load_rows(wu1, 32);
@@ -169,8 +175,12 @@ __device__ __forceinline__ void producer(const DecodeArgs& a, uint32_t smem_base
     // ---- q-vectors and partial-slot ids of this unit
     const int n_qv = wu.n_rows * a.G;
     const int n_pad = min(MAXQV, (n_qv + 15) & ~15);
-    if (lane == 0) wait_or_flag(sy, sy.q_empty, (ui & 1) ^ 1);
-    __syncwarp();
+    {
+      int go = 1;
+      if (lane == 0) go = wait_or_flag(sy, sy.q_empty, (ui & 1) ^ 1) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, go, 0) != 0;
+    }
+    if (!ok) break;
     for (int x = lane; x < MAXQV; x += 32) {  // every lane takes part in the shuffles
       const int r = min(x / a.G, MAXQV - 1);
       const int p_lo = __shfl_sync(0xffffffffu, ir0.part, r & 31), p_hi = __shfl_sync(0xffffffffu, ir1.part, r & 31);
@@ -196,7 +206,7 @@ __device__ __forceinline__ void producer(const DecodeArgs& a, uint32_t smem_base
     if (lane == 0) mv::mbar_arrive(sy.q_full);
     // ---- KV stages, 32 descriptors per window
     StageRegs nxt;
-    for (int s = 0; s < wu.n_stages; ++s) {
+    for (int s = 0; s < wu.n_stages && ok; ++s) {
       if ((s & 31) == 0) {
         if (s > 0) win = nxt;
         nxt = load_window(wu, s + 32);
@@ -207,8 +217,12 @@ __device__ __forceinline__ void producer(const DecodeArgs& a, uint32_t smem_base
       const int n_pages = __shfl_sync(0xffffffffu, win.b.y, src);
       const int b = issued % NSTAGES;
       const uint32_t bar = sy.full + 8 * b;
-      if (lane == 0) wait_or_flag(sy, sy.empty + 8 * b, ((issued / NSTAGES) & 1) ^ 1);  // every consumer warp has released the buffer
-      __syncwarp();
+      {
+        int go = 1;
+        if (lane == 0) go = wait_or_flag(sy, sy.empty + 8 * b, ((issued / NSTAGES) & 1) ^ 1) ? 1 : 0;  // every consumer warp has released the buffer
+        ok = __shfl_sync(0xffffffffu, go, 0) != 0;
+      }
+      if (!ok) break;
       if (lane == src) {  // the lane that holds the descriptor publishes the page slots' token counts and row masks
         meta->st_tokens[b] = uint32_t(win.b.x);
         meta->st_mask[b][0] = make_uint2(uint32_t(win.b.z), uint32_t(win.c.z));
@@ -233,6 +247,15 @@ __device__ __forceinline__ void producer(const DecodeArgs& a, uint32_t smem_base
     ir0 = nir0;
     ir1 = nir1;
     win = nwin;
+  }
+  if (!ok) {
+    // a wait ran out: what is still in flight must land before the CTA may return (a bulk copy that completes into the
+    // shared memory of a CTA that has left corrupts whoever runs there next)
+    mv::cp_async_wait_all();
+    if (lane == 0)
+      for (int k = 1; k <= min(issued, NSTAGES); ++k)
+        (void)mv::mbar_wait_bounded(sy.full + 8 * ((issued - k) % NSTAGES), ((issued - k) / NSTAGES) & 1, 20000000ull);
+    __syncwarp();
   }
 }
 
@@ -589,39 +612,26 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const float* __restri
   for (int e = 0; e < E; e += 2) *reinterpret_cast<__nv_bfloat162*>(o + e) = __floats2bfloat162_rn(acc[e] * inv, acc[e + 1] * inv);
 }
 
-struct TmapCache {  // the pools rarely change between calls: keep the last pairs of tensor maps
-  const void* k = nullptr;
-  const void* v = nullptr;
-  int64_t rows = 0;
-  int d = 0;
+struct KvMaps {
   CUtensorMap tm_k, tm_v;
 };
 
 template <int D>
 mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* kp, const void* vp, void* out,
                  void* ws, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(decode_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<D>::SMEM) != cudaSuccess) {
-      (void)cudaGetLastError();
+  static std::atomic<uint64_t> opted_in{0};  // per device
+  if (!mv::opt_in_smem(decode_attn_kernel<D>, Cfg<D>::SMEM, opted_in)) return MV_ERR_CUDA;
+  static thread_local mv::KeyedCache<KvMaps, 4> cache;  // the pools rarely change between calls
+  const int64_t rows = g->num_pages * g->n_kv_heads * 16 * Cfg<D>::HALVES;  // 128-byte rows of the pool
+  const mv::TmapKey key{mv::current_device(), kp, vp, nullptr, rows, D};
+  KvMaps* hit = cache.find(key);
+  if (!hit) {
+    hit = cache.claim(key);
+    if (!mv::make_tmap_bf16_2d(&hit->tm_k, kp, uint64_t(rows), 64, 16 * Cfg<D>::HALVES) ||
+        !mv::make_tmap_bf16_2d(&hit->tm_v, vp, uint64_t(rows), 64, 16 * Cfg<D>::HALVES)) {
+      cache.drop();
       return MV_ERR_CUDA;
     }
-    attr_set = true;
-  }
-  static thread_local TmapCache tc[4];
-  static thread_local int tc_next = 0;
-  const int64_t rows = g->num_pages * g->n_kv_heads * 16 * Cfg<D>::HALVES;  // 128-byte rows of the pool
-  TmapCache* hit = nullptr;
-  for (auto& c : tc)
-    if (c.k == kp && c.v == vp && c.rows == rows && c.d == D) hit = &c;
-  if (!hit) {
-    hit = &tc[tc_next];
-    tc_next = (tc_next + 1) % 4;
-    hit->k = nullptr;
-    if (!mv::make_tmap_bf16_2d(&hit->tm_k, kp, uint64_t(rows), 64, 16 * Cfg<D>::HALVES) ||
-        !mv::make_tmap_bf16_2d(&hit->tm_v, vp, uint64_t(rows), 64, 16 * Cfg<D>::HALVES))
-      return MV_ERR_CUDA;
-    hit->k = kp; hit->v = vp; hit->rows = rows; hit->d = D;
   }
   const int G = g->n_q_heads / g->n_kv_heads;
   const size_t vecs = size_t(P->stats.n_partials) * size_t(G);

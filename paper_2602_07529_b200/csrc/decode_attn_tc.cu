@@ -13,9 +13,13 @@
 // before it waits for the softmax of stage s, O += P V with P read from tensor memory) and a softmax group of
 // four warps (thread r = q-vector r: page-granular DAG mask, online softmax in log2 units with lazy rescaling
 // of O, P written back over S as packed bf16, at the unit's end the partial (max, sum, O) goes to the workspace).
+// Every wait is bounded.  Once one has run out (or another role's has), a role issues nothing further: it leaves its
+// loops, the producer waits for the copies it still has in flight, the issuer for its products, and the CTA meets at
+// the final barrier, frees its tensor memory and returns with MV_ERR_TIMEOUT in the plan's status word.
 // The q tile is 64 rows; the tensor core works on 128, the upper 64 being whatever follows in shared memory:
 // rows are independent, and those results are never read.
 #include "common.cuh"
+#include "tmap_cache.h"
 #include "umma.cuh"
 
 namespace {
@@ -38,11 +42,12 @@ constexpr float RESCALE_THRESHOLD = 8.f;
 
 struct Meta {  // one per half
   int32_t pv[MAXQV];            // partial vector index of q-vector x (partial * G + head in group) or -1
-  int32_t n_stages, n_qv;
+  int32_t n_stages, n_qv;       // header of the unit whose q tile is staged
   uint32_t st_tokens[NSTAGES];  // per stage buffer: valid tokens of the four page slots, a byte each
   uint32_t st_pages[NSTAGES];   // per stage buffer: page slots in use
   uint2 st_mask[NSTAGES][4];    // per stage buffer and page slot: rows that see the slot's node (lo, hi)
   uint64_t full[NSTAGES], empty[NSTAGES], q_full, q_empty, s_full[2], p_full[2], o_done, o_free;
+  uint64_t drained;             // issuer, after a wait ran out: its products in flight have completed
   int abort;
 };
 static_assert(sizeof(Meta) <= META_BYTES, "meta area");
@@ -73,13 +78,21 @@ struct Half {  // what every role of one half needs
 
 __device__ __forceinline__ uint32_t bar(const void* p) { return mv::smem_u32(p); }
 
-__device__ __forceinline__ void wait_or_flag(const Half& h, uint32_t b, uint32_t parity) {
+// Bounded wait.  False once a wait of this half has run out (this one or an earlier one, of any role): the caller then
+// issues nothing further and leaves its loops.
+__device__ __forceinline__ bool wait_or_flag(const Half& h, uint32_t b, uint32_t parity) {
   volatile int* abort = &h.meta->abort;
-  if (*abort) return;
-  if (!mv::mbar_wait_bounded(b, parity)) {
+  if (*abort) return false;
+  if (!mv::mbar_wait_bounded(b, parity, 2000000000ull, abort)) {
+    if (!*abort) atomicExch(h.status, int(MV_ERR_TIMEOUT));
     *abort = 1;
-    atomicExch(h.status, int(MV_ERR_TIMEOUT));
+    return false;
   }
+  return true;
+}
+// The same for a whole warp whose lanes must stay together (the tensor-memory loads and stores are warp-wide).
+__device__ __forceinline__ bool warp_wait(const Half& h, uint32_t b, uint32_t parity) {
+  return __all_sync(0xffffffffu, wait_or_flag(h, b, parity));
 }
 
 struct UnitRegs {
@@ -123,18 +136,19 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
     return r;
   };
   int issued = 0;
+  bool ok = true;  // warp-uniform: no wait of this half has run out
   const uint64_t kv_policy = mv::l2_policy_evict_first();  // the KV stream is read once per call
   UnitRegs wu1 = load_unit(u_begin + 1);
   mv::ItemRow ir0 = load_rows(wu, 0), ir1 = load_rows(wu, 32);
   StageRegs win = load_window(wu, 0);
-  for (int u = u_begin; u < u_end; ++u) {
+  for (int u = u_begin; u < u_end && ok; ++u) {
     const int ui = u - u_begin;
     const UnitRegs wu2 = load_unit(u + 2);
     const mv::ItemRow nir0 = load_rows(wu1, 0), nir1 = load_rows(wu1, 32);
     const StageRegs nwin = load_window(wu1, 0);
-    // ---- KV stages, 32 descriptors per window (called with s = 0, 1, 2, ... in order)
+    // ---- KV stages, 32 descriptors per window (called with s = 0, 1, 2, ... in order); false: a wait ran out, nothing issued
     StageRegs nxt;
-    auto issue_stage = [&](int s) {
+    auto issue_stage = [&](int s) -> bool {
       if ((s & 31) == 0) {
         if (s > 0) win = nxt;
         nxt = load_window(wu, s + 32);
@@ -145,8 +159,9 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
       const int n_pages = __shfl_sync(0xffffffffu, win.b.y, src);
       const int b = issued % NSTAGES;
       const uint32_t fb = bar(&meta->full[b]);
-      if (lane == 0) wait_or_flag(h, bar(&meta->empty[b]), ((issued / NSTAGES) & 1) ^ 1);
-      __syncwarp();
+      int go = 1;
+      if (lane == 0) go = wait_or_flag(h, bar(&meta->empty[b]), ((issued / NSTAGES) & 1) ^ 1) ? 1 : 0;
+      if (!__shfl_sync(0xffffffffu, go, 0)) return false;
       if (lane == src) {
         meta->st_tokens[b] = uint32_t(win.b.x);
         meta->st_pages[b] = uint32_t(win.b.y);
@@ -167,6 +182,7 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
         mv::tma_load_2d_hint(dst, kv ? tm_v : tm_k, 0, row, fb, kv_policy);
       }
       ++issued;
+      return true;
     };
     // Between units the first stages go out before the q tile is staged: they do not depend on it, and this keeps the ring
     // full while the producer waits for the previous unit to let go of the q tile (each stage still waits for its own
@@ -175,11 +191,16 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
     // after kernel entry, first stage long there), while the few KB of q requested first cost the stages nothing.
     int s_next = 0;
     if (ui != 0)
-      for (const int pre = min(wu.n_stages, NSTAGES); s_next < pre; ++s_next) issue_stage(s_next);
+      for (const int pre = min(wu.n_stages, NSTAGES); s_next < pre && ok; ++s_next) ok = issue_stage(s_next);
+    if (!ok) break;
     // ---- q-vectors (K-major tile, 128-byte swizzle: what the tensor core expects) and partial-slot ids
     const int n_qv = wu.n_rows * a.G;
-    if (lane == 0) wait_or_flag(h, bar(&meta->q_empty), (ui & 1) ^ 1);
-    __syncwarp();
+    {
+      int go = 1;
+      if (lane == 0) go = wait_or_flag(h, bar(&meta->q_empty), (ui & 1) ^ 1) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, go, 0) != 0;
+    }
+    if (!ok) break;
     for (int x = lane; x < MAXQV; x += 32) {
       const int r = min(x / a.G, MAXQV - 1);
       const int p_lo = __shfl_sync(0xffffffffu, ir0.part, r & 31), p_hi = __shfl_sync(0xffffffffu, ir1.part, r & 31);
@@ -197,10 +218,10 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
       const int r = min(x / a.G, MAXQV - 1);
       const int r_lo = __shfl_sync(0xffffffffu, ir0.row, r & 31), r_hi = __shfl_sync(0xffffffffu, ir1.row, r & 31);
       const int row = r < 32 ? r_lo : r_hi;
-      const bool ok = x < n_qv;
-      const bf16* src = a.q + (ok ? (int64_t(row) * a.Hq + wu.kvh * a.G + x % a.G) * D + c * 8 : 0);
+      const bool okq = x < n_qv;
+      const bf16* src = a.q + (okq ? (int64_t(row) * a.Hq + wu.kvh * a.G + x % a.G) * D + c * 8 : 0);
       const uint32_t dst = h.q_smem + (c >> 3) * (Q_BYTES / 2) + x * 128 + (((c & 7) ^ (x & 7)) << 4);
-      mv::cp_async_16(dst, src, ok ? 16 : 0);
+      mv::cp_async_16(dst, src, okq ? 16 : 0);
     }
     mv::cp_async_mbar_arrive_noinc(bar(&meta->q_full));
     __syncwarp();
@@ -208,8 +229,19 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
       mv::fence_proxy_async();  // the copies above are read by the tensor core (async proxy)
       mv::mbar_arrive(bar(&meta->q_full));
     }
-    for (; s_next < wu.n_stages; ++s_next) issue_stage(s_next);
+    for (; s_next < wu.n_stages && ok; ++s_next) ok = issue_stage(s_next);
     wu = wu1; wu1 = wu2; ir0 = nir0; ir1 = nir1; win = nwin;
+  }
+  if (!ok) {
+    // a wait ran out: nothing more is issued; what is still in flight must land before the CTA may return, since a
+    // bulk copy that completes into the shared memory of a CTA that has left corrupts whoever runs there next
+    mv::cp_async_wait_all();
+    if (lane == 0)
+      for (int k = 1; k <= min(issued, NSTAGES); ++k) {
+        const int e = issued - k;  // the last fills of the ring
+        (void)mv::mbar_wait_bounded(bar(&meta->full[e % NSTAGES]), (e / NSTAGES) & 1, 20000000ull);
+      }
+    __syncwarp();
   }
 }
 
@@ -231,9 +263,12 @@ __device__ __forceinline__ void issuer(const TcArgs& a, const Half& h) {
   constexpr uint32_t idesc_qk = mv::um::idesc_bf16(128, ST, 0, 0), idesc_pv = mv::um::idesc_bf16(128, D, 0, 1);
   int g = 0;  // stages consumed so far (ring position)
   int t = 0;  // stages whose scores were issued so far (S buffer = t & 1)
+  bool ok = true;  // false once a wait of this half ran out: nothing more is issued (a lane that saw the barrier complete
+                   // at the last moment may run on alone for a step; it issues nothing the others would not have)
   auto scores = [&](int stage_g) {  // S = Q K^T of ring entry stage_g into buffer t & 1
     const int sb = stage_g % NSTAGES;
-    wait_or_flag(h, bar(&meta->full[sb]), (stage_g / NSTAGES) & 1);
+    ok = ok && wait_or_flag(h, bar(&meta->full[sb]), (stage_g / NSTAGES) & 1);
+    if (!ok) return;
     mv::um::fence_after();
     const uint64_t k_desc = mv::um::smem_desc(h.stage_smem + sb * STAGE_BYTES, 16, 1024);
     const uint32_t s_t = h.tmem + (t & 1) * 64;
@@ -248,23 +283,27 @@ __device__ __forceinline__ void issuer(const TcArgs& a, const Half& h) {
     }
     ++t;
   };
-  for (int u = u_begin; u < u_end; ++u) {
+  for (int u = u_begin; u < u_end && ok; ++u) {
     const int ui = u - u_begin;
-    wait_or_flag(h, bar(&meta->q_full), ui & 1);
+    ok = wait_or_flag(h, bar(&meta->q_full), ui & 1);
+    if (!ok) break;
     mv::fence_proxy_async();  // the q tile was written with ordinary asynchronous copies; the tensor core reads it
     const int n = meta->n_stages;
     const int t0 = t;  // stage s of this unit is score tile t0 + s: S / P buffer (t0 + s) & 1
     scores(g);
+    if (!ok) break;
     if (n == 1 && lead) mv::um::commit(bar(&meta->q_empty));  // the unit's last scores are queued: q tile free once they ran
     for (int s = 0; s < n; ++s) {
       if (s + 1 < n) {
         scores(g + 1);
+        if (!ok) break;
         if (s + 2 == n && lead) mv::um::commit(bar(&meta->q_empty));
       }
-      if (s == 0 && ui > 0) wait_or_flag(h, bar(&meta->o_free), (ui - 1) & 1);  // the previous unit's O has been read
+      if (s == 0 && ui > 0) ok = wait_or_flag(h, bar(&meta->o_free), (ui - 1) & 1);  // the previous unit's O has been read
       const int sb = g % NSTAGES, T = t0 + s, pb = T & 1;
       const uint32_t n_pages = meta->st_pages[sb];
-      wait_or_flag(h, bar(&meta->p_full[pb]), (T >> 1) & 1);
+      ok = ok && wait_or_flag(h, bar(&meta->p_full[pb]), (T >> 1) & 1);
+      if (!ok) break;
       mv::um::fence_after();
       const uint64_t v_desc = mv::um::smem_desc(h.stage_smem + sb * STAGE_BYTES + KV_BYTES, KV_BYTES / 2, 1024);
       const uint32_t o_t = h.tmem + 128, p_t = h.tmem + pb * 64;
@@ -279,6 +318,12 @@ __device__ __forceinline__ void issuer(const TcArgs& a, const Half& h) {
       }
       ++g;
     }
+  }
+  __syncwarp();
+  if (*reinterpret_cast<volatile int*>(&meta->abort)) {
+    // products may still be in flight: they must have completed before the CTA frees its tensor memory
+    if (lead) mv::um::commit(bar(&meta->drained));
+    (void)mv::mbar_wait_bounded(bar(&meta->drained), 0, 20000000ull);
   }
 }
 
@@ -300,9 +345,11 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
     u_end = y.z;
   }
   int g = 0;  // stages consumed so far (ring position, score tile index and product index all advance together)
-  for (int u = u_begin; u < u_end; ++u) {
+  bool ok = true;    // warp-uniform: false once a wait of this half ran out
+  for (int u = u_begin; u < u_end && ok; ++u) {
     const int ui = u - u_begin;
-    wait_or_flag(h, bar(&meta->q_full), ui & 1);
+    ok = warp_wait(h, bar(&meta->q_full), ui & 1);
+    if (!ok) break;
     const int n = meta->n_stages, n_qv = meta->n_qv;
     const int pv = (r >= 0 && r < MAXQV) ? meta->pv[r] : -1;
     mv::mbar_arrive(bar(&meta->q_empty));  // header and slot ids are in registers
@@ -316,9 +363,11 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
     float m = -INFINITY, l = 0.f;
     for (int s = 0; s < n; ++s, ++g) {
       const int sb = g % NSTAGES, pb = g & 1;
-      wait_or_flag(h, bar(&meta->full[sb]), (g / NSTAGES) & 1);  // the stage's token counts and masks are visible
+      ok = warp_wait(h, bar(&meta->full[sb]), (g / NSTAGES) & 1);  // the stage's token counts and masks are visible
+      if (!ok) break;
       const uint32_t tok4 = meta->st_tokens[sb], n_pages = meta->st_pages[sb];
-      wait_or_flag(h, bar(&meta->s_full[pb]), (g >> 1) & 1);
+      ok = warp_wait(h, bar(&meta->s_full[pb]), (g >> 1) & 1);
+      if (!ok) break;
       mv::um::fence_after();
       const uint32_t s_t = lane_base + pb * 64;
       uint32_t sc[ST];
@@ -356,7 +405,8 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
         mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
       }
       if (s > 0) {  // O holds stages 0 .. s-1 of the unit once the previous product is done
-        wait_or_flag(h, bar(&meta->o_done), (g - 1) & 1);
+        ok = warp_wait(h, bar(&meta->o_done), (g - 1) & 1);
+        if (!ok) break;
         mv::um::fence_after();
       }
       if (warp_active) {
@@ -364,14 +414,14 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
         const bool move = mx > m + RESCALE_THRESHOLD || (m == -INFINITY && mx > -INFINITY);
         if (s > 0 && __any_sync(0xffffffffu, move)) {
           const float f = (move && m != -INFINITY) ? mv::fast_exp2(m - mx) : 1.f;
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            mv::um::ld32(o_t + c * 32, o);
+#pragma unroll 1
+          for (int c = 0; c < D / 16; ++c) {  // sixteen columns at a time: the scores of the stage are live in registers
+            uint32_t o[16];
+            mv::um::ld16(o_t + c * 16, o);
             mv::um::wait_ld();
 #pragma unroll
-            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * f);
-            mv::um::st32(o_t + c * 32, o);
+            for (int k = 0; k < 16; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * f);
+            mv::um::st16(o_t + c * 16, o);
           }
           l *= f;
         }
@@ -412,8 +462,10 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
       mv::um::fence_before();
       mv::mbar_arrive(bar(&meta->p_full[pb]));
     }
-    // ---- the unit's partial: (max, sum, unnormalised O) of this q-vector
-    wait_or_flag(h, bar(&meta->o_done), (g - 1) & 1);
+    if (!ok) break;
+    // ---- the unit's result: (max, sum, unnormalised O) of this q-vector
+    ok = warp_wait(h, bar(&meta->o_done), (g - 1) & 1);
+    if (!ok) break;
     mv::um::fence_after();
     if (warp_active) {
       float* po = a.part_o + int64_t(pv >= 0 ? pv : 0) * D;
@@ -461,6 +513,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) decode_tc_kernel(const TcArgs a, 
     }
     mv::mbar_init(bar(&meta->o_done), 1);    // one tcgen05.commit
     mv::mbar_init(bar(&meta->o_free), 128);  // the softmax group
+    mv::mbar_init(bar(&meta->drained), 1);   // one tcgen05.commit
     mv::mbar_fence_init();
     mv::fence_proxy_async();
   }
@@ -498,10 +551,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) decode_tc_kernel(const TcArgs a, 
   if (warp == 0) mv::um::tmem_dealloc(tmem_slot, 512);
 }
 
-struct TcMapCache {
-  const void* k = nullptr;
-  const void* v = nullptr;
-  int64_t rows = 0;
+struct TcMaps {
   CUtensorMap tm_k, tm_v;
 };
 
@@ -512,27 +562,18 @@ namespace mv {
 // merge kernel afterwards).  Partials land in `ws` exactly as the mma.sync kernel leaves them.
 mv_status decode_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* kp, const void* vp, void* ws,
                     cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
-      (void)cudaGetLastError();
+  static std::atomic<uint64_t> opted_in{0};  // per device
+  if (!mv::opt_in_smem(decode_tc_kernel, SMEM_BYTES, opted_in)) return MV_ERR_CUDA;
+  static thread_local mv::KeyedCache<TcMaps, 4> cache;  // the pools rarely change between calls
+  const int64_t rows = g->num_pages * g->n_kv_heads * 2 * 16;  // 128-byte rows of a pool
+  const mv::TmapKey key{mv::current_device(), kp, vp, nullptr, rows, 0};
+  TcMaps* hit = cache.find(key);
+  if (!hit) {
+    hit = cache.claim(key);
+    if (!mv::make_tmap_bf16_2d(&hit->tm_k, kp, uint64_t(rows), 64, 16) || !mv::make_tmap_bf16_2d(&hit->tm_v, vp, uint64_t(rows), 64, 16)) {
+      cache.drop();
       return MV_ERR_CUDA;
     }
-    attr_set = true;
-  }
-  static thread_local TcMapCache tc[4];
-  static thread_local int tc_next = 0;
-  const int64_t rows = g->num_pages * g->n_kv_heads * 2 * 16;  // 128-byte rows of a pool
-  TcMapCache* hit = nullptr;
-  for (auto& c : tc)
-    if (c.k == kp && c.v == vp && c.rows == rows) hit = &c;
-  if (!hit) {
-    hit = &tc[tc_next];
-    tc_next = (tc_next + 1) % 4;
-    hit->k = nullptr;
-    if (!mv::make_tmap_bf16_2d(&hit->tm_k, kp, uint64_t(rows), 64, 16) || !mv::make_tmap_bf16_2d(&hit->tm_v, vp, uint64_t(rows), 64, 16))
-      return MV_ERR_CUDA;
-    hit->k = kp; hit->v = vp; hit->rows = rows;
   }
   const int G = g->n_q_heads / g->n_kv_heads;
   const size_t vecs = size_t(P->stats.n_partials) * size_t(G);

@@ -212,14 +212,8 @@ template <int D>
 mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out,
                  cudaStream_t st) {
   constexpr int SMEM = BQ * D * 2 + 2 * NBUF * BK * D * 2;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(prefill_bf16_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess) {
-      (void)cudaGetLastError();
-      return MV_ERR_CUDA;
-    }
-    attr_set = true;
-  }
+  static std::atomic<uint64_t> opted_in{0};  // per device
+  if (!mv::opt_in_smem(prefill_bf16_kernel<D>, SMEM, opted_in)) return MV_ERR_CUDA;
   dim3 grid(int(P->stats.n_q_tiles) * 2, g->n_q_heads);
   prefill_bf16_kernel<D><<<grid, NTHREADS, SMEM, st>>>(
       static_cast<const bf16*>(q), static_cast<const bf16*>(k), static_cast<const bf16*>(v), static_cast<bf16*>(out),

@@ -19,6 +19,7 @@
 // column block, the pool layout of the decode kernels), keys are counted inside the node, and the causal range is the
 // tile's own node with the first query sitting at key index causal_base.
 #include "common.cuh"
+#include "tmap_cache.h"
 #include "umma.cuh"
 
 namespace {
@@ -37,7 +38,7 @@ constexpr int SMEM_BYTES = OFF_BAR + 256;
 constexpr float RESCALE_THRESHOLD = 8.f;  // log2 units: P stays below 2^8, well inside bf16 and fp32 range
 
 struct Bars {  // shared-memory addresses
-  uint32_t q_full, kv_full, kv_empty, s_full, p_full, o_done;
+  uint32_t q_full, kv_full, kv_empty, s_full, p_full, o_done, drained;
 };
 
 struct PrefillArgs {
@@ -81,17 +82,36 @@ struct TileIter {
   }
 };
 
-struct Waiter {  // bounded waits: after one ran out every later wait returns at once, so the CTA still ends
+// Bounded waits.  wait() is false once a wait of this CTA has run out (this one or an earlier one, of any role): the
+// caller then issues nothing further, leaves its loops, and the producer and the issuer wait (again bounded) for what
+// they still have in flight before the CTA frees its tensor memory and returns.
+struct Waiter {
   volatile int* abort;
   int32_t* status;
-  __device__ __forceinline__ void wait(uint32_t bar, uint32_t parity) const {
-    if (*abort) return;
-    if (!mv::mbar_wait_bounded(bar, parity)) {
+  __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
+    if (*abort) return false;
+    if (!mv::mbar_wait_bounded(bar, parity, 2000000000ull, abort)) {
+      if (!*abort) atomicExch(status, int(MV_ERR_TIMEOUT));
       *abort = 1;
-      atomicExch(status, int(MV_ERR_TIMEOUT));
+      return false;
     }
+    return true;
   }
+  // for a whole warp whose lanes must stay together (tensor-memory loads and stores are warp-wide)
+  __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) const { return __all_sync(0xffffffffu, wait(bar, parity)); }
+  __device__ __forceinline__ bool aborted() const { return *abort != 0; }
 };
+
+// After a wait ran out: the last fills of the ring (entries e - RING .. e - 1) and the Q tiles may still be in flight;
+// a bulk copy that completes into the shared memory of a CTA that has left corrupts whoever runs there next.
+__device__ __forceinline__ void drain_producer(const Bars& br, int e, int lane) {
+  if (lane == 0) {
+    (void)mv::mbar_wait_bounded(br.q_full, 0, 20000000ull);
+    for (int k = 1; k <= min(e, RING); ++k)
+      (void)mv::mbar_wait_bounded(br.kv_full + 8 * ((e - k) % RING), ((e - k) / RING) & 1, 20000000ull);
+  }
+  __syncwarp();
+}
 
 template <bool PAGED>
 __device__ __forceinline__ void producer_warp(const mv::QTile& qt, const PrefillArgs& a, int h0, int kvh, uint32_t smem_base,
@@ -124,11 +144,15 @@ __device__ __forceinline__ void producer_warp(const mv::QTile& qt, const Prefill
       for (int kv = 0; kv < 2; ++kv, ++e) {
         const int slot = e % RING;
         const uint32_t bar = br.kv_full + 8 * slot;
+        int go = 1;
         if (lane == 0) {
-          w.wait(br.kv_empty + 8 * slot, ((e / RING) & 1) ^ 1);
-          mv::mbar_arrive_expect_tx(bar, uint32_t(n_pg) * 4096u);
+          go = w.wait(br.kv_empty + 8 * slot, ((e / RING) & 1) ^ 1) ? 1 : 0;
+          if (go) mv::mbar_arrive_expect_tx(bar, uint32_t(n_pg) * 4096u);
         }
-        __syncwarp();
+        if (!__shfl_sync(0xffffffffu, go, 0)) {
+          drain_producer(br, e, lane);
+          return;
+        }
         if (page >= 0)
           mv::tma_load_2d(smem_base + OFF_RING + slot * TILE_BYTES + h * (TILE_BYTES / 2) + p * 2048, kv ? tm_v : tm_k, 0,
                           ((page * a.Hkv + kvh) * 2 + h) * 16, bar);
@@ -140,7 +164,10 @@ __device__ __forceinline__ void producer_warp(const mv::QTile& qt, const Prefill
   while (it.next(start, n, c)) {
     for (int kv = 0; kv < 2; ++kv, ++e) {
       const int slot = e % RING;
-      w.wait(br.kv_empty + 8 * slot, ((e / RING) & 1) ^ 1);
+      if (!w.wait(br.kv_empty + 8 * slot, ((e / RING) & 1) ^ 1)) {
+        drain_producer(br, e, 0);
+        return;
+      }
       const uint32_t bar = br.kv_full + 8 * slot;
       mv::mbar_arrive_expect_tx(bar, TILE_BYTES);
       const uint32_t dst = smem_base + OFF_RING + slot * TILE_BYTES;
@@ -184,11 +211,18 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
   const uint32_t s0 = tmem, s1 = tmem + 128, o0 = tmem + 256, o1 = tmem + 384;
   auto k_desc = [&](int e) { return mv::um::smem_desc(smem_base + OFF_RING + (e % RING) * TILE_BYTES, 16, 1024); };
   auto v_desc = [&](int e) { return mv::um::smem_desc(smem_base + OFF_RING + (e % RING) * TILE_BYTES, TILE_BYTES / 2, 1024); };
-  auto wait_full = [&](int e) { w.wait(br.kv_full + 8 * (e % RING), (e / RING) & 1); };
+  bool ok = true;  // false once a wait ran out: nothing more is issued
+  auto wait_full = [&](int e) { ok = ok && w.wait(br.kv_full + 8 * (e % RING), (e / RING) & 1); };
+  auto drain = [&]() {  // products may still be in flight: they must have completed before the tensor memory is freed
+    __syncwarp();
+    if (lead) mv::um::commit(br.drained);
+    (void)mv::mbar_wait_bounded(br.drained, 0, 20000000ull);
+  };
   auto release = [&](int e) { if (lead) mv::um::commit(br.kv_empty + 8 * (e % RING)); };
   auto cols = [](int n) { return ((n + 15) >> 4) << 4; };  // score columns computed; the softmax groups mask the rest
-  w.wait(br.q_full, 0);
+  ok = w.wait(br.q_full, 0);
   wait_full(0);
+  if (!ok) return drain();
   mv::um::fence_after();
   if (lead) {
     issue_qk(s0, q0, k_desc(0), cols(n_cur));
@@ -201,6 +235,7 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
     const int ev = 2 * j + 1, ek = 2 * j + 2;  // ring entries of V_j and K_{j+1}
     const int k_steps = (n_cur + 15) >> 4;
     wait_full(ev);
+    if (!ok) break;
     if (PAGED && (n_cur & 15) && lead) {
       // the last page of a node is not full: its rows past the last key hold whatever the pool held; V must be zero
       // where P is zero, or 0 * NaN would poison O
@@ -214,7 +249,8 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
     // the next K tile is waited for here, while P of head 0 is still being computed, not between the two products below:
     // that wait sat on head 0's chain (softmax -> P V -> next Q K^T -> softmax) in every step
     if (more) wait_full(ek);
-    w.wait(br.p_full, j & 1);
+    ok = ok && w.wait(br.p_full, j & 1);
+    if (!ok) break;
     mv::um::fence_after();
     if (lead) {
       issue_pv(o0, s0, v_desc(ev), j > 0, k_steps);
@@ -224,7 +260,8 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
         mv::um::commit(br.s_full);
       }
     }
-    w.wait(br.p_full + 8, j & 1);
+    ok = w.wait(br.p_full + 8, j & 1);
+    if (!ok) break;
     mv::um::fence_after();
     if (lead) {
       issue_pv(o1, s1, v_desc(ev), j > 0, k_steps);
@@ -240,6 +277,7 @@ __device__ __forceinline__ void mma_warp(const mv::QTile& qt, const PrefillArgs&
     n_cur = n_next;
     more = it.next(start, n_next, c);
   }
+  if (w.aborted()) drain();
 }
 
 // One softmax group = 128 threads = the 128 query rows of head `i` (0 or 1) of the CTA.
@@ -256,7 +294,7 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
   float m = -INFINITY, l = 0.f;  // running maximum (log2 units) and sum of this row
   int start, n, causal, j = 0;
   while (it.next(start, n, causal)) {
-    w.wait(s_full, j & 1);
+    if (!w.warp_wait(s_full, j & 1)) return;
     mv::um::fence_after();
     // all 128 columns are read: on a ragged tile the issuer computed only the leading ones, the rest holds an
     // older tile's scores and is masked below
@@ -284,7 +322,7 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
     const bool move = mx > m + RESCALE_THRESHOLD || (m == -INFINITY && mx > -INFINITY);
     if (j > 0 && __any_sync(0xffffffffu, move)) {
       const float f = (move && m != -INFINITY) ? mv::fast_exp2(m - mx) : 1.f;
-      w.wait(o_done, (j - 1) & 1);  // O_i holds tiles 0 .. j-1 and no product is writing it
+      if (!w.warp_wait(o_done, (j - 1) & 1)) return;  // O_i holds tiles 0 .. j-1 and no product is writing it
       mv::um::fence_after();
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
@@ -323,7 +361,7 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
     ++j;
   }
   if (j == 0) return;
-  w.wait(o_done, (j - 1) & 1);
+  if (!w.warp_wait(o_done, (j - 1) & 1)) return;
   mv::um::fence_after();
   const float inv = 1.f / l;
   bf16* dst = a.out + (int64_t(qi) * a.Hq + head) * D;
@@ -363,6 +401,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) prefill_tc_kernel(const PrefillAr
   br.s_full = mv::smem_u32(&bars[1 + 2 * RING]);
   br.p_full = mv::smem_u32(&bars[3 + 2 * RING]);
   br.o_done = mv::smem_u32(&bars[5 + 2 * RING]);
+  br.drained = mv::smem_u32(&bars[7 + 2 * RING]);
   if ((smem_base & 1023u) != 0) {  // the swizzle pattern is anchored at 1024-byte boundaries
     if (tid == 0) atomicExch(a.status, int(MV_ERR_UNSUPPORTED));
     return;
@@ -379,6 +418,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) prefill_tc_kernel(const PrefillAr
       mv::mbar_init(br.p_full + 8 * i, 128);  // every thread of the softmax group
       mv::mbar_init(br.o_done + 8 * i, 1);    // one tcgen05.commit
     }
+    mv::mbar_init(br.drained, 1);             // one tcgen05.commit, only after a wait ran out
     mv::mbar_fence_init();
     mv::fence_proxy_async();
   }
@@ -411,10 +451,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) prefill_tc_kernel(const PrefillAr
   if (warp == 2) mv::um::tmem_dealloc(tmem, 512);
 }
 
-struct TcMaps {  // the last problem's tensor maps (pointers and token count rarely change between calls)
-  const void *q = nullptr, *k = nullptr, *v = nullptr;
-  int64_t T = 0, pool_rows = 0;
-  int Hq = 0, Hkv = 0;
+struct TcMaps {  // the tensor maps of one problem (pointers and token count rarely change between calls)
   CUtensorMap tm_q, tm_k, tm_v;
 };
 
@@ -423,24 +460,22 @@ struct TcMaps {  // the last problem's tensor maps (pointers and token count rar
 namespace mv {
 // Tensor-core prefill for head_dim 128 and an even group size; the caller has validated the arguments.
 mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
-      (void)cudaGetLastError();
+  static std::atomic<uint64_t> opted_in{0};  // per device
+  if (!mv::opt_in_smem(prefill_tc_kernel<false>, SMEM_BYTES, opted_in)) return MV_ERR_CUDA;
+  const int64_t T = P->stats.n_new_tokens;
+  static thread_local mv::KeyedCache<TcMaps, 2> cache;
+  const mv::TmapKey key{mv::current_device(), q, k, v, T, (int64_t(g->n_q_heads) << 32) | int64_t(g->n_kv_heads)};
+  TcMaps* tcp = cache.find(key);
+  if (!tcp) {
+    tcp = cache.claim(key);
+    if (!mv::make_tmap_bf16_2d(&tcp->tm_q, q, uint64_t(T), uint64_t(g->n_q_heads) * D, BQ) ||
+        !mv::make_tmap_bf16_2d(&tcp->tm_k, k, uint64_t(T), uint64_t(g->n_kv_heads) * D, BK) ||
+        !mv::make_tmap_bf16_2d(&tcp->tm_v, v, uint64_t(T), uint64_t(g->n_kv_heads) * D, BK)) {
+      cache.drop();
       return MV_ERR_CUDA;
     }
-    attr_set = true;
   }
-  const int64_t T = P->stats.n_new_tokens;
-  static thread_local TcMaps tc;
-  if (!(tc.q == q && tc.k == k && tc.v == v && tc.T == T && tc.Hq == g->n_q_heads && tc.Hkv == g->n_kv_heads)) {
-    tc.q = nullptr;
-    if (!mv::make_tmap_bf16_2d(&tc.tm_q, q, uint64_t(T), uint64_t(g->n_q_heads) * D, BQ) ||
-        !mv::make_tmap_bf16_2d(&tc.tm_k, k, uint64_t(T), uint64_t(g->n_kv_heads) * D, BK) ||
-        !mv::make_tmap_bf16_2d(&tc.tm_v, v, uint64_t(T), uint64_t(g->n_kv_heads) * D, BK))
-      return MV_ERR_CUDA;
-    tc.q = q; tc.k = k; tc.v = v; tc.T = T; tc.Hq = g->n_q_heads; tc.Hkv = g->n_kv_heads;
-  }
+  const TcMaps& tc = *tcp;
   PrefillArgs a;
   a.q_tiles = mv::table<mv::QTile>(P, P->layout.q_tiles);
   a.ranges = mv::table<mv::KvRange>(P, P->layout.kv_ranges);
@@ -463,26 +498,24 @@ mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, con
 // the normalised output directly: no partials, no merge.  The caller has validated the arguments.
 mv_status append_tc(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_pages, const void* v_pages, void* out,
                     cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
-      (void)cudaGetLastError();
-      return MV_ERR_CUDA;
-    }
-    attr_set = true;
-  }
+  static std::atomic<uint64_t> opted_in{0};  // per device
+  if (!mv::opt_in_smem(prefill_tc_kernel<true>, SMEM_BYTES, opted_in)) return MV_ERR_CUDA;
   const int64_t T = P->stats.n_new_tokens;
   const int64_t pool_rows = g->num_pages * g->n_kv_heads * 2 * 16;  // 128-byte rows of a pool
-  static thread_local TcMaps tc;
-  if (!(tc.q == q_rot && tc.k == k_pages && tc.v == v_pages && tc.T == T && tc.Hq == g->n_q_heads && tc.Hkv == g->n_kv_heads &&
-        tc.pool_rows == pool_rows)) {
-    tc.q = nullptr;
-    if (!mv::make_tmap_bf16_2d(&tc.tm_q, q_rot, uint64_t(T), uint64_t(g->n_q_heads) * D, BQ) ||
-        !mv::make_tmap_bf16_2d(&tc.tm_k, k_pages, uint64_t(pool_rows), 64, 16) ||
-        !mv::make_tmap_bf16_2d(&tc.tm_v, v_pages, uint64_t(pool_rows), 64, 16))
+  static thread_local mv::KeyedCache<TcMaps, 2> cache;
+  const mv::TmapKey key{mv::current_device(), q_rot, k_pages, v_pages, T,
+                        (pool_rows << 16) ^ (int64_t(g->n_q_heads) << 8) ^ int64_t(g->n_kv_heads)};
+  TcMaps* tcp = cache.find(key);
+  if (!tcp) {
+    tcp = cache.claim(key);
+    if (!mv::make_tmap_bf16_2d(&tcp->tm_q, q_rot, uint64_t(T), uint64_t(g->n_q_heads) * D, BQ) ||
+        !mv::make_tmap_bf16_2d(&tcp->tm_k, k_pages, uint64_t(pool_rows), 64, 16) ||
+        !mv::make_tmap_bf16_2d(&tcp->tm_v, v_pages, uint64_t(pool_rows), 64, 16)) {
+      cache.drop();
       return MV_ERR_CUDA;
-    tc.q = q_rot; tc.k = k_pages; tc.v = v_pages; tc.T = T; tc.Hq = g->n_q_heads; tc.Hkv = g->n_kv_heads; tc.pool_rows = pool_rows;
+    }
   }
+  const TcMaps& tc = *tcp;
   PrefillArgs a;
   a.q_tiles = mv::table<mv::QTile>(P, P->layout.q_tiles);
   a.ranges = mv::table<mv::KvRange>(P, P->layout.kv_ranges);

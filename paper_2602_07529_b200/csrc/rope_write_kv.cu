@@ -3,12 +3,12 @@
 // For every new token t: rotate q and k by the position index the planner assigned (Sec. 4.2: positions
 // continue from the fork / join point), store k and v at the token's pool slot and emit the rotated q.
 // P(i) of Eq. 2 is taken to be the rotary embedding with half-split pairing: element i pairs with
-// i + d/2 and is rotated by pos * base^(-2i/d).  The angle, its cosine and sine are evaluated in double
-// precision and rounded to float (positions reach ~2e4, where a float angle alone would already be off
-// by ~1e-3 rad); the rotation is float.
+// i + d/2 and is rotated by pos * base^(-2i/d).  The angle and its reduction to the first octant are evaluated
+// in double precision (positions reach ~2e4, where a float angle alone would already be off by ~1e-3 rad);
+// cosine and sine of the reduced angle and the rotation are float.
 //
-// HBM-bound elementwise kernel: one CTA per token, 16-byte vector loads and stores, the cos/sin row of
-// the token is computed once into shared memory and reused by all heads.
+// HBM-bound elementwise kernel: one or four tokens per CTA, 16-byte vector loads and stores, the cos/sin
+// rows of the CTA's tokens are computed once into shared memory and reused by all heads.
 #include "common.cuh"
 
 namespace {
@@ -48,100 +48,141 @@ struct Vec16<__nv_bfloat16> {
   }
 };
 
-template <typename T, int D>
-__global__ void __launch_bounds__(128) rope_write_kv_kernel(const T* q, const T* k,
-                                                            const T* v, T* q_rot,
-                                                            T* k_rot, T* k_pages,
-                                                            T* v_pages,
-                                                            const int32_t* pos_id,
-                                                            const int64_t* slot, int n_tok, int Hq,
-                                                            int Hkv, double neg_log2_base_2_over_d) {
+// theta_i = base^(-2i/d) for i < d/2, evaluated once per launch on the host in double precision
+struct ThetaTable {
+  double theta[64];
+};
+
+// cos and sin of pos * theta.  The angle and its reduction to [-pi/4, pi/4] (two-term Cody-Waite with a 53-bit and a
+// residual piece of pi/2; pos * theta stays below 2^25, so k * PIO2_HI is exact to well under 1e-12) are double
+// precision; the reduced angle is rounded to float and its cosine and sine come from the accurate float routine
+// (no fast-math intrinsics), so both agree with the double-precision values to within two units in the last place
+// of a float.  Six double-precision instructions per (token, i) instead of a double-precision sincos: with the
+// latter the arithmetic, not HBM, bounded the kernel at prefill sizes.
+__device__ __forceinline__ void rope_cos_sin(int pos, double theta, float& c, float& s) {
+  constexpr double TWO_OVER_PI = 0.63661977236758134308;
+  constexpr double PIO2_HI = 1.57079632679489655800e+00;  // pi/2 rounded to double
+  constexpr double PIO2_LO = 6.12323399573676603587e-17;  // pi/2 - PIO2_HI
+  const double a = double(pos) * theta;
+  const double kf = rint(a * TWO_OVER_PI);
+  double r = fma(-kf, PIO2_HI, a);
+  r = fma(-kf, PIO2_LO, r);
+  float sr, cr;
+  sincosf(float(r), &sr, &cr);
+  const int k = int(kf) & 3;  // quadrant: angle = r + k * pi/2
+  const float ss = (k & 1) ? cr : sr, cc = (k & 1) ? sr : cr;
+  s = (k & 2) ? -ss : ss;
+  c = ((k + 1) & 2) ? -cc : cc;
+}
+
+// TPC tokens per CTA.  Phase 1: the CTA's (token, i) pairs get their cos / sin, one pair per thread, while the first
+// loads of phase 2 are already in flight; phase 2: 16-byte units of q, k (rotated) and v (copied) stream through.
+template <typename T, int D, int TPC>
+__global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                                                            T* __restrict__ q_rot, T* __restrict__ k_rot, T* __restrict__ k_pages,
+                                                            T* __restrict__ v_pages, const int32_t* __restrict__ pos_id,
+                                                            const int64_t* __restrict__ slot, int n_tok, int Hq, int Hkv,
+                                                            const __grid_constant__ ThetaTable tt) {
   constexpr int HALF = D / 2;
   constexpr int N = Vec16<T>::N;
   constexpr int CH = HALF / N;  // 16-byte chunks per half head
-  __shared__ float cs[HALF], sn[HALF];
-  const int t = blockIdx.x;
+  constexpr int VCH = D / N;    // 16-byte chunks per head
+  __shared__ float cs[TPC][HALF], sn[TPC][HALF];
+  __shared__ int64_t s_slot[TPC];
+  const int t0 = blockIdx.x * TPC;
   // a kernel launched behind this one with programmatic stream serialisation (the decode attention kernel) may become
   // resident and run its set-up now; it waits for this grid's completion before it reads what is written here
   mv::grid_dependency_launch_dependents();
-  if (t >= n_tok) return;
-  const int pos = pos_id[t];
-  const int64_t sl = slot[t];
-  for (int i = threadIdx.x; i < HALF; i += blockDim.x) {
-    // theta_i = base^(-2i/d) = 2^(-(2i/d) * log2(base)), in double
-    const double theta = exp2(double(i) * neg_log2_base_2_over_d);
-    double s, c;
-    sincos(double(pos) * theta, &s, &c);
-    cs[i] = float(c);
-    sn[i] = float(s);
+  const int n_here = min(TPC, n_tok - t0);
+  if (n_here <= 0) return;
+  for (int x = threadIdx.x; x < n_here * HALF; x += blockDim.x) {
+    const int tl = x / HALF, i = x % HALF;
+    float c, s;
+    rope_cos_sin(__ldg(pos_id + t0 + tl), tt.theta[i], c, s);
+    cs[tl][i] = c;
+    sn[tl][i] = s;
+    if (i == 0) s_slot[tl] = __ldg(slot + t0 + tl);
   }
   __syncthreads();
-  const int64_t page = sl >> 4, off = sl & 15;
   const int n_q_units = q ? Hq * CH : 0;
   const int n_k_units = Hkv * CH;
-  // rotated q and k
-  for (int u = threadIdx.x; u < n_q_units + n_k_units; u += blockDim.x) {
+  const int n_v_units = v_pages ? Hkv * VCH : 0;
+  const int per_tok = n_q_units + n_k_units + n_v_units;
+  for (int x = threadIdx.x; x < n_here * per_tok; x += blockDim.x) {
+    const int tl = x / per_tok, u = x % per_tok;
+    const int64_t t = t0 + tl;
+    const int64_t sl = s_slot[tl];
+    const int64_t page = sl >> 4, off = sl & 15;
+    if (u >= n_q_units + n_k_units) {  // v is stored unrotated
+      const int uu = u - n_q_units - n_k_units;
+      const int h = uu / VCH, c = uu % VCH;
+      const uint4 val = *reinterpret_cast<const uint4*>(v + (t * Hkv + h) * D + c * N);
+      const int e = c * N;
+      *reinterpret_cast<uint4*>(v_pages + (page * Hkv + h) * (16 * D) + (e >> 6) * 1024 + off * 64 + (e & 63)) = val;
+      continue;
+    }
     const bool is_q = u < n_q_units;
     const int uu = is_q ? u : u - n_q_units;
     const int h = uu / CH, c = uu % CH;
-    const T* src = is_q ? q + (int64_t(t) * Hq + h) * D : k + (int64_t(t) * Hkv + h) * D;
-    // pool element (page, head, token, c) lives in 64-element column block c / 64 of the (page, head) block
-    T* dst = is_q ? q_rot + (int64_t(t) * Hq + h) * D : k_pages + (page * Hkv + h) * (16 * D) + off * 64;
-    T* dst2 = is_q ? nullptr : k_rot + (int64_t(t) * Hkv + h) * D;
-    const bool w1 = is_q || k_pages != nullptr, w2 = !is_q && k_rot != nullptr;
+    const T* src = is_q ? q + (t * Hq + h) * D : k + (t * Hkv + h) * D;
     float lo[N], hi[N], olo[N], ohi[N];
     Vec16<T>::load(src + c * N, lo);
     Vec16<T>::load(src + HALF + c * N, hi);
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-      const float cc = cs[c * N + i], ss = sn[c * N + i];
+      const float cc = cs[tl][c * N + i], ss = sn[tl][c * N + i];
       olo[i] = lo[i] * cc - hi[i] * ss;
       ohi[i] = hi[i] * cc + lo[i] * ss;
     }
-    if (w1) {
-      if (is_q) {
-        Vec16<T>::store(dst + c * N, olo);
-        Vec16<T>::store(dst + HALF + c * N, ohi);
-      } else {
-        const int e0 = c * N, e1 = HALF + c * N;  // element indices inside the head vector
-        Vec16<T>::store(dst + (e0 >> 6) * 1024 + (e0 & 63), olo);
-        Vec16<T>::store(dst + (e1 >> 6) * 1024 + (e1 & 63), ohi);
-      }
+    if (is_q) {
+      T* dst = q_rot + (t * Hq + h) * D;
+      Vec16<T>::store(dst + c * N, olo);
+      Vec16<T>::store(dst + HALF + c * N, ohi);
+      continue;
     }
-    if (w2) {
+    if (k_pages != nullptr) {
+      // pool element (page, head, token, e) lives in 64-element column block e / 64 of the (page, head) block
+      T* dst = k_pages + (page * Hkv + h) * (16 * D) + off * 64;
+      const int e0 = c * N, e1 = HALF + c * N;
+      Vec16<T>::store(dst + (e0 >> 6) * 1024 + (e0 & 63), olo);
+      Vec16<T>::store(dst + (e1 >> 6) * 1024 + (e1 & 63), ohi);
+    }
+    if (k_rot != nullptr) {
+      T* dst2 = k_rot + (t * Hkv + h) * D;
       Vec16<T>::store(dst2 + c * N, olo);
       Vec16<T>::store(dst2 + HALF + c * N, ohi);
     }
   }
-  if (v_pages == nullptr) return;
-  // v is stored unrotated
-  constexpr int VCH = D / N;
-  for (int u = threadIdx.x; u < Hkv * VCH; u += blockDim.x) {
-    const int h = u / VCH, c = u % VCH;
-    const uint4 val = *reinterpret_cast<const uint4*>(v + (int64_t(t) * Hkv + h) * D + c * N);
-    const int e = c * N;
-    *reinterpret_cast<uint4*>(v_pages + (page * Hkv + h) * (16 * D) + (e >> 6) * 1024 + off * 64 + (e & 63)) = val;
-  }
+}
+
+template <typename T, int D>
+mv_status launch_d(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* q_rot,
+                   void* k_rot, void* k_pages, void* v_pages, cudaStream_t st) {
+  const int n = int(P->stats.n_new_tokens);
+  const int32_t* pos = mv::table<int32_t>(P, P->layout.pos_id);
+  const int64_t* slot = mv::table<int64_t>(P, P->layout.slot);
+  ThetaTable tt{};
+  const double c = -2.0 * log2(g->rope_base) / double(D);
+  for (int i = 0; i < D / 2; ++i) tt.theta[i] = exp2(double(i) * c);  // base^(-2i/d)
+  // few tokens (a decode step): one token per CTA spreads them over the SMs; many (prefill, history): four per CTA
+  // amortise the set-up and keep more 16-byte units in flight per thread
+  if (n < 2048)
+    rope_write_kv_kernel<T, D, 1><<<n, 256, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_rot, (T*)k_pages,
+                                                     (T*)v_pages, pos, slot, n, g->n_q_heads, g->n_kv_heads, tt);
+  else
+    rope_write_kv_kernel<T, D, 4><<<(n + 3) / 4, 256, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_rot,
+                                                               (T*)k_pages, (T*)v_pages, pos, slot, n, g->n_q_heads,
+                                                               g->n_kv_heads, tt);
+  mv::g_launches++;
+  if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
+  return MV_OK;
 }
 
 template <typename T>
 mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* q_rot,
                  void* k_rot, void* k_pages, void* v_pages, cudaStream_t st) {
-  const int n = int(P->stats.n_new_tokens);
-  const int32_t* pos = mv::table<int32_t>(P, P->layout.pos_id);
-  const int64_t* slot = mv::table<int64_t>(P, P->layout.slot);
-  const double c = -2.0 * log2(g->rope_base) / double(g->head_dim);
-  if (g->head_dim == 128)
-    rope_write_kv_kernel<T, 128><<<n, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_rot,
-                                                    (T*)k_pages, (T*)v_pages, pos, slot, n, g->n_q_heads,
-                                                    g->n_kv_heads, c);
-  else
-    rope_write_kv_kernel<T, 64><<<n, 128, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_rot,
-                                                   (T*)k_pages, (T*)v_pages, pos, slot, n, g->n_q_heads,
-                                                   g->n_kv_heads, c);
-  mv::g_launches++;
-  if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
-  return MV_OK;
+  return g->head_dim == 128 ? launch_d<T, 128>(P, g, q, k, v, q_rot, k_rot, k_pages, v_pages, st)
+                            : launch_d<T, 64>(P, g, q, k, v, q_rot, k_rot, k_pages, v_pages, st);
 }
 
 }  // namespace

@@ -443,3 +443,23 @@ def test_empty_batch_is_a_no_op():
     geom = B.make_geom(8, 2, 128, 4, "bf16")
     B.mv_rope_write_kv(plan, geom, None, None, None, None, None, None, None)
     torch.cuda.synchronize()
+
+
+def test_bounded_wait_runs_out_with_a_status_not_a_fault():
+    """A device-side wait that nothing completes: the one-thread probe kernel gives up after its limit (1 ms here),
+    MV_ERR_TIMEOUT arrives through the plan's status word, and the context keeps working.  (The attention kernels use
+    the same wait; making THEM time out would mean breaking their barrier protocol, which is never done on a GPU.)"""
+    B, rt = _B(), _rt()
+    wl = synth.config2(n_req=2, prefix=300, branches=3, branch_len=50)
+    st = rt.DecodeState(wl)
+    want = _np(st.step())
+    assert st.plan.read_status() == 0
+    B.mv_selftest_bounded_wait(st.plan, 1_000_000)
+    assert st.plan.read_status() == 7
+    assert B.mv_status_string(7).startswith("MV_ERR_TIMEOUT")
+    with pytest.raises(B.MvError):
+        B.mv_selftest_bounded_wait(st.plan, 10**10)           # limits beyond a tenth of a second are refused
+    st.plan.upload(st.pod.tables)                             # a fresh upload clears the word
+    assert st.plan.read_status() == 0
+    assert np.array_equal(_np(st.step()), want)
+    check_decode(wl, want)

@@ -273,6 +273,40 @@ def test_brute_force_eq3_tiny():
     assert max_abs(o0[16:], ref[16:]) > 1e-3
 
 
+def test_layerwise_visibility_follows_frontier_layers_not_node_numbering():
+    """Literal mode on a DAG whose numbering is not layer-sorted: node 3 (child of the prefix) is in layer 1,
+    node 2 (child of node 1) in layer 2, so node 2 must see node 3 although node 3's tokens come later in the
+    given order.  The paper lays its training sequence out frontier layer by frontier layer (Sec. 4.2, text above
+    Eq. 3); Eq. 3 is therefore evaluated by brute force on the tokens re-laid-out in that order, and the oracle's
+    output on the given order, permuted the same way, must agree.  Applying `j <= i` of the given order across
+    nodes would hide node 3 from node 2 and fail here."""
+    parents = [[], [0], [1], [0]]
+    lens = [5, 3, 4, 2]
+    reqs = [[(p, 0, n) for p, n in zip(parents, lens)]]
+    b = _mk(reqs, vis_mode=O.VIS_LAYERWISE)
+    t = O.plan_tables(b)
+    assert t["layer"].tolist() == [0, 1, 2, 1]
+    T, Hq, Hkv, d = sum(lens), 2, 1, 8
+    q, k, v = _rand((T, Hq, d), 30), _rand((T, Hkv, d), 31), _rand((T, Hkv, d), 32)
+    node_of_tok = [n for n, l in enumerate(lens) for _ in range(l)]
+    # frontier-layer order: nodes 0, 1, 3, 2 (stable inside a layer)
+    order = sorted(range(T), key=lambda i: (int(t["layer"][node_of_tok[i]]), i))
+    assert [node_of_tok[i] for i in order] == [0] * 5 + [1] * 3 + [3] * 2 + [2] * 4
+    qr, kr = O.rope_rotate(q, t["pos_id"]), O.rope_rotate(k, t["pos_id"])   # positions depend on the DAG, not on the layout
+    step = [node_of_tok[i] for i in order]
+    layer = [int(t["layer"][s]) for s in step]
+    ref_sorted = _brute_force_eq3(qr[order], kr[order], v[order], layer, step, 1.0 / math.sqrt(d))
+    ref = np.zeros_like(ref_sorted)
+    ref[order] = ref_sorted
+    got = O.prefill_request(b, 0, q, k, v)
+    assert max_abs(got, ref) < 1e-12
+    # the same brute force on the given order (node 3 after node 2) hides node 3 from node 2 and shows the later
+    # layer's node 2 to node 3: different results on exactly those two nodes
+    naive = _brute_force_eq3(qr, kr, v, [int(t["layer"][n]) for n in node_of_tok], node_of_tok, 1.0 / math.sqrt(d))
+    assert max_abs(naive[8:12], ref[8:12]) > 1e-3 and max_abs(naive[12:], ref[12:]) > 1e-3
+    assert max_abs(naive[:8], ref[:8]) < 1e-12
+
+
 def test_softmax_rows_sum_to_one_and_gqa_consistency():
     wl = synth.config1()
     b = batch_dict(wl.batch)

@@ -136,3 +136,19 @@ def test_append_tiles_in_the_plan_statistics():
     fresh = synth.build_batch([[([], 0, 300), ([0], 0, 70)]], rng=np.random.default_rng(5))
     st = B.Plan(fresh, 0, 8, 4).stats()
     assert st["prefill_ready"] == 1 and st["append_tiles"] == 0 and st["n_q_tiles"] == 3 + 1
+
+
+def test_tensor_map_cache_is_keyed_by_device_pointers_and_extent():
+    """The launchers' tensor-map cache (four entries, oldest replaced): the same pointers on another device, another row
+    count or another extra word are different entries; a fifth key evicts the first."""
+    probe = B.mv_selftest_tmap_cache
+    k, v = 0x7F0000001000, 0x7F0000201000
+    assert probe(0, k, v, 0, 4096, 128, reset=True) is False      # first sight: cached now
+    assert probe(0, k, v, 0, 4096, 128) is True
+    assert probe(1, k, v, 0, 4096, 128) is False                  # same addresses, second device of the process
+    assert probe(0, k, v, 0, 8192, 128) is False                  # the pool grew
+    assert probe(0, k, v, 0, 4096, 64) is False                   # other head_dim
+    assert probe(0, k, v, 0, 4096, 128) is True and probe(1, k, v, 0, 4096, 128) is True
+    assert probe(0, v, k, 0, 4096, 128) is False                  # K and V swapped: fifth key, evicts the oldest entry
+    assert probe(0, k, v, 0, 4096, 128) is False                  # ... which was the first one
+    assert probe(0, k, v, k, 4096, 128) is False                  # a third pointer is part of the key
