@@ -3,12 +3,17 @@
 
 A step is one pass of the whole decode hot path over one synthetic batch: DAG planning on the host
 (mv_plan_dag), table upload, RoPE with adaptive positions fused into the KV write (mv_rope_write_kv) and
-multi-branch decode attention (mv_dag_decode_attn).  The workload is the multi-branch decode step with
-Llama-3-8B attention geometry (16 requests x 4 branches, 2048-token shared prefix, bf16 paged KV).
+multi-branch decode attention (mv_dag_decode_attn).  The headline workload is the large serving mix
+(128 requests, Llama-3-70B attention geometry, prefixes of 512 to 16 384 tokens, 2 to 8 sibling branches, a
+join in a quarter of the requests); the other workloads run as named legs of the same line: the multi-branch
+decode step and the random layered DAG (decode), RoPE + cache write on a decode step and on the 17K-token
+prefill, the topology-masked prefill, node append, and the tiny float32 fork/join example.
 Successive steps rotate over several independent KV pool copies whose total exceeds L2 several times, so
-every step streams its KV from HBM.
+every step streams its KV from HBM.  Every timed loop is repeated until it has run for at least half a second;
+the figures are medians over the repeats.  After its timing each leg checks the buffers it timed against the
+CPU oracle (outside the timed region).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload config2|config3|config5]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload config5|config3|config2]
 
 N > 1 (under torchrun): every rank draws its own batch of the same shape (requests are independent, there is no
 collective on the path); the time is the maximum over ranks, the value the sum of the rows over ranks.
@@ -32,9 +37,16 @@ import numpy as np
 
 METRIC = "dag_decode_attn_query_tokens_per_s"
 UNIT = "query-tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_attn_kernel launch on this workload, taken from the
-# ncu capture summarised in profiles/ (None until a capture exists for the current kernel).
-NCU_TRAFFIC_BYTES = {"config2": 210_300_000}
+MIN_LEG_SECONDS = 0.5
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the leg's dominant kernel, per workload, with the
+# summary under profiles/ that holds the capture (None where the kernel has no capture of its own; see "scaled").
+NCU_TRAFFIC = {
+    "config2": {"bytes": 210_300_000, "kernel": "decode_tc_kernel", "profile": "profiles/decode_tc_kernel_config2.md"},
+    "config3": {"bytes": None, "kernel": "decode_tc_kernel", "profile": "profiles/decode_tc_kernel_config3.md"},
+    "config5": {"bytes": None, "kernel": "decode_tc_kernel", "profile": None},
+}
+BF16_TOL = (2e-2, 1e-2)   # max-abs, relative L2 against the float64 oracle
+F32_TOL = 1e-4
 
 
 def _peaks():
@@ -52,14 +64,20 @@ def _workload(name, rank=0):
     return multirank.rank_workload({"config2": synth.config2, "config3": synth.config3, "config5": synth.config5}[name], rank)
 
 
-class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons of one GPU through NVML (read-only) while the benchmark runs."""
+def _batch_dict(batch):
+    return {f.name: getattr(batch, f.name) for f in dataclasses.fields(batch)}
 
-    def __init__(self, index: int, period_s: float = 0.02):
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML (read-only) while the benchmark runs: every 5 ms
+    while ``active`` is set, plus one sample whenever ``sample_now`` is called (start and end of every timed region)."""
+
+    def __init__(self, index: int, period_s: float = 0.005):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop_evt = threading.Event()
+        self._lock = threading.Lock()
         self.active = False
         self.ok = False
         try:
@@ -71,46 +89,68 @@ class ClockSampler(threading.Thread):
             self.ok = True
         except Exception:
             self.ok = False
+        nv = getattr(self, "nv", None)
+        self.names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                      "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                      "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                      "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+                      "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80)}
 
-    def run(self):
+    def sample_now(self):
         if not self.ok:
             return
         nv = self.nv
-        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
-                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
-                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
-                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
-                 "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80)}
+        try:
+            mhz = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            try:
+                r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+            except Exception:
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            with self._lock:
+                self.samples.append(mhz)
+                for k, bit in self.names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+        except Exception:
+            pass
+
+    def run(self):
         while not self._stop_evt.is_set():
             if self.active:
-                try:
-                    self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
-                    try:
-                        r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
-                    except Exception:
-                        r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
-                    for k, bit in names.items():
-                        if r & bit:
-                            self.reasons.add(k)
-                except Exception:
-                    pass
+                self.sample_now()
             time.sleep(self.period)
 
     def stop(self):
         self._stop_evt.set()
 
     def summary(self):
-        if not self.samples:
+        with self._lock:
+            s, r = list(self.samples), sorted(self.reasons)
+        if not s:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
-        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        return {"sm_mhz": float(np.median(s)), "sm_max_mhz": self.max_mhz, "reasons": r, "samples": len(s)}
+
+
+class Region:
+    """Marks a timed region for the clock sampler."""
+
+    def __init__(self, sampler):
+        self.s = sampler
+
+    def __enter__(self):
+        self.s.sample_now()
+        self.s.active = True
+
+    def __exit__(self, *exc):
+        self.s.active = False
+        self.s.sample_now()
 
 
 def _oracle_sample(wl, budget_s: float):
     """Times the CPU oracle, as it stands, on whole requests of the workload until ~budget_s is used."""
     from oracle import medverse_oracle as O
     from paper_2602_07529_b200 import synth
-    b = {f.name: getattr(wl.batch, f.name) for f in dataclasses.fields(wl.batch)}
+    b = _batch_dict(wl.batch)
     rows, t_used, n_req = 0, 0.0, 0
     for r in range(wl.batch.n_req):
         vals = synth.request_values(wl, r)      # input generation is not timed
@@ -155,6 +195,207 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------------------------------------ helpers
+
+def _bf16_err(got, want):
+    got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
+    return float(np.max(np.abs(got - want))), float(np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-300))
+
+
+def _median_launch_ms(torch, fn, warmup=5, min_launches=20, min_seconds=None, max_launches=4000):
+    """Median CUDA-event time of one call of ``fn(i)``: at least ``warmup`` untimed and ``min_launches`` timed calls,
+    and as many more as it takes for the timed calls to add up to ``min_seconds``."""
+    min_seconds = MIN_LEG_SECONDS if min_seconds is None else min(min_seconds, MIN_LEG_SECONDS)
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    times, total, i = [], 0.0, warmup
+    while len(times) < min_launches or (total < min_seconds and len(times) < max_launches):
+        batch = []
+        for _ in range(10):
+            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn(i)
+            c.record()
+            batch.append((a, c))
+            i += 1
+        torch.cuda.synchronize()
+        for a, c in batch:
+            t = a.elapsed_time(c)
+            times.append(t)
+            total += t * 1e-3
+    return float(np.median(times)), float(np.min(times)), len(times), float(np.median(times[:min_launches]))
+
+
+def _decode_parity(wl, got, requests):
+    """The step's output rows of the listed requests against the oracle: (max-abs, relative L2, rows checked)."""
+    from oracle import medverse_oracle as O
+    from paper_2602_07529_b200 import synth
+    b = _batch_dict(wl.batch)
+    first, acc = [], 0
+    for r in range(wl.batch.n_req):
+        first.append(acc)
+        acc += int(sum(int(wl.batch.node_new[n]) for n in wl.batch.request_nodes(r)))
+    g, w = [], []
+    for r in requests:
+        vals = synth.request_values(wl, r)
+        o = O.decode_request(b, r, vals["q"], vals["k"], vals["v"], base=wl.geom.rope_base)
+        w.append(o)
+        g.append(got[first[r]:first[r] + o.shape[0]])
+    g, w = np.concatenate(g, 0), np.concatenate(w, 0)
+    err, rel = _bf16_err(g, w)
+    return {"max_abs": err, "rel_l2": rel, "rows": int(g.shape[0]), "requests": len(requests),
+            "ok": bool(np.isfinite(g).all() and err <= BF16_TOL[0] and rel <= BF16_TOL[1])}
+
+
+def _parity_requests(wl, how_many):
+    """Which requests a leg checks: all of them if that is at most ``how_many``; else the shortest and the longest
+    context, every other request evenly spread, requests with a join first."""
+    b = wl.batch
+    n = b.n_req
+    if n <= how_many:
+        return list(range(n))
+    prefix = np.asarray([int(b.node_len[b.node_off[r]]) for r in range(n)])
+    joins = [r for r in range(n) if len(b.parents_of(int(b.node_off[r + 1]) - 1)) > 1]
+    pick = [int(np.argmin(prefix)), int(np.argmax(prefix))] + joins[:max(1, how_many // 3)]
+    for r in np.linspace(0, n - 1, how_many).astype(int):
+        if len(set(pick)) >= how_many:
+            break
+        pick.append(int(r))
+    return sorted(set(pick))[:how_many]
+
+
+class DecodeLeg:
+    """One decode workload resident on the device, with what its timed loops need marshalled once."""
+
+    def __init__(self, torch, wl, dev, chunk=0):
+        from paper_2602_07529_b200 import binding as B, runtime
+        self.torch, self.B, self.wl, self.dev = torch, B, wl, dev
+        g, b = wl.geom, wl.batch
+        self.pool_bytes = 2 * b.num_pages * g.n_kv_heads * g.page_size * g.head_dim * 2
+        self.n_pools = max(2, min(8, int(np.ceil(1.0e9 / self.pool_bytes))))
+        self.st = runtime.DecodeState(wl, dev, chunk_tokens=chunk, n_pool_copies=self.n_pools)
+        st = self.st
+        self.stats = st.plan.stats()
+        self.rows = self.stats["n_new_tokens"]
+        kv_tok_bytes = g.n_kv_heads * g.head_dim * 2 * 2
+        qo_bytes = 2 * self.rows * g.n_q_heads * g.head_dim * 2
+        self.algo_bytes = self.stats["unique_kv_tokens"] * kv_tok_bytes + qo_bytes
+        self.naive_bytes = self.stats["per_row_kv_tokens"] * kv_tok_bytes + qo_bytes
+        # ring of plans / table buffers so that re-planning never races an upload in flight
+        self.RING = 4
+        self.plans = [B.Plan(b, chunk, g.n_kv_heads, g.group) for _ in range(self.RING)]
+        self.tables = [torch.empty(max(256, self.plans[0].device_bytes() * 2), dtype=torch.uint8, device=dev) for _ in range(self.RING)]
+        self.ring_ev = [torch.cuda.Event() for _ in range(self.RING)]
+        self.up_ev = [torch.cuda.Event() for _ in range(self.RING)]
+        self.stream = torch.cuda.current_stream()
+        # the table upload of a step goes through a copy stream, so that it travels while the previous step's kernels run
+        self.copy_stream = torch.cuda.Stream(device=dev)
+        vp_ = C.c_void_p
+        self.sp, self.csp = vp_(self.stream.cuda_stream), vp_(self.copy_stream.cuda_stream)
+        # every pointer the timed loop passes is fixed: marshal them once, so that the host side of a step is the
+        # library calls themselves (a C caller has no per-call marshalling either)
+        self.cb = self.plans[0].c_batch
+        self.gref, self.cbref = C.byref(st.geom), C.byref(self.cb)
+        self.plan_refs = [C.byref(p._h) for p in self.plans]
+        self.tab_ptr = [vp_(t.data_ptr()) for t in self.tables]
+        self.tab_len = [t.numel() for t in self.tables]
+        self.pool_ptr = [(vp_(kp.data_ptr()), vp_(vp.data_ptr())) for kp, vp in st.pools]
+        self.q_p, self.k_p, self.v_p, self.qrot_p, self.out_p, self.ws_p = (
+            vp_(t.data_ptr()) for t in (st.q, st.k, st.v, st.q_rot, st.out, st.workspace))
+        self.ws_bytes = st.workspace.numel()
+        self.lib = B.lib
+
+    def step(self, i, ev_pair=None):
+        lib, s = self.lib, i % self.RING
+        self.ring_ev[s].synchronize()
+        h = self.plans[s]._h
+        rc = lib.mv_plan_dag(self.cbref, self.plan_refs[s])
+        rc |= lib.mv_plan_upload(h, self.tab_ptr[s], self.tab_len[s], self.csp)
+        self.up_ev[s].record(self.copy_stream)
+        self.stream.wait_event(self.up_ev[s])
+        kp, vp = self.pool_ptr[i % self.n_pools]
+        rc |= lib.mv_rope_write_kv(h, self.gref, self.q_p, self.k_p, self.v_p, self.qrot_p, None, kp, vp, self.sp)
+        if ev_pair is not None:
+            ev_pair[0].record(self.stream)
+        rc |= lib.mv_dag_decode_attn(h, self.gref, self.qrot_p, kp, vp, self.out_p, self.ws_p, self.ws_bytes, self.sp)
+        if ev_pair is not None:
+            ev_pair[1].record(self.stream)
+        self.ring_ev[s].record(self.stream)
+        if rc:
+            raise RuntimeError(f"library call failed with status {rc}")
+
+    def timed_steps(self, K, W, barrier, region, agree=lambda n: n, max_repeats=200):
+        """W warm-up steps, then repeats of exactly K timed steps (barrier + synchronise on both sides of each repeat)
+        until the repeats add up to min_seconds: the number of repeats follows from the first one (``agree`` makes the
+        ranks of a multi-GPU run settle on one number).  Returns per repeat the K-step time and the per-call decode times."""
+        torch = self.torch
+        for i in range(W):
+            self.step(i)
+        barrier()
+        stride = max(1, K // 500)   # the decode call is timed per launch on a subsample of the steps (every step for short runs)
+        reps, n, n_reps = [], W, 1
+        with region:
+            while len(reps) < n_reps:
+                pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range((K + stride - 1) // stride)]
+                ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                barrier()
+                ev0.record(self.stream)
+                for i in range(K):
+                    self.step(n + i, pairs[i // stride] if i % stride == 0 else None)
+                ev1.record(self.stream)
+                barrier()
+                n += K
+                reps.append((ev0.elapsed_time(ev1), [a.elapsed_time(c) for a, c in pairs]))
+                if len(reps) == 1:
+                    n_reps = agree(int(min(max_repeats, max(1, np.ceil(MIN_LEG_SECONDS / max(reps[0][0] * 1e-3, 1e-6))))))
+        return reps
+
+    def burst_ms(self, n=50):
+        """Back-to-back mv_dag_decode_attn calls (no events in between) over the rotating pools: time per call."""
+        torch = self.torch
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(self.stream)
+        for i in range(n):
+            kp, vp = self.pool_ptr[i % self.n_pools]
+            self.lib.mv_dag_decode_attn(self.plans[0]._h, self.gref, self.qrot_p, kp, vp, self.out_p, self.ws_p, self.ws_bytes, self.sp)
+        c.record(self.stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(c) / n
+
+    def roofline(self, decode_ms, decode_ms_min, peaks, name):
+        achieved = self.algo_bytes / (decode_ms * 1e-3) / 1e9
+        tr = NCU_TRAFFIC.get(name, {})
+        return {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": tr.get("bytes"), "traffic_source": tr.get("profile"),
+                "peak_source": peaks["source"],
+                "kernel": "decode_tc_kernel + decode_merge_kernel (one mv_dag_decode_attn call; the traffic figure is decode_tc_kernel alone)",
+                "algorithmic_bytes": self.algo_bytes, "launch_ms_mean": decode_ms, "launch_ms_min": decode_ms_min,
+                "frac_of_nominal_8TBs": achieved / 8000.0, "naive_per_row_GBs": self.naive_bytes / (decode_ms * 1e-3) / 1e9,
+                "decode_query_tokens_per_s": self.rows / (decode_ms * 1e-3)}
+
+    def parity(self, how_many):
+        self.torch.cuda.synchronize()
+        got = self.st.out.float().cpu().numpy()
+        return _decode_parity(self.wl, got, _parity_requests(self.wl, how_many))
+
+    def rope_leg(self, peaks):
+        """mv_rope_write_kv alone on this step's new tokens (read q, k, v; write q_rot and the K / V pool slots)."""
+        g, st = self.wl.geom, self.st
+        n = self.rows
+        nbytes = 2 * n * (g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim * 2
+        def call(i):
+            kp, vp = self.pool_ptr[i % self.n_pools]
+            self.lib.mv_rope_write_kv(self.plans[0]._h, self.gref, self.q_p, self.k_p, self.v_p, self.qrot_p, None, kp, vp, self.sp)
+        self.plans[0].upload(self.tables[0])
+        ms, ms_min, launches, _ = _median_launch_ms(self.torch, call, min_seconds=0.1)
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        return {"workload": self.wl.name, "tokens": int(n), "ms": ms, "ms_min": ms_min, "launches": launches, "algorithmic_bytes": nbytes,
+                "GBs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0,
+                "note": "a decode step's few tokens: launch-bound, the fraction is reported for completeness"}
+
+
 def run_ours(args):
     import torch
     from paper_2602_07529_b200 import binding as B, multirank, runtime, synth
@@ -172,214 +413,234 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     peaks = _peaks()
 
-    wl = _workload(args.workload, rank)
-    g, b = wl.geom, wl.batch
-    pool_bytes = 2 * b.num_pages * g.n_kv_heads * g.page_size * g.head_dim * 2
-    n_pools = max(2, min(8, int(np.ceil(1.0e9 / pool_bytes))))
-    st = runtime.DecodeState(wl, dev, chunk_tokens=args.chunk, n_pool_copies=n_pools)
-    stats = st.plan.stats()
-    rows = stats["n_new_tokens"]
-    kv_tok_bytes = g.n_kv_heads * g.head_dim * 2 * 2
-    qo_bytes = 2 * rows * g.n_q_heads * g.head_dim * 2
-    algo_bytes = stats["unique_kv_tokens"] * kv_tok_bytes + qo_bytes
-    naive_bytes = stats["per_row_kv_tokens"] * kv_tok_bytes + qo_bytes
-
-    # ---- ring of plans / table buffers so that re-planning never races an upload in flight
-    RING = 4
-    plans = [B.Plan(b, args.chunk, g.n_kv_heads, g.group) for _ in range(RING)]
-    tables = [torch.empty(max(256, plans[0].device_bytes() * 2), dtype=torch.uint8, device=dev) for _ in range(RING)]
-    ring_ev = [torch.cuda.Event() for _ in range(RING)]
-    cb = plans[0].c_batch
-    stream = torch.cuda.current_stream()
-    sp = C.c_void_p(stream.cuda_stream)
-    geom = st.geom
-    lib = B.lib
-    ws_bytes = st.workspace.numel()
-
-    # every pointer the timed loop passes is fixed: marshal them once, so that the host side of a step is the library
-    # calls themselves (a C caller has no per-call marshalling either)
-    vp_ = C.c_void_p
-    gref, cbref = C.byref(geom), C.byref(cb)
-    plan_refs = [C.byref(p._h) for p in plans]
-    tab_ptr = [vp_(t.data_ptr()) for t in tables]
-    tab_len = [t.numel() for t in tables]
-    pool_ptr = [(vp_(kp.data_ptr()), vp_(vp.data_ptr())) for kp, vp in st.pools]
-    q_p, k_p, v_p, qrot_p, out_p, ws_p = (vp_(t.data_ptr()) for t in (st.q, st.k, st.v, st.q_rot, st.out, st.workspace))
-    plan_dag, plan_upload, rope_write_kv, dag_decode_attn = lib.mv_plan_dag, lib.mv_plan_upload, lib.mv_rope_write_kv, lib.mv_dag_decode_attn
-
-    # the table upload of a step goes through a copy stream, so that it travels while the previous step's kernels run
-    copy_stream = torch.cuda.Stream(device=dev)
-    csp = C.c_void_p(copy_stream.cuda_stream)
-    up_ev = [torch.cuda.Event() for _ in range(RING)]
-
-    def step(i, ev_pair=None):
-        s = i % RING
-        ring_ev[s].synchronize()
-        h = plans[s]._h
-        rc = plan_dag(cbref, plan_refs[s])
-        rc |= plan_upload(h, tab_ptr[s], tab_len[s], csp)
-        up_ev[s].record(copy_stream)
-        stream.wait_event(up_ev[s])
-        kp, vp = pool_ptr[i % n_pools]
-        rc |= rope_write_kv(h, gref, q_p, k_p, v_p, qrot_p, None, kp, vp, sp)
-        if ev_pair is not None:
-            ev_pair[0].record(stream)
-        rc |= dag_decode_attn(h, gref, qrot_p, kp, vp, out_p, ws_p, ws_bytes, sp)
-        if ev_pair is not None:
-            ev_pair[1].record(stream)
-        ring_ev[s].record(stream)
-        if rc:
-            raise RuntimeError(f"library call failed with status {rc}")
-
     def barrier():
         torch.cuda.synchronize()
         if dist is not None:
             dist.barrier()
             torch.cuda.synchronize()
 
+    def agree(n):   # the largest of the ranks' proposals, so that every rank runs the same number of repeats
+        if dist is None:
+            return n
+        t = torch.tensor([int(n)], dtype=torch.int64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return int(t.item())
+
     sampler = ClockSampler(local)
     sampler.start()
-    K, W = args.steps, max(args.warmup, 0)
-    for i in range(W):
-        step(i)
-    barrier()
-    # the decode call is timed per launch on a subsample of the steps (every step for short runs)
-    stride = max(1, K // 2000)
-    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range((K + stride - 1) // stride)]
+    region = Region(sampler)
+
+    # ---- headline: the decode step on the named workload
+    wl = _workload(args.workload, rank)
+    leg = DecodeLeg(torch, wl, dev, args.chunk)
+    g, b, rows, stats = wl.geom, wl.batch, leg.rows, leg.stats
+    K, W = args.steps, max(args.warmup, 3)
     launches0 = B.mv_launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler.active = True
-    ev0.record(stream)
-    for i in range(K):
-        step(W + i, pairs[i // stride] if i % stride == 0 else None)
-    ev1.record(stream)
-    barrier()
-    sampler.active = False
-    launches = B.mv_launch_count() - launches0
-    total_ms, job_rows = multirank.reduce_job(ev0.elapsed_time(ev1), rows * K, dist, dev)
-    decode_ms = float(np.mean([a.elapsed_time(c) for a, c in pairs]))
-    decode_ms_min = float(np.min([a.elapsed_time(c) for a, c in pairs]))
+    reps = leg.timed_steps(K, W, barrier, region, agree)
+    launches_all = B.mv_launch_count() - launches0
+    # the repeat with the median K-step time stands for the run; the maximum over ranks of that time counts
+    order = np.argsort([r[0] for r in reps])
+    med = reps[int(order[len(order) // 2])]
+    total_ms, job_rows = multirank.reduce_job(med[0], rows * K, dist, dev)
+    calls = np.concatenate([r[1] for r in reps])
+    decode_ms, decode_ms_min = float(np.mean(calls)), float(np.min(calls))
 
     # ---- end to end through the host-buffer entry point: H2D of the step's q/k/v + plan, D2H of the output
+    st = leg.st
     qh, kh, vh = (t.cpu().pin_memory() for t in (st.q, st.k, st.v))
     oh = torch.empty_like(qh).pin_memory()
-    staging = torch.empty(B.mv_decode_step_staging_bytes(plans[0], geom) * 2, dtype=torch.uint8, device=dev)
-    Ke = max(1, min(K, 2000))
-
+    staging = torch.empty(B.mv_decode_step_staging_bytes(leg.plans[0], st.geom) * 2, dtype=torch.uint8, device=dev)
+    vp_ = C.c_void_p
     qh_p, kh_p, vh_p, oh_p, stg_p, stg_len = (vp_(qh.data_ptr()), vp_(kh.data_ptr()), vp_(vh.data_ptr()), vp_(oh.data_ptr()),
                                               vp_(staging.data_ptr()), staging.numel())
-    decode_step_host = lib.mv_decode_step_host_batch
+    decode_step_host = B.lib.mv_decode_step_host_batch
+    stream = leg.stream
 
     def e2e_step(i):
-        kp, vp = pool_ptr[i % n_pools]
-        rc = decode_step_host(cbref, plan_refs[0], gref, qh_p, kh_p, vh_p, oh_p, kp, vp, stg_p, stg_len, sp)
+        kp, vp = leg.pool_ptr[i % leg.n_pools]
+        rc = decode_step_host(leg.cbref, leg.plan_refs[0], leg.gref, qh_p, kh_p, vh_p, oh_p, kp, vp, stg_p, stg_len, leg.sp)
         stream.synchronize()     # the caller consumes the output before it can form the next step
         if rc:
             raise RuntimeError(f"mv_decode_step_host failed with status {rc}")
 
+    Ke = max(1, min(K, 500))
     for i in range(min(W, 20)):
         e2e_step(i)
-    barrier()
-    sampler.active = True
-    t0 = time.perf_counter()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(Ke):
-        e2e_step(i)
-    e1.record(stream)
-    barrier()
-    sampler.active = False
-    e2e_wall_ms = 1e3 * (time.perf_counter() - t0)
-    e2e_ms, e2e_rows = multirank.reduce_job(e0.elapsed_time(e1), rows * Ke, dist, dev)
-    # parity guard on the buffers the timed run used: the e2e output equals the device-path output bit for bit
-    same = bool(torch.equal(oh, st.out.cpu()))
-    h2d = int(plans[0].device_bytes() + qh.numel() * 2 + kh.numel() * 2 + vh.numel() * 2)
+    e2e_reps, n_e2e = [], 1
+    with region:
+        while len(e2e_reps) < n_e2e:
+            barrier()
+            t0 = time.perf_counter()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(Ke):
+                e2e_step(i)
+            e1.record(stream)
+            barrier()
+            e2e_reps.append((e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)))
+            if len(e2e_reps) == 1:
+                n_e2e = agree(int(min(100, max(1, np.ceil(MIN_LEG_SECONDS / max(e2e_reps[0][0] * 1e-3, 1e-6))))))
+    e2e_med = sorted(e2e_reps)[len(e2e_reps) // 2]
+    e2e_ms, e2e_rows = multirank.reduce_job(e2e_med[0], rows * Ke, dist, dev)
+    same = bool(torch.equal(oh, st.out.cpu()))   # the e2e output equals the device-path output bit for bit
+    h2d = int(leg.plans[0].device_bytes() + qh.numel() * 2 + kh.numel() * 2 + vh.numel() * 2)
     d2h = int(oh.numel() * 2)
 
     # ---- host planner alone
+    n_plan = 200 if stats["n_new_tokens"] < 200 else 50
     t0 = time.perf_counter()
-    for _ in range(200):
-        lib.mv_plan_dag(C.byref(cb), C.byref(plans[1]._h))
-    planner_us = 1e6 * (time.perf_counter() - t0) / 200
+    for _ in range(n_plan):
+        B.lib.mv_plan_dag(leg.cbref, leg.plan_refs[1])
+    planner_us = 1e6 * (time.perf_counter() - t0) / n_plan
+    burst_ms = leg.burst_ms()
 
-    extra = {}
-    if rank == 0 and not args.no_prefill:
-        extra["prefill"] = _prefill_leg(torch, B, runtime, synth, dev, peaks)
-        extra["append"] = _append_leg(torch, B, runtime, synth, dev, peaks)
+    legs, parity = {}, {}
+    if rank == 0:
+        # parity of the buffers the timed run used (outside every timed region)
+        parity["decode_" + args.workload] = leg.parity(16)
+        if world == 1 and not args.no_legs:   # the legs belong to the single-GPU line; an N-GPU run holds N GPUs meanwhile
+            legs, leg_parity = _legs(torch, B, runtime, synth, dev, peaks, region, torch.cuda.synchronize, args, leg)
+            parity.update(leg_parity)
     sampler.stop()
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
-    cpu = None
-    if world == 1 or rank == 0:
-        v, n_rows, n_req, t_used, cores = _oracle_sample(wl, args.cpu_budget)
-        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"{n_req} whole request(s) = {n_rows} of {rows} rows of {wl.name}, {t_used:.1f} s, float64 numpy"}
-    step_ms = total_ms / K
-    achieved = algo_bytes / (decode_ms * 1e-3) / 1e9
+    v, n_rows, n_req, t_used, cores = _oracle_sample(wl, args.cpu_budget)
+    cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"{n_req} whole request(s) = {n_rows} of {rows} rows of {wl.name}, {t_used:.1f} s, float64 numpy"}
     line = {
         "metric": METRIC, "value": job_rows / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
-        "warmup": W, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "warmup": W, "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "requests": int(b.n_req), "rows": int(rows), "n_q_heads": g.n_q_heads,
                    "n_kv_heads": g.n_kv_heads, "head_dim": g.head_dim, "page_size": g.page_size,
                    "unique_kv_tokens": stats["unique_kv_tokens"], "per_row_kv_tokens": stats["per_row_kv_tokens"],
-                   "chunk_tokens": stats["chunk_tokens"], "work_items": stats["n_items"] * g.n_kv_heads,
-                   "l2": f"steps rotate over {n_pools} independent KV pool copies ({n_pools * pool_bytes / 1e9:.2f} GB in total, "
-                         f"{algo_bytes / 1e6:.0f} MB read per step) so every step streams from HBM",
+                   "chunk_tokens": stats["chunk_tokens"], "work_items": stats["n_items"],
+                   "repeats": len(reps), "repeat_rule": f"every timed loop is repeated until it has run {MIN_LEG_SECONDS} s; medians over the repeats",
+                   "l2": f"steps rotate over {leg.n_pools} independent KV pool copies ({leg.n_pools * leg.pool_bytes / 1e9:.2f} GB in total, "
+                         f"{leg.algo_bytes / 1e6:.0f} MB read per step) so every step streams from HBM",
                    "step": "mv_plan_dag + mv_plan_upload (copy stream) + mv_rope_write_kv + mv_dag_decode_attn",
                    "parallelism": (f"{world} ranks, one batch each, sharded by request, no collective" if world > 1 else "single")},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                     "peak_source": peaks["source"], "kernel": "decode_tc_kernel + decode_merge_kernel (one mv_dag_decode_attn call; the traffic figure is decode_tc_kernel alone)",
-                     "algorithmic_bytes": algo_bytes, "launch_ms_mean": decode_ms, "launch_ms_min": decode_ms_min,
-                     "frac_of_nominal_8TBs": achieved / 8000.0, "naive_per_row_GBs": naive_bytes / (decode_ms * 1e-3) / 1e9,
-                     "decode_query_tokens_per_s": rows / (decode_ms * 1e-3)},
+        "roofline": leg.roofline(decode_ms, decode_ms_min, peaks, args.workload),
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_rows / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": Ke, "ms_per_step": e2e_ms / Ke, "wall_ms_per_step": e2e_wall_ms / Ke,
+                "steps": Ke, "repeats": len(e2e_reps), "ms_per_step": e2e_ms / Ke, "wall_ms_per_step": e2e_med[1] / Ke,
                 "call": "mv_decode_step_host_batch (pinned host q/k/v in, planning inside the call while they travel, host out), stream synchronised every step",
                 "matches_device_path": same},
-        "gpu_launches": int(launches),
+        "gpu_launches": int(3 * K),
+        "gpu_launches_all_repeats": int(launches_all),
         "planner_us": planner_us,
+        "decode_burst_ms": burst_ms,
         "clocks": sampler.summary(),
+        "parity": parity,
     }
-    line.update(extra)
+    line["roofline"]["burst_ms"] = burst_ms
+    line["roofline"]["burst_frac"] = leg.algo_bytes / (burst_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]
+    line.update(legs)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------ legs
+
+def _legs(torch, B, runtime, synth, dev, peaks, region, barrier, args, headline_leg):
+    legs, parity = {}, {}
+    del headline_leg.st.pools[1:]          # the headline's extra pool copies are no longer needed
+    torch.cuda.empty_cache()
+    # ---- the other decode workloads, timed like the headline
+    for name in ("config2", "config3", "config5"):
+        if name == args.workload:
+            continue
+        if name == "config5" and args.workload != "config5":
+            continue   # the serving mix is either the headline or left out (its set-up takes the longest)
+        wl = _workload(name)
+        leg = DecodeLeg(torch, wl, dev)
+        K = 200 if name == "config2" else 100
+        reps = leg.timed_steps(K, 10, barrier, region)
+        calls = np.concatenate([r[1] for r in reps])
+        step_ms = float(np.median([r[0] for r in reps])) / K
+        rl = leg.roofline(float(np.mean(calls)), float(np.min(calls)), peaks, name)
+        burst = leg.burst_ms()
+        legs["decode_" + name] = {
+            "workload": wl.name, "rows": int(leg.rows), "ms": rl["launch_ms_mean"], "ms_min": rl["launch_ms_min"], "ms_per_step": step_ms,
+            "steps": K, "repeats": len(reps), "query_tokens_per_s": leg.rows / (step_ms * 1e-3),
+            "algorithmic_bytes": leg.algo_bytes, "GBs": rl["achieved"], "frac": rl["frac"], "frac_of_nominal_8TBs": rl["frac_of_nominal_8TBs"],
+            "traffic": rl["traffic"], "traffic_source": rl["traffic_source"], "burst_ms": burst,
+            "burst_frac": leg.algo_bytes / (burst * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "unique_kv_tokens": leg.stats["unique_kv_tokens"], "l2": f"{leg.n_pools} pool copies, {leg.n_pools * leg.pool_bytes / 1e9:.2f} GB"}
+        parity["decode_" + name] = leg.parity(16)
+        if name == "config2":
+            with region:
+                legs["rope_write_kv_config2"] = leg.rope_leg(peaks)
+        del leg
+        torch.cuda.empty_cache()
+    with region:
+        legs["prefill"], legs["rope_write_kv_config4"], p4 = _prefill_leg(torch, B, runtime, synth, dev, peaks)
+        legs["append"], pa = _append_leg(torch, B, runtime, synth, dev, peaks)
+        legs["prefill_config1_f32"], p1 = _config1_leg(torch, B, runtime, synth, dev)
+    parity["prefill_config4"], parity["append"], parity["prefill_config1"] = p4, pa, p1
+    return legs, parity
+
+
 def _prefill_leg(torch, B, runtime, synth, dev, peaks):
-    """Topology-masked prefill of the ~16K-token DAG sequence: useful (mask-aware) TFLOP/s of mv_dag_prefill_attn."""
+    """Topology-masked prefill of the ~16K-token DAG sequence: useful (mask-aware) TFLOP/s of mv_dag_prefill_attn, and
+    mv_rope_write_kv alone over the same tokens (q, k rotated; k, v written to token order and to the page pool)."""
+    from oracle import medverse_oracle as O
     wl = synth.config4()
-    st = runtime.PrefillState(wl, dev, with_pool=False)
+    st = runtime.PrefillState(wl, dev, with_pool=True)
     stats = st.plan.stats()
     g = wl.geom
     flops = 4.0 * g.head_dim * g.n_q_heads * stats["visible_pairs"]
     st.step()
-    torch.cuda.synchronize()
-    evs = []
-    for _ in range(5):
-        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        B.mv_dag_prefill_attn(st.plan, st.geom, st.q_rot, st.k_rot, st.v, st.out)
-        c.record()
-        evs.append((a, c))
-    torch.cuda.synchronize()
-    ms = float(np.median([a.elapsed_time(c) for a, c in evs]))
-    tf = flops / (ms * 1e-3) / 1e12
-    return {"workload": wl.name, "tokens": stats["n_new_tokens"], "ms": ms, "useful_tflops": tf,
-            "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"], "frac_of_nominal_2250": tf / 2250.0,
-            "visible_pairs": stats["visible_pairs"], "tile_pairs": stats["tile_pairs"],
-            "executed_tflops": 4.0 * g.head_dim * g.n_q_heads * stats["tile_pairs"] / (ms * 1e-3) / 1e12}
+    ms, ms_min, launches, ms20 = _median_launch_ms(torch, lambda i: B.mv_dag_prefill_attn(st.plan, st.geom, st.q_rot, st.k_rot, st.v, st.out))
+    tf, tf20 = flops / (ms * 1e-3) / 1e12, flops / (ms20 * 1e-3) / 1e12
+    prefill = {"workload": wl.name, "tokens": stats["n_new_tokens"], "ms": ms, "ms_min": ms_min, "launches": launches, "warmup": 5,
+               "useful_tflops": tf, "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+               "ms_first_20_launches": ms20, "useful_tflops_first_20_launches": tf20,
+               "frac_of_measured_bf16_peak": tf20 / peaks["bf16_tflops"],
+               "peak_note": "the median over the whole half-second loop runs under the power cap and is set against the sustained "
+                            "matmul peak; the first 20 launches after warm-up run like a burst and are set against the burst peak",
+               "frac_of_nominal_2250": tf20 / 2250.0,
+               "visible_pairs": stats["visible_pairs"], "tile_pairs": stats["tile_pairs"],
+               "executed_tflops": 4.0 * g.head_dim * g.n_q_heads * stats["tile_pairs"] / (ms * 1e-3) / 1e12}
+    # parity on the timed buffers: sampled rows (every node's first and last rows, tile-boundary rows, random rows)
+    b = wl.batch
+    rows, start = set(), 0
+    for n in range(b.n_nodes):
+        ln = int(b.node_new[n])
+        rows.update(start + t for t in (0, ln - 1, 127, 128) if 0 <= t < ln)
+        start += ln
+    rows.update(int(x) for x in np.random.default_rng(4).choice(start, size=96, replace=False))
+    rows = sorted(rows)
+    vals = synth.request_values(wl, 0)
+    want = O.prefill_request(_batch_dict(b), 0, vals["q"], vals["k"], vals["v"], base=g.rope_base, rows=rows)
+    got = st.out.float().cpu().numpy()[rows]
+    err, rel = _bf16_err(got, want)
+    parity = {"max_abs": err, "rel_l2": rel, "rows": len(rows), "ok": bool(err <= BF16_TOL[0] and rel <= BF16_TOL[1])}
+    # RoPE + cache write over the same 17K tokens, every output the call has (q_rot, k_rot, K and V pool slots)
+    n = stats["n_new_tokens"]
+    rd = n * (g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim * 2
+    wr = n * (g.n_q_heads + 3 * g.n_kv_heads) * g.head_dim * 2      # q_rot, k_rot, K slots, V slots
+    rms, rms_min, rl, _ = _median_launch_ms(torch, lambda i: B.mv_rope_write_kv(st.plan, st.geom, st.q, st.k, st.v, st.q_rot, st.k_rot,
+                                                                              st.k_pages, st.v_pages), min_seconds=0.2)
+    gbs = (rd + wr) / (rms * 1e-3) / 1e9
+    pos = O.plan_tables(_batch_dict(b))["pos_id"]
+    sel = np.asarray(rows[:64])
+    qerr = float(np.max(np.abs(st.q_rot.float().cpu().numpy()[sel] - O.rope_rotate(vals["q"][sel], pos[sel], g.rope_base))))
+    rope = {"workload": wl.name, "tokens": int(n), "ms": rms, "ms_min": rms_min, "launches": rl, "algorithmic_bytes": int(rd + wr),
+            "bytes_note": "read q, k, v; write q_rot, k_rot and the K / V pool slots (one more K write than the 2*n*(Hq+2Hkv)*d*B figure)",
+            "GBs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0,
+            "q_rot_max_abs_vs_oracle": qerr, "ok": bool(qerr <= 2.0 ** -8 * 6)}
+    return prefill, rope, parity
 
 
 def _append_leg(torch, B, runtime, synth, dev, peaks, new_tokens=128):
     """Node append on the multi-branch workload: every branch receives ``new_tokens`` tokens at once against the paged
     cache (the tiled form of mv_dag_decode_attn).  Useful flops count every (new token, visible key) pair once."""
+    from oracle import medverse_oracle as O
     wl = synth.config2(new_tokens=new_tokens)
     st = runtime.DecodeState(wl, dev, n_pool_copies=2)
     stats = st.plan.stats()
@@ -392,38 +653,67 @@ def _append_leg(torch, B, runtime, synth, dev, peaks, new_tokens=128):
         for v in range(1, hi - lo):
             pairs += int(nw[v] * (ln[0] + ln[v]) + nw[v] * (nw[v] + 1) // 2)
     flops = 4.0 * g.head_dim * g.n_q_heads * pairs
-    for i in range(3):
+    for i in range(2):
         st.step(i % 2)
-    torch.cuda.synchronize()
-    evs = []
-    for i in range(10):
+
+    def call(i):
         kp, vp = st.pools[i % 2]
-        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
         B.mv_dag_decode_attn(st.plan, st.geom, st.q_rot, kp, vp, st.out, st.workspace)
-        c.record()
-        evs.append((a, c))
+    ms, ms_min, launches, ms20 = _median_launch_ms(torch, call)
+    tf, tf20 = flops / (ms * 1e-3) / 1e12, flops / (ms20 * 1e-3) / 1e12
+    out = {"workload": f"{wl.name}, {new_tokens} new tokens per branch", "rows": stats["n_new_tokens"],
+           "query_tiles": stats["append_tiles"], "ms": ms, "ms_min": ms_min, "launches": launches, "warmup": 5,
+           "query_tokens_per_s": stats["n_new_tokens"] / (ms * 1e-3),
+           "visible_pairs": pairs, "useful_tflops": tf, "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+           "ms_first_20_launches": ms20, "useful_tflops_first_20_launches": tf20, "frac_of_measured_bf16_peak": tf20 / peaks["bf16_tflops"]}
+    # parity: sampled rows of two requests
     torch.cuda.synchronize()
-    ms = float(np.median([a.elapsed_time(c) for a, c in evs]))
-    tf = flops / (ms * 1e-3) / 1e12
-    return {"workload": f"{wl.name}, {new_tokens} new tokens per branch", "rows": stats["n_new_tokens"],
-            "query_tiles": stats["append_tiles"], "ms": ms, "query_tokens_per_s": stats["n_new_tokens"] / (ms * 1e-3),
-            "visible_pairs": pairs, "useful_tflops": tf, "frac_of_measured_bf16_peak": tf / peaks["bf16_tflops"]}
+    got_all = st.out.float().cpu().numpy()
+    per_req = 4 * new_tokens
+    bd = _batch_dict(b)
+    g_rows, w_rows = [], []
+    for r in (0, b.n_req - 1):
+        vals = synth.request_values(wl, r)
+        rows = sorted({0, 1, new_tokens - 1, new_tokens, 2 * new_tokens + 63, 3 * new_tokens + 64, per_req - 1})
+        o = O.append_request(bd, r, vals["q"], vals["k"], vals["v"], base=g.rope_base, rows=rows)
+        w_rows.append(o[rows])
+        g_rows.append(got_all[r * per_req:(r + 1) * per_req][rows])
+    err, rel = _bf16_err(np.concatenate(g_rows), np.concatenate(w_rows))
+    return out, {"max_abs": err, "rel_l2": rel, "rows": int(sum(x.shape[0] for x in g_rows)), "ok": bool(err <= BF16_TOL[0] and rel <= BF16_TOL[1])}
+
+
+def _config1_leg(torch, B, runtime, synth, dev):
+    """The tiny float32 fork/join prefill (240 tokens): launch-bound; time and full parity."""
+    from oracle import medverse_oracle as O
+    wl = synth.config1()
+    st = runtime.PrefillState(wl, dev)
+    st.step()
+    ms, ms_min, launches, _ = _median_launch_ms(torch, lambda i: B.mv_dag_prefill_attn(st.plan, st.geom, st.q_rot, st.k_rot, st.v, st.out),
+                                                 min_seconds=0.05)
+    vals = synth.request_values(wl, 0)
+    want = O.prefill_request(_batch_dict(wl.batch), 0, vals["q"], vals["k"], vals["v"])
+    err = float(np.max(np.abs(st.out.float().cpu().numpy() - want)))
+    return ({"workload": wl.name, "tokens": 240, "ms": ms, "ms_min": ms_min, "launches": launches},
+            {"max_abs": err, "rows": 240, "ok": bool(err <= F32_TOL)})
 
 
 def main():
+    global MIN_LEG_SECONDS
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20000)
-    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="config2", choices=["config2", "config3", "config5"])
+    ap.add_argument("--workload", default="config5", choices=["config2", "config3", "config5"])
     ap.add_argument("--chunk", type=int, default=0, help="decode split-KV chunk tokens (0 = automatic)")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for the CPU baseline")
-    ap.add_argument("--no-prefill", action="store_true")
+    ap.add_argument("--no-legs", "--no-prefill", dest="no_legs", action="store_true", help="headline workload only")
+    ap.add_argument("--min-seconds", type=float, default=MIN_LEG_SECONDS,
+                    help="every timed loop is repeated until it has run this long (short values are for profiler captures)")
     args = ap.parse_args()
+    MIN_LEG_SECONDS = args.min_seconds
     if args.impl == "reference":
-        if args.steps == 20000:
+        if args.steps == 300 and args.warmup == 20:
             args.steps, args.warmup = 3, 1
         run_reference(args)
     else:

@@ -154,7 +154,7 @@ typedef struct {
   int64_t max_node_new;        /* most new tokens any node receives                                         */
 } mv_plan_stats;
 
-enum { MV_OP_ROPE_WRITE_KV = 0, MV_OP_DECODE_ATTN = 1, MV_OP_PREFILL_ATTN = 2 };
+enum { MV_OP_ROPE_WRITE_KV = 0, MV_OP_DECODE_ATTN = 1, MV_OP_PREFILL_ATTN = 2, MV_OP_PREFILL_ATTN_BWD = 3 };
 
 /* DAG -> segment planner (Eq. 1 layering; Eq. 3 / Sec. 4.3 visibility; Sec. 4.2 positions; Sec. 3.2 KV index
  * lists).  Host only, integers only, deterministic.
@@ -183,7 +183,9 @@ mv_status mv_plan_upload(mv_plan* plan, void* device_buf, size_t device_buf_byte
 void mv_plan_destroy(mv_plan* plan);
 
 /* Workspace bytes (device, caller-owned, 256-byte aligned) an op needs for this plan and geometry.
- * MV_OP_DECODE_ATTN: split-KV partial outputs and softmax statistics.  The other ops need none (0). */
+ * MV_OP_DECODE_ATTN: split-KV partial outputs and softmax statistics.  MV_OP_PREFILL_ATTN: the optional per-(token,
+ * query head) log-sum-exp, n_new_tokens * n_q_heads floats (the call also runs without a workspace).
+ * MV_OP_PREFILL_ATTN_BWD: as many floats again.  MV_OP_ROPE_WRITE_KV needs none (0). */
 size_t mv_workspace_bytes(const mv_plan* plan, const mv_attn_geom* geom, int op);
 
 /* RoPE with adaptive positions fused into the KV-cache write (P(i) of Eq. 2 at the indices of Sec. 4.2).
@@ -262,10 +264,35 @@ mv_status mv_dag_decode_attn_static(const mv_plan* plan, const mv_attn_geom* geo
  *   v      device [T][n_kv_heads][head_dim]
  *   out    device [T][n_q_heads][head_dim]
  * dtype MV_F32 runs a float32 SIMT kernel, MV_BF16 the tensor-core kernel (float32 accumulation).
- * The plan must be prefill_ready, else MV_ERR_UNSUPPORTED.  workspace may be NULL (none needed). */
+ * The plan must be prefill_ready, else MV_ERR_UNSUPPORTED.
+ *   workspace  NULL, or device, 16-byte aligned, mv_workspace_bytes(plan, geom, MV_OP_PREFILL_ATTN) bytes: receives
+ *              lse[i][h] = log2 sum_j 2^(sm_scale * log2(e) * <q_i, k_j> + M_ij) as float [T][n_q_heads], which
+ *              mv_dag_prefill_attn_bwd takes.  Only the tcgen05 kernel (MV_BF16, head_dim 128, even group size,
+ *              16-byte aligned tensors) writes it; with any other shape a non-NULL workspace is MV_ERR_UNSUPPORTED. */
 mv_status mv_dag_prefill_attn(const mv_plan* plan, const mv_attn_geom* geom, const void* q_rot,
                               const void* k_rot, const void* v, void* out, void* workspace,
                               size_t workspace_bytes, void* cuda_stream);
+
+/* Backward of mv_dag_prefill_attn: the attention the model is fine-tuned through (Sec. 5.1) is Eq. 2 with the mask of
+ * Eq. 3 over the flattened training sequence at the position indices of Sec. 4.2.  Given dout = d loss / d out, with
+ * P_ij = softmax_j(sm_scale * <q_i, k_j> + M_ij) per query head and delta_i = <dout_i, out_i>:
+ *   dv[j]     = sum_i P_ij dout[i]                                    (summed over the query heads of j's KV head)
+ *   dS_ij     = P_ij * (<dout[i], v[j]> - delta_i)
+ *   dq_rot[i] = sm_scale * sum_j dS_ij k_rot[j],   dk_rot[j] = sm_scale * sum_i dS_ij q_rot[i]   (summed over the group)
+ * The gradients are with respect to the position-embedded q_rot and k_rot (the rotation of mv_rope_write_kv is a fixed
+ * orthogonal map per token).  Masked pairs contribute nothing; key tiles walk the transposed visibility (which query
+ * runs see this key's node), so ranges no query can see are never visited.
+ *   q_rot, k_rot, v, out   device, as given to / written by mv_dag_prefill_attn (bf16)
+ *   dout      device [T][n_q_heads][head_dim] bf16
+ *   lse       device [T][n_q_heads] float, as written by mv_dag_prefill_attn into its workspace
+ *   dq_rot    device [T][n_q_heads][head_dim] bf16, out;  dk_rot, dv  device [T][n_kv_heads][head_dim] bf16, out
+ *   workspace device, 256-byte aligned, mv_workspace_bytes(plan, geom, MV_OP_PREFILL_ATTN_BWD) bytes (scratch)
+ * All tensors 16-byte aligned.  MV_BF16, head_dim 128 and an even group size only (MV_ERR_UNSUPPORTED otherwise); the plan
+ * must be prefill_ready.  Deterministic (no atomics).  Errors: MV_ERR_INVALID_ARG, MV_ERR_UNSUPPORTED, MV_ERR_WORKSPACE,
+ * MV_ERR_CUDA. */
+mv_status mv_dag_prefill_attn_bwd(const mv_plan* plan, const mv_attn_geom* geom, const void* q_rot, const void* k_rot,
+                                  const void* v, const void* out, const void* dout, const void* lse, void* dq_rot,
+                                  void* dk_rot, void* dv, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* One decode step with HOST inputs and outputs (the end-to-end form of the path: Sec. 4.3 Phase II, one
  * frontier step).  Copies q, k, v (host, preferably page-locked, [n_rows][heads][head_dim]) to the device

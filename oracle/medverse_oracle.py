@@ -27,7 +27,9 @@ Pins (see tests, "-m 'not gpu'"): a linear chain equals dense causal attention w
 RoPE at 0..T-1 evaluated by an independent routine; sibling KV perturbation leaves a
 branch bit-identical; sibling order permutation invariance; fp64 brute force on tiny
 inputs; RoPE shift invariance; the fork/join positions of the tiny worked example;
-diamond closure; Floyd-Warshall reachability; GQA head consistency.
+diamond closure; Floyd-Warshall reachability; GQA head consistency; the backward pass by
+central finite differences of the forward, by torch's autograd on a linear chain, and by
+"a branch's output gradient leaves its siblings' dK and dV at zero".
 Absolute attention values: parity unpinned by the paper (it prints none); pinned only
 through the reductions above.
 """
@@ -360,3 +362,64 @@ def append_request(batch, r, q_raw, k_raw, v, base=10000.0, scale=None, rows=Non
             ri += 1
     return out
 
+
+
+# ----------------------------------------------------------------------------- backward (fine-tuning, Sec. 5.1)
+
+def masked_attention_backward(q, k, v, allow, dout, scale=None):
+    """Gradient of ``masked_attention`` with respect to its (position-embedded) q, k and v, by the definition.
+
+    The model is fine-tuned through exactly this attention: the mask of Eq. 3 over the flattened training sequence at
+    the position indices of Sec. 4.2 (Sec. 5.1).  For one query head, with S = scale * Q K^T + M, P = softmax(S) row by
+    row and O = P V, a perturbation dO of the output gives
+        dV = P^T dO,   dP = dO V^T,   dS_ij = P_ij * (dP_ij - sum_l P_il dP_il)   (the softmax Jacobian, row by row),
+        dQ = scale * dS K,   dK = scale * dS^T Q,
+    and a KV head collects dK and dV from every query head of its group.  Masked pairs have P = 0, hence dS = 0.
+    q [Tq, Hq, d], k / v [Tk, Hkv, d], allow [Tq, Tk] bool, dout [Tq, Hq, d].  Returns (dq, dk, dv) in float64.
+    """
+    q = np.asarray(q, np.float64)
+    k = np.asarray(k, np.float64)
+    v = np.asarray(v, np.float64)
+    dout = np.asarray(dout, np.float64)
+    Tq, Hq, d = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    dq = np.zeros_like(q)
+    dk = np.zeros_like(k)
+    dv = np.zeros_like(v)
+    for h in range(Hq):
+        kh, vh = k[:, h // G, :], v[:, h // G, :]
+        s = scale * (q[:, h, :] @ kh.T)
+        s = np.where(allow, s, -np.inf)
+        p = np.exp(s - s.max(axis=1, keepdims=True))
+        p = p / p.sum(axis=1, keepdims=True)
+        do = dout[:, h, :]
+        dv[:, h // G, :] += p.T @ do
+        dp = do @ vh.T
+        ds = p * (dp - (p * dp).sum(axis=1, keepdims=True))
+        dq[:, h, :] = scale * (ds @ kh)
+        dk[:, h // G, :] += scale * (ds.T @ q[:, h, :])
+    return dq, dk, dv
+
+
+def prefill_backward_request(batch, r, q_raw, k_raw, v, dout, base=10000.0, scale=None):
+    """Backward of ``prefill_request``: the flattened DAG sequence of request r, every token new.  Returns (dq_rot,
+    dk_rot, dv): the gradients with respect to the position-embedded queries and keys (the rotation itself is a fixed
+    orthogonal map per token; its transpose takes these back to the raw q and k) and to v, all float64, given the
+    gradient ``dout`` [T, Hq, d] of the output."""
+    lo, hi, parents, layer, vis, tot, start = _request_layout(batch, r)
+    tok_node, tok_index, pos = [], [], []
+    for v_local in range(hi - lo):
+        if int(batch["node_len"][lo + v_local]) != 0:
+            raise ValueError("prefill expects every token to be new")
+        for t in range(tot[v_local]):
+            tok_node.append(v_local)
+            tok_index.append(t)
+            pos.append(start[v_local] + t)
+    allow = allowed_mask(tok_node, tok_index, vis)
+    pos = np.asarray(pos, np.int64)
+    qr = rope_rotate(q_raw, pos, base)
+    kr = rope_rotate(k_raw, pos, base)
+    return masked_attention_backward(qr, kr, v, allow, dout, scale)

@@ -18,7 +18,7 @@ MV_OK = 0
 STATUS_NAMES = {0: "MV_OK", 1: "MV_ERR_INVALID_ARG", 2: "MV_ERR_NOT_TOPOLOGICAL", 3: "MV_ERR_PAGE_CAPACITY",
                 4: "MV_ERR_UNSUPPORTED", 5: "MV_ERR_WORKSPACE", 6: "MV_ERR_CUDA", 7: "MV_ERR_TIMEOUT"}
 MV_F32, MV_BF16 = 0, 1
-OP_ROPE_WRITE_KV, OP_DECODE_ATTN, OP_PREFILL_ATTN = 0, 1, 2
+OP_ROPE_WRITE_KV, OP_DECODE_ATTN, OP_PREFILL_ATTN, OP_PREFILL_ATTN_BWD = 0, 1, 2, 3
 TABLES = {"layer": (0, np.int32), "pos_start": (1, np.int32), "pos_id": (2, np.int32), "slot": (3, np.int64),
           "qnode": (4, np.int32), "qnode_tok_off": (5, np.int32), "seg_off": (6, np.int32),
           "seg_node": (7, np.int32), "seg_len": (8, np.int32), "kv_len": (9, np.int64)}
@@ -27,7 +27,7 @@ WORK_TABLES = {"stages": 10, "units": 11, "item_rows": 12, "cta_unit_off": 13, "
 
 EXPORTS = ["mv_plan_dag", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_bytes", "mv_plan_upload",
            "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
-           "mv_dag_prefill_attn", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_decode_step_host_batch", "mv_status_string",
+           "mv_dag_prefill_attn", "mv_dag_prefill_attn_bwd", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_decode_step_host_batch", "mv_status_string",
            "mv_launch_count", "mv_plan_read_status", "mv_dag_decode_attn_static",
            "mv_static_workspace_bytes", "mv_selftest_bounded_wait", "mv_selftest_tmap_cache",
            "mv_sched_create", "mv_sched_destroy", "mv_sched_add_request", "mv_sched_step", "mv_sched_rows",
@@ -86,6 +86,7 @@ def _load():
     lib.mv_rope_write_kv.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 8
     lib.mv_dag_decode_attn.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp, sz, vp]
     lib.mv_dag_prefill_attn.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp, sz, vp]
+    lib.mv_dag_prefill_attn_bwd.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 10 + [sz, vp]
     lib.mv_dag_decode_attn_static.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp]
     lib.mv_static_workspace_bytes.argtypes = []
     lib.mv_static_workspace_bytes.restype = sz
@@ -261,6 +262,12 @@ def mv_dag_prefill_attn(plan: Plan, geom: _Geom, q_rot, k_rot, v, out, workspace
     nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(lib.mv_dag_prefill_attn(plan.handle, C.byref(geom), _ptr(q_rot), _ptr(k_rot), _ptr(v), _ptr(out),
                                    _ptr(workspace), nbytes, _stream_ptr(stream)), "mv_dag_prefill_attn")
+
+
+def mv_dag_prefill_attn_bwd(plan: Plan, geom: _Geom, q_rot, k_rot, v, out, dout, lse, dq_rot, dk_rot, dv, workspace, stream=None):
+    _check(lib.mv_dag_prefill_attn_bwd(plan.handle, C.byref(geom), _ptr(q_rot), _ptr(k_rot), _ptr(v), _ptr(out), _ptr(dout), _ptr(lse),
+                                       _ptr(dq_rot), _ptr(dk_rot), _ptr(dv), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream_ptr(stream)), "mv_dag_prefill_attn_bwd")
 
 
 def mv_decode_step_staging_bytes(plan: Plan, geom: _Geom) -> int:

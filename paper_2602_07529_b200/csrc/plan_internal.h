@@ -56,9 +56,13 @@ struct KvRange {
   int32_t pages;   // paged form: index of the node's first page in the page table; flat form: 0
 };
 
+// Backward of the prefill (flat form only): the transposed lists.  A key tile is 128 keys of one node (QTile with
+// q_start / q_len read as the tile's first key and key count); its ranges (KvRange with kv_start / kv_len read as a
+// run of QUERY tokens) list the queries that see the tile: every token of every other node that sees the tile's node, and,
+// in the tile's own node, the queries from the tile's first key on (causal = 1: query i sees key j only if j <= i).
 struct DeviceLayout {  // byte offsets into the device table buffer (all multiples of 256)
   size_t pos_id = 0, slot = 0, stages = 0, units = 0, cta_unit_off = 0, cta_head = 0, item_rows = 0, rowkv_part_off = 0, sched = 0,
-         q_tiles = 0, kv_ranges = 0, page_tab = 0, total = 0;
+         q_tiles = 0, kv_ranges = 0, page_tab = 0, k_tiles = 0, q_ranges = 0, total = 0;
 };
 
 }  // namespace mv
@@ -77,6 +81,8 @@ struct mv_plan {
   int32_t sched_zero[64] = {};  // device-side status words ([2] = status of bounded waits), uploaded as zeros
   std::vector<mv::QTile> q_tiles;
   std::vector<mv::KvRange> kv_ranges;
+  std::vector<mv::QTile> k_tiles;        // backward: key tiles (see above), heaviest first
+  std::vector<mv::KvRange> q_ranges;     // backward: the query runs that see a key tile
   std::vector<int32_t> page_tab;         // paged tiles only: the batch's page ids
   mv_plan_stats stats{};
   int32_t page_size = 16;

@@ -57,6 +57,8 @@ extern "C" mv_status mv_plan_upload(mv_plan* P, void* device_buf, size_t device_
   put(h, L.q_tiles, P->q_tiles);
   put(h, L.kv_ranges, P->kv_ranges);
   put(h, L.page_tab, P->page_tab);
+  put(h, L.k_tiles, P->k_tiles);
+  put(h, L.q_ranges, P->q_ranges);
   // only the bytes in use travel (the tail of the last table)
   if (cudaMemcpyAsync(device_buf, h, need, cudaMemcpyHostToDevice, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
     (void)cudaGetLastError();
@@ -83,6 +85,9 @@ extern "C" size_t mv_workspace_bytes(const mv_plan* P, const mv_attn_geom* g, in
     const size_t ml = (vecs * 2 * sizeof(float) + 255) & ~size_t(255);
     return o + ml + 256;
   }
+  const size_t row_heads = size_t(P->stats.n_new_tokens) * size_t(g->n_q_heads);
+  // prefill: the optional per-(row, head) log-sum-exp; backward: the per-(row, head) dot products of dO and O
+  if (op == MV_OP_PREFILL_ATTN || op == MV_OP_PREFILL_ATTN_BWD) return (row_heads * sizeof(float) + 255) & ~size_t(255);
   return 0;
 }
 

@@ -108,7 +108,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   P->seg_off.assign(1, 0);
   P->seg_node.clear(); P->seg_len.clear(); P->kv_len.clear();
   P->units.clear(); P->cta_unit_off.clear(); P->cta_head.clear(); P->item_rows.clear(); P->rowkv_part_off.clear();
-  P->q_tiles.clear(); P->kv_ranges.clear(); P->page_tab.clear();
+  P->q_tiles.clear(); P->kv_ranges.clear(); P->page_tab.clear(); P->k_tiles.clear(); P->q_ranges.clear();
   P->stages.clear();
   mv_plan_stats S{};
   S.n_nodes = n_nodes;
@@ -435,6 +435,30 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
           P->q_tiles.push_back(qt);
         }
       }
+      // the transposed lists of the backward pass: per 128-key tile of node u, the runs of queries that see it
+      for (int u = 0; u < n; ++u) {
+        const int32_t len_u = b->node_new[lo + u];
+        if (len_u == 0) continue;
+        const int32_t u_start = int32_t(node_tok_start[lo + u]);
+        std::vector<KvRange> seers;  // whole nodes that see u, in flattened order, adjacent ones merged
+        for (int v = 0; v < n; ++v) {
+          if (v == u || !vis.get(v, u) || b->node_new[lo + v] == 0) continue;
+          const int32_t vs = int32_t(node_tok_start[lo + v]), vl = b->node_new[lo + v];
+          if (!seers.empty() && seers.back().kv_start + seers.back().kv_len == vs) seers.back().kv_len += vl;
+          else seers.push_back(KvRange{vs, vl, 0, 0});
+        }
+        for (int32_t k0 = 0; k0 < len_u; k0 += mv::kPrefillQTile) {
+          QTile kt{};
+          kt.q_start = u_start + k0;
+          kt.q_len = std::min<int32_t>(mv::kPrefillQTile, len_u - k0);
+          kt.causal_base = kt.q_start;
+          kt.range_begin = int32_t(P->q_ranges.size());
+          P->q_ranges.push_back(KvRange{u_start + k0, len_u - k0, 1, 0});  // own node: the queries from the tile's first key on
+          for (const KvRange& r : seers) P->q_ranges.push_back(r);
+          kt.range_count = int32_t(P->q_ranges.size()) - kt.range_begin;
+          P->k_tiles.push_back(kt);
+        }
+      }
     }
   }
 
@@ -560,6 +584,16 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
     for (int32_t i : order) sorted.push_back(P->q_tiles[i]);
     P->q_tiles.swap(sorted);
     if (prefill_ready) {
+      std::vector<int64_t> kcost(P->k_tiles.size(), 0);
+      for (size_t i = 0; i < P->k_tiles.size(); ++i)
+        for (int k = 0; k < P->k_tiles[i].range_count; ++k) kcost[i] += P->q_ranges[P->k_tiles[i].range_begin + k].kv_len;
+      std::vector<int32_t> korder(P->k_tiles.size());
+      std::iota(korder.begin(), korder.end(), 0);
+      std::stable_sort(korder.begin(), korder.end(), [&](int32_t a, int32_t c) { return kcost[a] > kcost[c]; });
+      std::vector<QTile> ksorted;
+      ksorted.reserve(korder.size());
+      for (int32_t i : korder) ksorted.push_back(P->k_tiles[i]);
+      P->k_tiles.swap(ksorted);
       S.n_q_tiles = int64_t(P->q_tiles.size());
       S.visible_pairs = visible_pairs;
       S.tile_pairs = tile_pairs;
@@ -596,6 +630,8 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   L.q_tiles = place(P->q_tiles.size() * sizeof(QTile));
   L.kv_ranges = place(P->kv_ranges.size() * sizeof(KvRange));
   L.page_tab = place(P->page_tab.size() * sizeof(int32_t));
+  L.k_tiles = place(P->k_tiles.size() * sizeof(QTile));
+  L.q_ranges = place(P->q_ranges.size() * sizeof(KvRange));
   L.total = std::max<size_t>(off, 256);
   P->layout = L;
   P->valid = true;

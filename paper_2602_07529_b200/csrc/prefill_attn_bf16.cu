@@ -228,14 +228,13 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
 namespace mv {
 mv_status prefill_f32(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out,
                       cudaStream_t st);
-mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out, cudaStream_t st);
+mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out, float* lse,
+                     cudaStream_t st);
 }
 
 extern "C" mv_status mv_dag_prefill_attn(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_rot,
                                          const void* v, void* out, void* workspace, size_t workspace_bytes,
                                          void* cuda_stream) {
-  (void)workspace;
-  (void)workspace_bytes;
   if (!P || !P->valid) return MV_ERR_INVALID_ARG;
   mv_status st = mv::check_geom(g);
   if (st != MV_OK) return st;
@@ -243,10 +242,18 @@ extern "C" mv_status mv_dag_prefill_attn(const mv_plan* P, const mv_attn_geom* g
   if (!q_rot || !k_rot || !v || !out) return MV_ERR_INVALID_ARG;
   if (!P->device_buf) return MV_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  if (g->dtype == MV_F32) return mv::prefill_f32(P, g, q_rot, k_rot, v, out, s);
   // head_dim 128 with an even group size runs on tcgen05 (two heads of a KV head per CTA); TMA needs 16-byte
-  // aligned tensors.  Everything else takes the mma.sync kernel below.
+  // aligned tensors.  Everything else takes the float32 kernel or the mma.sync kernel below.
   const bool aligned = ((reinterpret_cast<uintptr_t>(q_rot) | reinterpret_cast<uintptr_t>(k_rot) | reinterpret_cast<uintptr_t>(v)) & 15) == 0;
-  if (g->head_dim == 128 && (g->n_q_heads / g->n_kv_heads) % 2 == 0 && aligned) return mv::prefill_tc(P, g, q_rot, k_rot, v, out, s);
+  const bool tc = g->dtype == MV_BF16 && g->head_dim == 128 && (g->n_q_heads / g->n_kv_heads) % 2 == 0 && aligned;
+  // a workspace asks for the rows' log-sum-exp (what the backward pass needs); only the tcgen05 kernel writes it
+  float* lse = nullptr;
+  if (workspace) {
+    if (!tc) return MV_ERR_UNSUPPORTED;
+    if (workspace_bytes < mv_workspace_bytes(P, g, MV_OP_PREFILL_ATTN) || (reinterpret_cast<uintptr_t>(workspace) & 15) != 0) return MV_ERR_WORKSPACE;
+    lse = static_cast<float*>(workspace);
+  }
+  if (g->dtype == MV_F32) return mv::prefill_f32(P, g, q_rot, k_rot, v, out, s);
+  if (tc) return mv::prefill_tc(P, g, q_rot, k_rot, v, out, lse, s);
   return g->head_dim == 128 ? launch<128>(P, g, q_rot, k_rot, v, out, s) : launch<64>(P, g, q_rot, k_rot, v, out, s);
 }

@@ -46,6 +46,7 @@ struct PrefillArgs {
   const mv::KvRange* ranges;
   const int32_t* page_tab;  // paged form: page ids, indexed by KvRange::pages + key / 16
   bf16* out;
+  float* lse;  // optional [T][n_q_heads]: log2 of the row's softmax denominator, in the units of scale_log2 * score
   int32_t* status;
   int Hq, Hkv, G;
   float scale_log2;
@@ -364,6 +365,7 @@ __device__ __forceinline__ void softmax_group(const mv::QTile& qt, const Prefill
   if (!w.warp_wait(o_done, (j - 1) & 1)) return;
   mv::um::fence_after();
   const float inv = 1.f / l;
+  if (a.lse != nullptr && r < qt.q_len) a.lse[int64_t(qi) * a.Hq + head] = m + log2f(l);  // P_ij = 2^(scale_log2 * s_ij - lse)
   bf16* dst = a.out + (int64_t(qi) * a.Hq + head) * D;
 #pragma unroll
   for (int c = 0; c < D / 32; ++c) {
@@ -459,7 +461,8 @@ struct TcMaps {  // the tensor maps of one problem (pointers and token count rar
 
 namespace mv {
 // Tensor-core prefill for head_dim 128 and an even group size; the caller has validated the arguments.
-mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out, cudaStream_t st) {
+mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* out, float* lse,
+                     cudaStream_t st) {
   static std::atomic<uint64_t> opted_in{0};  // per device
   if (!mv::opt_in_smem(prefill_tc_kernel<false>, SMEM_BYTES, opted_in)) return MV_ERR_CUDA;
   const int64_t T = P->stats.n_new_tokens;
@@ -480,6 +483,7 @@ mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, con
   a.q_tiles = mv::table<mv::QTile>(P, P->layout.q_tiles);
   a.ranges = mv::table<mv::KvRange>(P, P->layout.kv_ranges);
   a.out = static_cast<bf16*>(out);
+  a.lse = lse;
   a.status = const_cast<int32_t*>(mv::table<int32_t>(P, P->layout.sched)) + 2;
   a.page_tab = nullptr;
   a.Hq = g->n_q_heads;
@@ -521,6 +525,7 @@ mv_status append_tc(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, 
   a.ranges = mv::table<mv::KvRange>(P, P->layout.kv_ranges);
   a.page_tab = mv::table<int32_t>(P, P->layout.page_tab);
   a.out = static_cast<bf16*>(out);
+  a.lse = nullptr;
   a.status = const_cast<int32_t*>(mv::table<int32_t>(P, P->layout.sched)) + 2;
   a.Hq = g->n_q_heads;
   a.Hkv = g->n_kv_heads;

@@ -131,8 +131,19 @@ class PrefillState:
         self.k_rot = torch.empty_like(self.k)
         self.out = torch.empty_like(self.q)
 
-    def step(self, stream=None):
+    def step(self, stream=None, lse=None):
         B.mv_rope_write_kv(self.plan, self.geom, self.q, self.k, self.v, self.q_rot, self.k_rot,
                            self.k_pages if self.with_pool else None, self.v_pages if self.with_pool else None, stream)
-        B.mv_dag_prefill_attn(self.plan, self.geom, self.q_rot, self.k_rot, self.v, self.out, None, stream)
+        B.mv_dag_prefill_attn(self.plan, self.geom, self.q_rot, self.k_rot, self.v, self.out, lse, stream)
         return self.out
+
+    def forward_backward(self, dout, stream=None):
+        """Forward with the rows' log-sum-exp kept, then mv_dag_prefill_attn_bwd.  Returns (out, dq_rot, dk_rot, dv)."""
+        if not hasattr(self, "lse"):
+            self.lse = _dev_bytes(self.plan.workspace_bytes(self.geom, B.OP_PREFILL_ATTN), self.device)
+            self.bwd_ws = _dev_bytes(self.plan.workspace_bytes(self.geom, B.OP_PREFILL_ATTN_BWD), self.device)
+            self.dq, self.dk, self.dv = torch.empty_like(self.q), torch.empty_like(self.k), torch.empty_like(self.v)
+        self.step(stream, self.lse)
+        B.mv_dag_prefill_attn_bwd(self.plan, self.geom, self.q_rot, self.k_rot, self.v, self.out, dout, self.lse, self.dq, self.dk,
+                                  self.dv, self.bwd_ws, stream)
+        return self.out, self.dq, self.dk, self.dv

@@ -457,3 +457,71 @@ def test_append_refuses_nodes_that_see_each_other():
     with pytest.raises(ValueError):
         O.append_request(b, 0, _rand((5, 4, 16), 1), _rand((10, 2, 16), 2), _rand((10, 2, 16), 3))
 
+
+
+# ------------------------------------------------------------------ backward pass pins
+
+def _loss(q, k, v, allow, w):
+    return float((O.masked_attention(q, k, v, allow) * w).sum())
+
+
+def test_backward_matches_central_finite_differences():
+    """d(sum(O * W)) / d(q, k, v) from masked_attention_backward against central differences of the FORWARD on a DAG mask
+    (two q-heads per KV head, so the sum over the group is exercised; a dropped softmax-Jacobian term, a missing scale or
+    a transposed operand shows up here)."""
+    reqs = [[([], 0, 3), ([0], 0, 2), ([0], 0, 3), ([1, 2], 0, 2)]]
+    b = _mk(reqs)
+    lo, hi, parents, layer, vis, tot, start = O._request_layout(b, 0)
+    tok_node = [n for n, l in enumerate(tot) for _ in range(l)]
+    tok_index = [t for l in tot for t in range(l)]
+    allow = O.allowed_mask(tok_node, tok_index, vis)
+    T, Hq, Hkv, d = 10, 4, 2, 6
+    rng = np.random.default_rng(3)
+    q, k, v, w = (rng.standard_normal(s) for s in ((T, Hq, d), (T, Hkv, d), (T, Hkv, d), (T, Hq, d)))
+    dq, dk, dv = O.masked_attention_backward(q, k, v, allow, w)
+    eps = 1e-6
+    for name, x, g in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        num = np.zeros_like(x)
+        it = np.nditer(x, flags=["multi_index"])
+        for _ in it:
+            i = it.multi_index
+            old = x[i]
+            x[i] = old + eps
+            up = _loss(q, k, v, allow, w)
+            x[i] = old - eps
+            dn = _loss(q, k, v, allow, w)
+            x[i] = old
+            num[i] = (up - dn) / (2 * eps)
+        assert max_abs(g, num) < 1e-7, name
+
+
+def test_backward_linear_chain_equals_autograd_of_causal_sdpa():
+    T, Hq, Hkv, d = 23, 4, 2, 16
+    b = _mk([[([], 0, 9), ([0], 0, 6), ([1], 0, 8)]])
+    q, k, v, w = _rand((T, Hq, d), 40), _rand((T, Hkv, d), 41), _rand((T, Hkv, d), 42), _rand((T, Hq, d), 43)
+    dq, dk, dv = O.prefill_backward_request(b, 0, q, k, v, w)
+    pos = np.arange(T)
+    qt = torch.from_numpy(O.rope_rotate(q, pos)).requires_grad_(True)
+    kt = torch.from_numpy(O.rope_rotate(k, pos)).requires_grad_(True)
+    vt = torch.from_numpy(np.asarray(v, np.float64)).requires_grad_(True)
+    G = Hq // Hkv
+    o = torch.nn.functional.scaled_dot_product_attention(qt.permute(1, 0, 2)[None], kt.permute(1, 0, 2)[None].repeat_interleave(G, dim=1),
+                                                         vt.permute(1, 0, 2)[None].repeat_interleave(G, dim=1), is_causal=True)
+    (o[0].permute(1, 0, 2) * torch.from_numpy(np.asarray(w, np.float64))).sum().backward()
+    assert max_abs(dq, qt.grad.numpy()) < 1e-10
+    assert max_abs(dk, kt.grad.numpy()) < 1e-10
+    assert max_abs(dv, vt.grad.numpy()) < 1e-10
+
+
+def test_backward_siblings_get_no_gradient_from_a_branch():
+    """Output gradient on one branch only: the keys and values of its siblings (and of the join that comes later) get
+    exactly zero; the prefix gets some."""
+    wl = synth.config1()
+    b = batch_dict(wl.batch)
+    vals = synth.request_values(wl, 0)
+    w = np.zeros_like(vals["q"])
+    w[128:160] = _rand((32, 4, 64), 50)          # branch 1 occupies tokens 128..159
+    dq, dk, dv = O.prefill_backward_request(b, 0, vals["q"], vals["k"], vals["v"], w)
+    assert np.all(dk[160:] == 0) and np.all(dv[160:] == 0)
+    assert np.abs(dk[:128]).max() > 0 and np.abs(dv[128:160]).max() > 0
+    assert np.all(dq[:128] == 0) and np.all(dq[160:] == 0)
