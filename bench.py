@@ -38,12 +38,15 @@ import numpy as np
 METRIC = "dag_decode_attn_query_tokens_per_s"
 UNIT = "query-tokens/s"
 MIN_LEG_SECONDS = 0.5
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the leg's dominant kernel, per workload, with the
-# summary under profiles/ that holds the capture (None where the kernel has no capture of its own; see "scaled").
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the leg's dominant kernel (decode_tc_kernel), per workload,
+# with the summary under profiles/ that holds the capture.  The serving mix holds too much memory for a counter capture
+# (the profiling rule keeps those to a few GB): its figure is the layered-DAG capture scaled by the algorithmic bytes
+# (traffic is 1.0 % above them there: partials and plan tables, which grow with the stream).
 NCU_TRAFFIC = {
-    "config2": {"bytes": 210_300_000, "kernel": "decode_tc_kernel", "profile": "profiles/decode_tc_kernel_config2.md"},
-    "config3": {"bytes": None, "kernel": "decode_tc_kernel", "profile": "profiles/decode_tc_kernel_config3.md"},
-    "config5": {"bytes": None, "kernel": "decode_tc_kernel", "profile": None},
+    "config2": {"bytes": 210_100_000, "kernel": "decode_tc_kernel", "profile": "profiles/decode_tc_kernel_config2.md"},
+    "config3": {"bytes": 801_500_000, "kernel": "decode_tc_kernel", "profile": "profiles/decode_tc_kernel_config3.md"},
+    "config5": {"bytes": 3_944_000_000, "kernel": "decode_tc_kernel",
+                "profile": "profiles/decode_tc_kernel_config3.md (scaled by algorithmic bytes, 3904.4 / 793.4 MB)"},
 }
 BF16_TOL = (2e-2, 1e-2)   # max-abs, relative L2 against the float64 oracle
 F32_TOL = 1e-4
@@ -227,8 +230,9 @@ def _median_launch_ms(torch, fn, warmup=5, min_launches=20, min_seconds=None, ma
     return float(np.median(times)), float(np.min(times)), len(times), float(np.median(times[:min_launches]))
 
 
-def _decode_parity(wl, got, requests):
-    """The step's output rows of the listed requests against the oracle: (max-abs, relative L2, rows checked)."""
+def _decode_parity(wl, got, requests, heads=None):
+    """The step's output rows of the listed requests against the oracle: (max-abs, relative L2, rows checked).  ``heads``:
+    the (first query head, query heads, ...) slice the output holds when the run is sharded by KV head."""
     from oracle import medverse_oracle as O
     from paper_2602_07529_b200 import synth
     b = _batch_dict(wl.batch)
@@ -240,7 +244,7 @@ def _decode_parity(wl, got, requests):
     for r in requests:
         vals = synth.request_values(wl, r)
         o = O.decode_request(b, r, vals["q"], vals["k"], vals["v"], base=wl.geom.rope_base)
-        w.append(o)
+        w.append(o if heads is None else o[:, heads[0]:heads[0] + heads[1]])
         g.append(got[first[r]:first[r] + o.shape[0]])
     g, w = np.concatenate(g, 0), np.concatenate(w, 0)
     err, rel = _bf16_err(g, w)
@@ -268,13 +272,16 @@ def _parity_requests(wl, how_many):
 class DecodeLeg:
     """One decode workload resident on the device, with what its timed loops need marshalled once."""
 
-    def __init__(self, torch, wl, dev, chunk=0):
+    def __init__(self, torch, wl, dev, chunk=0, heads=None):
         from paper_2602_07529_b200 import binding as B, runtime
         self.torch, self.B, self.wl, self.dev = torch, B, wl, dev
         g, b = wl.geom, wl.batch
+        if heads is not None:   # this rank's slice of the KV heads (sharding by KV head)
+            g = dataclasses.replace(g, n_q_heads=heads[1], n_kv_heads=heads[3])
+        self.geom_local, self.heads = g, heads
         self.pool_bytes = 2 * b.num_pages * g.n_kv_heads * g.page_size * g.head_dim * 2
         self.n_pools = max(2, min(8, int(np.ceil(1.0e9 / self.pool_bytes))))
-        self.st = runtime.DecodeState(wl, dev, chunk_tokens=chunk, n_pool_copies=self.n_pools)
+        self.st = runtime.DecodeState(wl, dev, chunk_tokens=chunk, n_pool_copies=self.n_pools, heads=heads)
         st = self.st
         self.stats = st.plan.stats()
         self.rows = self.stats["n_new_tokens"]
@@ -296,7 +303,7 @@ class DecodeLeg:
         # every pointer the timed loop passes is fixed: marshal them once, so that the host side of a step is the
         # library calls themselves (a C caller has no per-call marshalling either)
         self.cb = self.plans[0].c_batch
-        self.gref, self.cbref = C.byref(st.geom), C.byref(self.cb)
+        self.gref, self.cbref, self.tref = C.byref(st.geom), C.byref(self.cb), C.byref(self.plans[0].c_tuning)
         self.plan_refs = [C.byref(p._h) for p in self.plans]
         self.tab_ptr = [vp_(t.data_ptr()) for t in self.tables]
         self.tab_len = [t.numel() for t in self.tables]
@@ -310,7 +317,7 @@ class DecodeLeg:
         lib, s = self.lib, i % self.RING
         self.ring_ev[s].synchronize()
         h = self.plans[s]._h
-        rc = lib.mv_plan_dag(self.cbref, self.plan_refs[s])
+        rc = lib.mv_plan_dag(self.cbref, self.gref, self.tref, self.plan_refs[s])
         rc |= lib.mv_plan_upload(h, self.tab_ptr[s], self.tab_len[s], self.csp)
         self.up_ev[s].record(self.copy_stream)
         self.stream.wait_event(self.up_ev[s])
@@ -378,11 +385,11 @@ class DecodeLeg:
     def parity(self, how_many):
         self.torch.cuda.synchronize()
         got = self.st.out.float().cpu().numpy()
-        return _decode_parity(self.wl, got, _parity_requests(self.wl, how_many))
+        return _decode_parity(self.wl, got, _parity_requests(self.wl, how_many), self.heads)
 
     def rope_leg(self, peaks):
         """mv_rope_write_kv alone on this step's new tokens (read q, k, v; write q_rot and the K / V pool slots)."""
-        g, st = self.wl.geom, self.st
+        g, st = self.geom_local, self.st
         n = self.rows
         nbytes = 2 * n * (g.n_q_heads + 2 * g.n_kv_heads) * g.head_dim * 2
         def call(i):
@@ -431,9 +438,15 @@ def run_ours(args):
     region = Region(sampler)
 
     # ---- headline: the decode step on the named workload
-    wl = _workload(args.workload, rank)
-    leg = DecodeLeg(torch, wl, dev, args.chunk)
-    g, b, rows, stats = wl.geom, wl.batch, leg.rows, leg.stats
+    by_heads = args.shard == "heads" and world > 1
+    heads = None
+    if by_heads:   # every rank takes the same batch and a slice of its KV heads (with their query heads and pools)
+        wl = _workload(args.workload, 0)
+        heads = multirank.head_slice(wl.geom.n_q_heads, wl.geom.n_kv_heads, rank, world)
+    else:
+        wl = _workload(args.workload, rank)
+    leg = DecodeLeg(torch, wl, dev, args.chunk, heads)
+    g, b, rows, stats = leg.geom_local, wl.batch, leg.rows, leg.stats
     K, W = args.steps, max(args.warmup, 3)
     launches0 = B.mv_launch_count()
     reps = leg.timed_steps(K, W, barrier, region, agree)
@@ -442,6 +455,8 @@ def run_ours(args):
     order = np.argsort([r[0] for r in reps])
     med = reps[int(order[len(order) // 2])]
     total_ms, job_rows = multirank.reduce_job(med[0], rows * K, dist, dev)
+    if by_heads:
+        job_rows = rows * K    # every rank computed (its heads of) the same rows
     calls = np.concatenate([r[1] for r in reps])
     decode_ms, decode_ms_min = float(np.mean(calls)), float(np.min(calls))
 
@@ -482,6 +497,21 @@ def run_ours(args):
                 n_e2e = agree(int(min(100, max(1, np.ceil(MIN_LEG_SECONDS / max(e2e_reps[0][0] * 1e-3, 1e-6))))))
     e2e_med = sorted(e2e_reps)[len(e2e_reps) // 2]
     e2e_ms, e2e_rows = multirank.reduce_job(e2e_med[0], rows * Ke, dist, dev)
+    if by_heads:
+        e2e_rows = rows * Ke
+    # sharding by KV head: the all-gather that puts the ranks' output slices together stands outside the path (the output
+    # projection can consume the slices where they are); timed on its own, after the timed steps
+    gather_ms = None
+    if by_heads:
+        multirank.gather_heads(st.out, dist)
+        barrier()
+        ga, gc = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ga.record(stream)
+        for _ in range(20):
+            full_out = multirank.gather_heads(st.out, dist)
+        gc.record(stream)
+        barrier()
+        gather_ms, _ = multirank.reduce_job(ga.elapsed_time(gc) / 20, 0, dist, dev)
     same = bool(torch.equal(oh, st.out.cpu()))   # the e2e output equals the device-path output bit for bit
     h2d = int(leg.plans[0].device_bytes() + qh.numel() * 2 + kh.numel() * 2 + vh.numel() * 2)
     d2h = int(oh.numel() * 2)
@@ -490,7 +520,7 @@ def run_ours(args):
     n_plan = 200 if stats["n_new_tokens"] < 200 else 50
     t0 = time.perf_counter()
     for _ in range(n_plan):
-        B.lib.mv_plan_dag(leg.cbref, leg.plan_refs[1])
+        B.lib.mv_plan_dag(leg.cbref, leg.gref, leg.tref, leg.plan_refs[1])
     planner_us = 1e6 * (time.perf_counter() - t0) / n_plan
     burst_ms = leg.burst_ms()
 
@@ -512,7 +542,7 @@ def run_ours(args):
            "sample": f"{n_req} whole request(s) = {n_rows} of {rows} rows of {wl.name}, {t_used:.1f} s, float64 numpy"}
     line = {
         "metric": METRIC, "value": job_rows / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
-        "warmup": W, "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "warmup": W, "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "strong" if by_heads else "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "requests": int(b.n_req), "rows": int(rows), "n_q_heads": g.n_q_heads,
                    "n_kv_heads": g.n_kv_heads, "head_dim": g.head_dim, "page_size": g.page_size,
@@ -522,7 +552,9 @@ def run_ours(args):
                    "l2": f"steps rotate over {leg.n_pools} independent KV pool copies ({leg.n_pools * leg.pool_bytes / 1e9:.2f} GB in total, "
                          f"{leg.algo_bytes / 1e6:.0f} MB read per step) so every step streams from HBM",
                    "step": "mv_plan_dag + mv_plan_upload (copy stream) + mv_rope_write_kv + mv_dag_decode_attn",
-                   "parallelism": (f"{world} ranks, one batch each, sharded by request, no collective" if world > 1 else "single")},
+                   "parallelism": ((f"{world} ranks, one batch, sharded by KV head ({g.n_kv_heads} KV heads and {g.n_q_heads} query heads per rank), "
+                                    "no collective on the path; NCCL all-gather of the output timed separately") if by_heads else
+                                   (f"{world} ranks, one batch each, sharded by request, no collective" if world > 1 else "single"))},
         "roofline": leg.roofline(decode_ms, decode_ms_min, peaks, args.workload),
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_rows / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -532,6 +564,7 @@ def run_ours(args):
         "gpu_launches": int(3 * K),
         "gpu_launches_all_repeats": int(launches_all),
         "planner_us": planner_us,
+        "all_gather_out_ms": gather_ms,
         "decode_burst_ms": burst_ms,
         "clocks": sampler.summary(),
         "parity": parity,
@@ -578,10 +611,10 @@ def _legs(torch, B, runtime, synth, dev, peaks, region, barrier, args, headline_
         del leg
         torch.cuda.empty_cache()
     with region:
-        legs["prefill"], legs["rope_write_kv_config4"], p4 = _prefill_leg(torch, B, runtime, synth, dev, peaks)
+        legs["prefill"], legs["rope_write_kv_config4"], p4, (legs["prefill_backward"], pb) = _prefill_leg(torch, B, runtime, synth, dev, peaks)
         legs["append"], pa = _append_leg(torch, B, runtime, synth, dev, peaks)
         legs["prefill_config1_f32"], p1 = _config1_leg(torch, B, runtime, synth, dev)
-    parity["prefill_config4"], parity["append"], parity["prefill_config1"] = p4, pa, p1
+    parity["prefill_config4"], parity["append"], parity["prefill_config1"], parity["prefill_backward_config4"] = p4, pa, p1, pb
     return legs, parity
 
 
@@ -634,7 +667,50 @@ def _prefill_leg(torch, B, runtime, synth, dev, peaks):
             "bytes_note": "read q, k, v; write q_rot, k_rot and the K / V pool slots (one more K write than the 2*n*(Hq+2Hkv)*d*B figure)",
             "GBs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0,
             "q_rot_max_abs_vs_oracle": qerr, "ok": bool(qerr <= 2.0 ** -8 * 6)}
-    return prefill, rope, parity
+    return prefill, rope, parity, _backward_leg(torch, B, O, synth, st, wl, flops, peaks)
+
+
+def _backward_leg(torch, B, O, synth, st, wl, fwd_flops, peaks):
+    """mv_dag_prefill_attn_bwd on the same 17K-token DAG: useful flops are the five products of the definition over the
+    visible pairs (2.5 x the forward's); the kernels run seven (dQ and dK/dV each rebuild the scores)."""
+    g, b = wl.geom, wl.batch
+    T = st.q.shape[0]
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(7)
+    dout_h = torch.randn(T, g.n_q_heads, g.head_dim, generator=gen, dtype=torch.float32).to(torch.bfloat16)
+    dout = dout_h.to(st.q.device)
+    st.forward_backward(dout)
+    ms, ms_min, launches, ms20 = _median_launch_ms(torch, lambda i: B.mv_dag_prefill_attn_bwd(
+        st.plan, st.geom, st.q_rot, st.k_rot, st.v, st.out, dout, st.lse, st.dq, st.dk, st.dv, st.bwd_ws), min_launches=10)
+    flops = 2.5 * fwd_flops
+    tf, tf20 = flops / (ms * 1e-3) / 1e12, flops / (ms20 * 1e-3) / 1e12
+    leg = {"workload": wl.name, "tokens": int(T), "ms": ms, "ms_min": ms_min, "launches": launches, "kernels_per_call": 3,
+           "useful_tflops": tf, "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+           "ms_first_launches": ms20, "useful_tflops_first_launches": tf20, "frac_of_measured_bf16_peak": tf20 / peaks["bf16_tflops"],
+           "executed_over_useful": 7.0 / 5.0}
+    # parity through linearity (the dense oracle over 17K x 17K pairs does not fit): one more call with an output gradient
+    # that is nonzero on a few sampled rows; dQ there, and dK / dV everywhere, against the oracle on those rows alone
+    rows = sorted({0, 128, 4095, 4096, T - 1, T - 513} | {int(x) for x in np.random.default_rng(12).choice(T, size=18, replace=False)})
+    sparse = torch.zeros_like(dout_h)
+    sparse[rows] = dout_h[rows]
+    st.forward_backward(sparse.to(st.q.device))
+    torch.cuda.synchronize()
+    bd = _batch_dict(b)
+    lo, hi, parents, layer, vis, tot, start = O._request_layout(bd, 0)
+    tok_node = [n for n, l in enumerate(tot) for _ in range(l)]
+    tok_index = [t for l in tot for t in range(l)]
+    pos = np.asarray([start[n] + t for n, l in enumerate(tot) for t in range(l)], np.int64)
+    vals = synth.request_values(wl, 0)
+    wq, wk, wv = O.masked_attention_backward(O.rope_rotate(vals["q"][rows], pos[rows], g.rope_base), O.rope_rotate(vals["k"], pos, g.rope_base),
+                                             vals["v"], O.allowed_mask(tok_node, tok_index, vis, rows), sparse.float().numpy()[rows])
+    errs = {}
+    ok = True
+    for name, got, want in (("dq", st.dq.float().cpu().numpy()[rows], wq), ("dk", st.dk.float().cpu().numpy(), wk), ("dv", st.dv.float().cpu().numpy(), wv)):
+        err, rel = _bf16_err(got, want)
+        errs[name] = {"max_abs": err, "rel_l2": rel}
+        ok = ok and rel <= BF16_TOL[1] and err <= BF16_TOL[0] * max(1.0, float(np.abs(want).max()))
+    errs.update({"rows": len(rows), "ok": bool(ok), "how": "linearity: output gradient nonzero on sampled rows only"})
+    return leg, errs
 
 
 def _append_leg(torch, B, runtime, synth, dev, peaks, new_tokens=128):
@@ -706,6 +782,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config5", choices=["config2", "config3", "config5"])
     ap.add_argument("--chunk", type=int, default=0, help="decode split-KV chunk tokens (0 = automatic)")
+    ap.add_argument("--shard", default="requests", choices=["requests", "heads"],
+                    help="N > 1: every rank its own batch (requests, weak scaling) or one batch cut by KV head (heads, strong scaling)")
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for the CPU baseline")
     ap.add_argument("--no-legs", "--no-prefill", dest="no_legs", action="store_true", help="headline workload only")
     ap.add_argument("--min-seconds", type=float, default=MIN_LEG_SECONDS,

@@ -85,15 +85,6 @@ typedef struct {
   int32_t page_size;         /* 16 */
   int32_t vis_mode;          /* mv_vis_mode */
   int32_t pos_mode;          /* mv_pos_mode */
-  int32_t chunk_tokens;      /* decode: longest KV slice of one work unit in tokens (multiple of page_size);
-                                0 = no limit (slices are cut only where a CTA's equal share of the step ends)  */
-  int32_t n_kv_heads;        /* scheduling: KV heads of the geometry the plan will run with (0 = 8);
-                                mv_dag_decode_attn returns MV_ERR_UNSUPPORTED for any other head count         */
-  int32_t group_size;        /* scheduling: n_q_heads / n_kv_heads (0 = 8).  A node's row set is split so
-                                that rows * group_size <= 64; mv_dag_decode_attn returns MV_ERR_UNSUPPORTED if
-                                the geometry's real group size breaks that bound                               */
-  int32_t sched_ctas;        /* scheduling: CTAs the decode kernel runs with (0 = 296, two per SM of a 148-SM
-                                part); the step's KV stream is cut into that many equal shares                 */
 } mv_dag_batch;
 
 typedef struct {
@@ -103,6 +94,14 @@ typedef struct {
   float sm_scale;      /* softmax scale; 0 means 1/sqrt(head_dim) */
   double rope_base;    /* theta_i = rope_base^(-2i/head_dim) */
 } mv_attn_geom;
+
+/* Optional tuning of the decode work lists (all zero = the defaults). */
+typedef struct {
+  int32_t chunk_tokens;      /* longest KV slice of one work unit in tokens (multiple of page_size);
+                                0 = no limit (slices are cut only where a CTA's equal share of the step ends)  */
+  int32_t sched_ctas;        /* shares the step's KV stream is cut into = half-CTAs the decode kernel runs with
+                                (0 = 296, two per SM of a 148-SM part)                                         */
+} mv_plan_tuning;
 
 typedef struct mv_plan mv_plan;
 
@@ -145,7 +144,7 @@ typedef struct {
                                   rounded up to whole 128x64 tiles                                         */
   int64_t max_page_id;         /* largest page id referenced                                                */
   int64_t max_item_rows;       /* decode: largest row set of a work item                                    */
-  int64_t sched_kv_heads, sched_group; /* the scheduling hints in effect                                    */
+  int64_t sched_kv_heads, sched_group; /* head counts the decode work lists were cut for (0: no geometry yet) */
   int64_t n_ctas;              /* decode: CTAs the step was cut for                                         */
   int64_t max_cta_cost;        /* decode: largest share handed to one CTA, in tokens of one KV head (a unit
                                   counts as its tokens + 48)                                                */
@@ -158,13 +157,24 @@ enum { MV_OP_ROPE_WRITE_KV = 0, MV_OP_DECODE_ATTN = 1, MV_OP_PREFILL_ATTN = 2, M
 
 /* DAG -> segment planner (Eq. 1 layering; Eq. 3 / Sec. 4.3 visibility; Sec. 4.2 positions; Sec. 3.2 KV index
  * lists).  Host only, integers only, deterministic.
- *   batch  host, read during the call only.
+ *   batch  host, read during the call only: the paper-level description of the step, nothing else.
+ *   geom   host, optional.  The canonical tables, mv_rope_write_kv and the prefill calls need no geometry.  The decode
+ *          kernels' work lists are cut for a head count (units are per KV head; a node's rows are grouped so that
+ *          rows * group size <= 64), so only n_q_heads and n_kv_heads are read.  With geom == NULL the plan keeps a copy
+ *          of the batch instead and mv_plan_bind_geometry cuts the lists later, for any supported geometry; until then
+ *          mv_dag_decode_attn returns MV_ERR_UNSUPPORTED.
+ *   tuning host, optional (NULL = defaults).
  *   plan   in/out: if *plan is NULL a new plan is created; otherwise the existing plan is re-planned in
  *          place and its host buffers are reused (no allocation once they are large enough).  The caller
  *          must not re-plan while an mv_plan_upload of the same plan is still in flight on a stream.
- * Errors: MV_ERR_INVALID_ARG, MV_ERR_NOT_TOPOLOGICAL, MV_ERR_PAGE_CAPACITY.  On error *plan is unchanged
- * if it was NULL and left in an unusable-but-destroyable state otherwise. */
-mv_status mv_plan_dag(const mv_dag_batch* batch, mv_plan** plan);
+ * Errors: MV_ERR_INVALID_ARG, MV_ERR_NOT_TOPOLOGICAL, MV_ERR_PAGE_CAPACITY, MV_ERR_UNSUPPORTED (head counts).  On
+ * error *plan is unchanged if it was NULL and left in an unusable-but-destroyable state otherwise. */
+mv_status mv_plan_dag(const mv_dag_batch* batch, const mv_attn_geom* geom, const mv_plan_tuning* tuning, mv_plan** plan);
+
+/* Cuts (or re-cuts) the decode work lists of a plan that was made without a geometry, for `geom`'s head counts.  The
+ * plan's canonical tables do not change; its device tables do: upload it again before the next kernel call.
+ * Errors: MV_ERR_INVALID_ARG, MV_ERR_UNSUPPORTED (the plan was made with a geometry and kept no copy of its batch). */
+mv_status mv_plan_bind_geometry(mv_plan* plan, const mv_attn_geom* geom, const mv_plan_tuning* tuning);
 
 /* Canonical table access for parity checks.  *host_ptr points into the plan; *count is in elements. */
 mv_status mv_plan_table(const mv_plan* plan, int which, const void** host_ptr, int64_t* count);

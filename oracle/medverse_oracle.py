@@ -423,3 +423,58 @@ def prefill_backward_request(batch, r, q_raw, k_raw, v, dout, base=10000.0, scal
     qr = rope_rotate(q_raw, pos, base)
     kr = rope_rotate(k_raw, pos, base)
     return masked_attention_backward(qr, kr, v, allow, dout, scale)
+
+
+# ----------------------------------------------------------------------------- FP8 (e4m3) KV cache variant
+# Not in the paper: a storage format for the cache that halves the bytes a decode step streams.  K (position-embedded)
+# and V are stored as 8-bit floats with 4 exponent and 3 mantissa bits (the "e4m3" format of the OCP 8-bit floating
+# point specification: bias 7, no infinities, largest finite value 448, subnormals down to 2^-9), divided by one scale
+# per KV head: stored = round_e4m3(x / scale[head]), saturating at +-448; the attention then runs on stored * scale.
+
+E4M3_MAX = 448.0
+
+
+def round_e4m3(x):
+    """Round to the nearest e4m3 value (ties to even), saturating at +-448; returns float64 holding e4m3-representable
+    values.  Written from the format's definition: for |x| in [2^e, 2^(e+1)), e in [-6, 8], the spacing is 2^(e-3);
+    below 2^-6 (subnormals) the spacing is 2^-9."""
+    x = np.asarray(x, np.float64)
+    a = np.minimum(np.abs(x), E4M3_MAX)
+    e = np.floor(np.log2(np.maximum(a, 2.0 ** -6)))          # exponent of the binade (subnormals share the lowest one)
+    step = 2.0 ** (e - 3)
+    q = np.round(a / step) * step                             # numpy rounds half to even
+    q = np.minimum(q, E4M3_MAX)
+    return np.sign(x) * q
+
+
+def quantise_kv_e4m3(x, scale):
+    """x [T, Hkv, d] -> the values the FP8 cache holds, already multiplied back by the per-head scale [Hkv]."""
+    s = np.asarray(scale, np.float64)[None, :, None]
+    return round_e4m3(np.asarray(x, np.float64) / s) * s
+
+
+def decode_request_fp8(batch, r, q_raw, k_raw, v, k_scale, v_scale, base=10000.0, scale=None, rows=None):
+    """``decode_request`` with the cache in the FP8 format: every key is position-embedded (float64 RoPE on the given
+    values), rounded to float32 (the precision the rotation is carried out in), quantised with ``k_scale`` and read back;
+    every value is quantised with ``v_scale``.  Queries are not quantised here (what a kernel does to them internally is
+    covered by the tolerance)."""
+    lo, hi, parents, layer, vis, tot, start = _request_layout(batch, r)
+    tok_off = np.concatenate([[0], np.cumsum(tot)]).astype(np.int64)
+    frontier = [vl for vl in range(hi - lo) if int(batch["node_new"][lo + vl]) > 0]
+    q_raw = np.asarray(q_raw)
+    out = np.full((len(frontier), q_raw.shape[1], q_raw.shape[2]), np.nan, np.float64)
+    for ri, vl in enumerate(frontier):
+        if rows is not None and ri not in rows:
+            continue
+        ks, vs, pos = [], [], []
+        for u in vis[vl]:
+            a, b = int(tok_off[u]), int(tok_off[u + 1])
+            ks.append(k_raw[a:b])
+            vs.append(v[a:b])
+            pos.extend(range(start[u], start[u] + (b - a)))
+        kk = rope_rotate(np.concatenate(ks, 0), pos, base).astype(np.float32)
+        kk = quantise_kv_e4m3(kk, k_scale)
+        vv = quantise_kv_e4m3(np.concatenate(vs, 0), v_scale)
+        qq = rope_rotate(q_raw[ri:ri + 1], [start[vl] + tot[vl] - 1], base)
+        out[ri] = masked_attention(qq, kk, vv, np.ones((1, kk.shape[0]), dtype=bool), scale)[0]
+    return out

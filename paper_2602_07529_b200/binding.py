@@ -25,7 +25,7 @@ TABLES = {"layer": (0, np.int32), "pos_start": (1, np.int32), "pos_id": (2, np.i
 # the decode kernels' work lists as int32 words (read by tests that replay them on the host)
 WORK_TABLES = {"stages": 10, "units": 11, "item_rows": 12, "cta_unit_off": 13, "rowkv_part_off": 14}
 
-EXPORTS = ["mv_plan_dag", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_bytes", "mv_plan_upload",
+EXPORTS = ["mv_plan_dag", "mv_plan_bind_geometry", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_bytes", "mv_plan_upload",
            "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
            "mv_dag_prefill_attn", "mv_dag_prefill_attn_bwd", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_decode_step_host_batch", "mv_status_string",
            "mv_launch_count", "mv_plan_read_status", "mv_dag_decode_attn_static",
@@ -43,9 +43,11 @@ class MvError(RuntimeError):
 class _DagBatch(C.Structure):
     _fields_ = [("n_req", C.c_int32), ("node_off", C.c_void_p), ("node_len", C.c_void_p), ("node_new", C.c_void_p),
                 ("parent_off", C.c_void_p), ("parent_idx", C.c_void_p), ("page_off", C.c_void_p),
-                ("page_idx", C.c_void_p), ("page_size", C.c_int32), ("vis_mode", C.c_int32), ("pos_mode", C.c_int32),
-                ("chunk_tokens", C.c_int32), ("n_kv_heads", C.c_int32), ("group_size", C.c_int32),
-                ("sched_ctas", C.c_int32)]
+                ("page_idx", C.c_void_p), ("page_size", C.c_int32), ("vis_mode", C.c_int32), ("pos_mode", C.c_int32)]
+
+
+class _Tuning(C.Structure):
+    _fields_ = [("chunk_tokens", C.c_int32), ("sched_ctas", C.c_int32)]
 
 
 class _Geom(C.Structure):
@@ -73,7 +75,8 @@ def _load():
                           "(there is no CPU fallback)")
     lib = C.CDLL(LIB_PATH)
     vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
-    lib.mv_plan_dag.argtypes = [C.POINTER(_DagBatch), C.POINTER(vp)]
+    lib.mv_plan_dag.argtypes = [C.POINTER(_DagBatch), C.POINTER(_Geom), C.POINTER(_Tuning), C.POINTER(vp)]
+    lib.mv_plan_bind_geometry.argtypes = [vp, C.POINTER(_Geom), C.POINTER(_Tuning)]
     lib.mv_plan_table.argtypes = [vp, C.c_int, C.POINTER(vp), C.POINTER(i64)]
     lib.mv_plan_get_stats.argtypes = [vp, C.POINTER(_Stats)]
     lib.mv_plan_device_bytes.argtypes = [vp]
@@ -158,23 +161,42 @@ def geom_of(workload) -> _Geom:
     return make_geom(g.n_q_heads, g.n_kv_heads, g.head_dim, workload.batch.num_pages, g.dtype, g.page_size, 0.0, g.rope_base)
 
 
-class Plan:
-    """Owner of an ``mv_plan*``.  ``Plan(batch)`` plans; ``plan.replan(batch)`` recycles the same object."""
+def _heads_geom(n_kv_heads: int, group_size: int) -> "_Geom":
+    """A geometry that carries head counts only (all mv_plan_dag reads of it)."""
+    return _Geom(int(n_kv_heads) * int(group_size), int(n_kv_heads), 128, 16, 0, MV_BF16, 0.0, 10000.0)
 
-    def __init__(self, batch=None, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0, sched_ctas: int = 0):
+
+class Plan:
+    """Owner of an ``mv_plan*``.  ``Plan(batch)`` plans; ``plan.replan(batch)`` recycles the same object.
+
+    The decode work lists are cut for a head count: give ``geom`` (a geometry struct) or ``n_kv_heads`` and
+    ``group_size``; with neither the plan has canonical tables and prefill tiles only, until ``bind_geometry``."""
+
+    def __init__(self, batch=None, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0, sched_ctas: int = 0, geom=None):
         self._h = C.c_void_p(None)
         self._keep = None
         if batch is not None:
-            self.replan(batch, chunk_tokens, n_kv_heads, group_size, sched_ctas)
+            self.replan(batch, chunk_tokens, n_kv_heads, group_size, sched_ctas, geom)
 
-    def replan(self, batch, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0, sched_ctas: int = 0):
+    def replan(self, batch, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0, sched_ctas: int = 0, geom=None):
         arrs = [_i32(getattr(batch, n)) for n in ("node_off", "node_len", "node_new", "parent_off", "parent_idx",
                                                    "page_off", "page_idx")]
         self._keep = arrs
         b = _DagBatch(int(batch.n_req), *[a.ctypes.data for a in arrs], int(batch.page_size), int(batch.vis_mode),
-                      int(batch.pos_mode), int(chunk_tokens), int(n_kv_heads), int(group_size), int(sched_ctas))
+                      int(batch.pos_mode))
         self.c_batch = b
-        _check(lib.mv_plan_dag(C.byref(b), C.byref(self._h)), "mv_plan_dag")
+        if geom is None and n_kv_heads > 0 and group_size > 0:
+            geom = _heads_geom(n_kv_heads, group_size)
+        self.c_geom = geom
+        self.c_tuning = _Tuning(int(chunk_tokens), int(sched_ctas))
+        _check(lib.mv_plan_dag(C.byref(b), C.byref(geom) if geom is not None else None, C.byref(self.c_tuning), C.byref(self._h)),
+               "mv_plan_dag")
+        return self
+
+    def bind_geometry(self, geom, chunk_tokens: int = 0, sched_ctas: int = 0):
+        """Cuts the decode work lists of a plan made without a geometry (upload the plan again afterwards)."""
+        self.c_geom, self.c_tuning = geom, _Tuning(int(chunk_tokens), int(sched_ctas))
+        _check(lib.mv_plan_bind_geometry(self._h, C.byref(geom), C.byref(self.c_tuning)), "mv_plan_bind_geometry")
         return self
 
     @property
@@ -231,8 +253,8 @@ class Plan:
             pass
 
 
-def mv_plan_dag(batch, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0, sched_ctas: int = 0) -> Plan:
-    return Plan(batch, chunk_tokens, n_kv_heads, group_size, sched_ctas)
+def mv_plan_dag(batch, chunk_tokens: int = 0, n_kv_heads: int = 0, group_size: int = 0, sched_ctas: int = 0, geom=None) -> Plan:
+    return Plan(batch, chunk_tokens, n_kv_heads, group_size, sched_ctas, geom)
 
 
 def mv_rope_write_kv(plan: Plan, geom: _Geom, q, k, v, q_rot, k_rot, k_pages, v_pages, stream=None):

@@ -98,7 +98,7 @@ extern "C" mv_status mv_decode_step_host_batch(const mv_dag_batch* batch, mv_pla
   char* base = static_cast<char*>(staging);
   // the copies travel while the host plans the step
   if (!copy_in(base, F, q_host, k_host, v_host, static_cast<cudaStream_t>(cuda_stream))) return MV_ERR_CUDA;
-  st = mv_plan_dag(batch, plan);
+  st = mv_plan_dag(batch, g, nullptr, plan);
   if (st != MV_OK) return st;
   mv_plan* P = *plan;
   if (P->stats.n_new_tokens != n) return MV_ERR_INVALID_ARG;

@@ -94,4 +94,10 @@ struct mv_plan {
   bool pinned_is_cuda = false;
   // where the last upload put the tables
   void* device_buf = nullptr;
+  // a plan made without a geometry keeps its batch, so that mv_plan_bind_geometry can cut the decode work lists later
+  struct SavedBatch {
+    bool kept = false;
+    std::vector<int32_t> node_off, node_len, node_new, parent_off, parent_idx, page_off, page_idx;
+    int32_t n_req = 0, page_size = 16, vis_mode = 0, pos_mode = 0;
+  } saved;
 };

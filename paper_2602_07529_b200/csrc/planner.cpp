@@ -45,8 +45,6 @@ mv_status check_batch(const mv_dag_batch* b) {
   if (b->page_size != 16) return MV_ERR_INVALID_ARG;
   if (b->vis_mode != MV_VIS_ANCESTORS && b->vis_mode != MV_VIS_LAYERWISE) return MV_ERR_INVALID_ARG;
   if (b->pos_mode != MV_POS_MAX_PARENT_END && b->pos_mode != MV_POS_FRONTIER_ALIGNED) return MV_ERR_INVALID_ARG;
-  if (b->chunk_tokens < 0 || (b->chunk_tokens % b->page_size) != 0) return MV_ERR_INVALID_ARG;
-  if (b->n_kv_heads < 0 || b->group_size < 0 || b->sched_ctas < 0) return MV_ERR_INVALID_ARG;
   if (b->node_off[0] != 0) return MV_ERR_INVALID_ARG;
   for (int r = 0; r < b->n_req; ++r)
     if (b->node_off[r + 1] < b->node_off[r]) return MV_ERR_INVALID_ARG;
@@ -65,10 +63,13 @@ mv_status check_batch(const mv_dag_batch* b) {
 
 }  // namespace
 
-extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
+namespace {
+// kv_heads == 0: no geometry yet (canonical tables and prefill tiles only; the decode work lists are left out)
+mv_status plan_impl(const mv_dag_batch* b, int kv_heads, int group, int chunk_tokens, int sched_ctas, mv_plan** out) {
   if (!out) return MV_ERR_INVALID_ARG;
   mv_status st = check_batch(b);
   if (st != MV_OK) return st;
+  if (chunk_tokens < 0 || (chunk_tokens % b->page_size) != 0 || sched_ctas < 0) return MV_ERR_INVALID_ARG;
 
   const int ps = b->page_size;
   const int n_nodes = b->node_off[b->n_req];
@@ -144,8 +145,8 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   std::vector<Seg>& segs = sc.segs;
   node_tok_start.assign(size_t(n_nodes), 0);  // flattened index of a node's first NEW token
   int64_t unique_tokens = 0, per_row_tokens = 0, visible_pairs = 0, tile_pairs = 0;
-  const int sched_kv_heads = b->n_kv_heads > 0 ? b->n_kv_heads : 8;
-  const int sched_group = b->group_size > 0 ? b->group_size : 8;
+  const bool cut_lists = kv_heads > 0;  // the decode work lists need the head counts
+  const int sched_kv_heads = kv_heads, sched_group = std::max(1, group);
   const int max_rows_per_item = std::max(1, 64 / sched_group);
 
   // decode streams: one per (request, row group): a run of stages and the rows of the group; cut into work
@@ -154,7 +155,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   seg_rows.clear();
   stage_plain.clear();  // per stage: four full pages seen by the whole row group
   constexpr int kStage = 64;  // tokens per stage of the decode kernel's pipeline
-  const int chunk = b->chunk_tokens;  // 0: units are cut only where a CTA's share ends
+  const int chunk = chunk_tokens;  // 0: units are cut only where a CTA's share ends
 
   int64_t new_tok_count = 0;
   for (int r = 0; r < b->n_req; ++r) {
@@ -254,7 +255,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
         if (u != v && b->node_new[lo + u] > 0 && vis.get(v, u)) decode_ready = false;
     }
     // ---- decode streams of this request: per row group, the stages of every node at least one of its rows sees
-    if (decode_ready) {
+    if (decode_ready && cut_lists) {
       req_rows.clear();  // rows of the request, ascending: one per new token, node after node
       row_node.clear();  // local node of each row
       row_tok.clear();   // which of its node's new tokens the row is
@@ -463,9 +464,9 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   }
 
   // ---- decode: cut the stream of (row-group stream, KV head) stage runs into n_ctas shares of equal cost
-  if (decode_ready) {
+  if (decode_ready && cut_lists) {
     const int64_t n_rows = new_tok_count;
-    const int n_ctas = b->sched_ctas > 0 ? b->sched_ctas : 296;
+    const int n_ctas = sched_ctas > 0 ? sched_ctas : 296;
     // Cost model in token equivalents, fitted to per-share times measured on the device (a full unmasked stage takes
     // about 1.4 us of a half-CTA's time = 80; a unit's q hand-over and epilogue 2.4 us; a stage whose pages are not all
     // full and seen by every row takes the masked softmax path, +0.3 us).
@@ -608,7 +609,7 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   S.decode_ready = decode_ready && new_tok_count > 0;
   S.prefill_ready = prefill_ready && new_tok_count > 0;
   S.sched_kv_heads = sched_kv_heads;
-  S.sched_group = sched_group;
+  S.sched_group = cut_lists ? sched_group : 0;
   S.unique_kv_tokens = unique_tokens;
   S.per_row_kv_tokens = per_row_tokens;
   S.max_node_new = max_new;
@@ -637,6 +638,59 @@ extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, mv_plan** out) {
   P->valid = true;
   *out = P;
   return MV_OK;
+}
+
+mv_status heads_of(const mv_attn_geom* g, int* kv_heads, int* group) {
+  if (g->n_q_heads <= 0 || g->n_kv_heads <= 0) return MV_ERR_INVALID_ARG;
+  if (g->n_q_heads % g->n_kv_heads != 0) return MV_ERR_UNSUPPORTED;
+  *kv_heads = g->n_kv_heads;
+  *group = g->n_q_heads / g->n_kv_heads;
+  return MV_OK;
+}
+}  // namespace
+
+extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, const mv_attn_geom* geom, const mv_plan_tuning* tuning, mv_plan** out) {
+  int kv_heads = 0, group = 0;
+  if (geom) {
+    const mv_status st = heads_of(geom, &kv_heads, &group);
+    if (st != MV_OK) return st;
+  }
+  const mv_status st = plan_impl(b, kv_heads, group, tuning ? tuning->chunk_tokens : 0, tuning ? tuning->sched_ctas : 0, out);
+  if (st != MV_OK) return st;
+  mv_plan::SavedBatch& sv = (*out)->saved;
+  sv.kept = false;
+  if (!geom) {  // keep the batch: the work lists are cut when a geometry is bound
+    const int n_nodes = b->node_off[b->n_req];
+    sv.n_req = b->n_req; sv.page_size = b->page_size; sv.vis_mode = b->vis_mode; sv.pos_mode = b->pos_mode;
+    sv.node_off.assign(b->node_off, b->node_off + b->n_req + 1);
+    auto copy = [&](std::vector<int32_t>& v, const int32_t* p, size_t n) { if (n) v.assign(p, p + n); else v.clear(); };
+    copy(sv.node_len, b->node_len, size_t(n_nodes));
+    copy(sv.node_new, b->node_new, size_t(n_nodes));
+    copy(sv.parent_off, b->parent_off, n_nodes ? size_t(n_nodes) + 1 : 0);
+    copy(sv.parent_idx, b->parent_idx, n_nodes ? size_t(b->parent_off[n_nodes]) : 0);
+    copy(sv.page_off, b->page_off, n_nodes ? size_t(n_nodes) + 1 : 0);
+    copy(sv.page_idx, b->page_idx, n_nodes ? size_t(b->page_off[n_nodes]) : 0);
+    sv.kept = true;
+  }
+  return MV_OK;
+}
+
+extern "C" mv_status mv_plan_bind_geometry(mv_plan* P, const mv_attn_geom* geom, const mv_plan_tuning* tuning) {
+  if (!P || !P->valid || !geom) return MV_ERR_INVALID_ARG;
+  if (!P->saved.kept) return MV_ERR_UNSUPPORTED;
+  int kv_heads = 0, group = 0;
+  const mv_status hs = heads_of(geom, &kv_heads, &group);
+  if (hs != MV_OK) return hs;
+  const mv_plan::SavedBatch& sv = P->saved;
+  mv_dag_batch b{};
+  b.n_req = sv.n_req;
+  b.node_off = sv.node_off.data();
+  b.node_len = sv.node_len.data(); b.node_new = sv.node_new.data();
+  b.parent_off = sv.parent_off.data(); b.parent_idx = sv.parent_idx.data();
+  b.page_off = sv.page_off.data(); b.page_idx = sv.page_idx.data();
+  b.page_size = sv.page_size; b.vis_mode = sv.vis_mode; b.pos_mode = sv.pos_mode;
+  // planning is deterministic, so the canonical tables come out as they were; the saved batch is not touched by it
+  return plan_impl(&b, kv_heads, group, tuning ? tuning->chunk_tokens : 0, tuning ? tuning->sched_ctas : 0, &P);
 }
 
 extern "C" mv_status mv_plan_table(const mv_plan* P, int which, const void** host_ptr, int64_t* count) {

@@ -4,6 +4,8 @@ every step of the path (planning, RoPE + cache write, attention) is a call into 
 """
 from __future__ import annotations
 
+import dataclasses
+
 import numpy as np
 import torch
 
@@ -46,9 +48,10 @@ class PlanOnDevice:
         return self.plan.stats()
 
 
-def _stack_values(wl: synth.Workload, which: str, device):
+def _stack_values(wl: synth.Workload, which: str, device, heads=None):
     """Concatenate per-request raw values on the device.  which = 'history' (tokens already in the pool),
-    'new' (this step's tokens) or 'all' (every token, for prefill)."""
+    'new' (this step's tokens) or 'all' (every token, for prefill).  ``heads`` = (first query head, query heads, first
+    KV head, KV heads) keeps only that head slice (sharding by KV head: the values are drawn for the whole geometry)."""
     dt = torch_dtype(wl.geom)
     b = wl.batch
     qs, ks, vs = [], [], []
@@ -72,20 +75,29 @@ def _stack_values(wl: synth.Workload, which: str, device):
         if which != "history":
             qs.append(torch.from_numpy(vals["q"]).to(dt))
     g = wl.geom
+    if heads is not None:
+        q0, nq, k0, nk = heads
+        qs = [x[:, q0:q0 + nq].contiguous() for x in qs]
+        ks = [x[:, k0:k0 + nk].contiguous() for x in ks]
+        vs = [x[:, k0:k0 + nk].contiguous() for x in vs]
+    hq, hkv = (g.n_q_heads, g.n_kv_heads) if heads is None else (heads[1], heads[3])
     cat = lambda xs, h: (torch.cat(xs, 0) if xs else torch.zeros(0, h, g.head_dim, dtype=dt)).to(device)
-    q = cat(qs, g.n_q_heads) if which != "history" else None
-    return q, cat(ks, g.n_kv_heads), cat(vs, g.n_kv_heads)
+    q = cat(qs, hq) if which != "history" else None
+    return q, cat(ks, hkv), cat(vs, hkv)
 
 
 class DecodeState:
     """Pools holding the history of a decode workload, plus this step's inputs, plan and workspace."""
 
     def __init__(self, wl: synth.Workload, device="cuda", chunk_tokens: int = 0, canary: bool = False,
-                 n_pool_copies: int = 1):
+                 n_pool_copies: int = 1, heads=None):
         assert wl.kind == "decode"
         self.wl, self.device = wl, device
         g, b = wl.geom, wl.batch
-        self.geom = B.geom_of(wl)
+        if heads is not None:   # this process owns a slice of the KV heads, their query heads and their pools
+            g = dataclasses.replace(g, n_q_heads=heads[1], n_kv_heads=heads[3])
+        self.local_geom = g
+        self.geom = B.make_geom(g.n_q_heads, g.n_kv_heads, g.head_dim, b.num_pages, g.dtype, g.page_size, 0.0, g.rope_base)
         dt = torch_dtype(g)
         shape = pool_shape(b.num_pages, g)
         fill = float("nan") if canary else 0.0
@@ -94,13 +106,13 @@ class DecodeState:
         # history -> pools through the library's own RoPE + cache-write call
         hist = synth.DagBatch(b.n_req, b.node_off, np.zeros_like(b.node_len), b.node_len, b.parent_off, b.parent_idx,
                               b.page_off, b.page_idx, b.page_size, b.num_pages, b.vis_mode, b.pos_mode)
-        _, kh, vh = _stack_values(wl, "history", device)
+        _, kh, vh = _stack_values(wl, "history", device, heads)
         hp = PlanOnDevice(hist, device, geom=g)
         for kp, vp in self.pools:
             B.mv_rope_write_kv(hp.plan, self.geom, None, kh, vh, None, None, kp, vp)
         torch.cuda.synchronize()
         del kh, vh, hp
-        self.q, self.k, self.v = _stack_values(wl, "new", device)
+        self.q, self.k, self.v = _stack_values(wl, "new", device, heads)
         self.pod = PlanOnDevice(b, device, chunk_tokens, geom=g)
         self.plan = self.pod.plan
         self.q_rot = torch.empty_like(self.q)

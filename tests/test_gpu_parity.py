@@ -463,3 +463,47 @@ def test_bounded_wait_runs_out_with_a_status_not_a_fault():
     assert st.plan.read_status() == 0
     assert np.array_equal(_np(st.step()), want)
     check_decode(wl, want)
+
+
+def test_decode_kv_head_slices_put_together_equal_the_full_step():
+    """Sharding by KV head on one GPU: the library runs once per half of the KV heads (each with its own pools and its
+    own plan cut for four heads); the slices put side by side along the head axis match the oracle like the full run."""
+    rt = _rt()
+    from paper_2602_07529_b200 import multirank
+    wl = synth.config3(n_req=4, prefix=700)
+    full = _np(rt.DecodeState(wl).step())
+    parts = []
+    for rank in range(2):
+        sl = multirank.head_slice(wl.geom.n_q_heads, wl.geom.n_kv_heads, rank, 2)
+        st = rt.DecodeState(wl, heads=sl)
+        assert st.plan.stats()["sched_kv_heads"] == 4 and st.q.shape[1] == 16 and st.pools[0][0].shape[1] == 4
+        parts.append(_np(st.step()))
+        assert st.plan.read_status() == 0
+    got = np.concatenate(parts, axis=1)
+    assert got.shape == full.shape
+    check_decode(wl, got)
+    assert max_abs(got, full) <= 2e-2 and rel_l2(got, full) <= 4e-3     # two roundings of the same values
+
+
+def test_decode_with_a_geometry_bound_after_planning():
+    """mv_plan_dag without a geometry, mv_plan_bind_geometry afterwards: the decode call refuses the unbound plan and runs
+    the bound one, for two different geometries on the same batch."""
+    B, rt = _B(), _rt()
+    for hq, hkv in ((32, 8), (4, 4)):
+        wl = synth.config2(n_req=2, prefix=260, branches=3, branch_len=70)
+        wl.geom = synth.Geometry(hq, hkv, 128, 16, "bf16")
+        st = rt.DecodeState(wl)
+        want = _np(st.step())
+        plan = B.Plan(wl.batch)
+        buf = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+        plan.upload(buf)
+        kp, vp = st.pools[0]
+        with pytest.raises(B.MvError) as e:
+            B.mv_dag_decode_attn(plan, st.geom, st.q_rot, kp, vp, st.out, st.workspace)
+        assert e.value.status == 4
+        plan.bind_geometry(st.geom)
+        plan.upload(buf)
+        st.out.zero_()
+        B.mv_dag_decode_attn(plan, st.geom, st.q_rot, kp, vp, st.out, st.workspace)
+        torch.cuda.synchronize()
+        assert np.array_equal(_np(st.out), want)

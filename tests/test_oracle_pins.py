@@ -525,3 +525,49 @@ def test_backward_siblings_get_no_gradient_from_a_branch():
     assert np.all(dk[160:] == 0) and np.all(dv[160:] == 0)
     assert np.abs(dk[:128]).max() > 0 and np.abs(dv[128:160]).max() > 0
     assert np.all(dq[:128] == 0) and np.all(dq[160:] == 0)
+
+
+# ------------------------------------------------------------------ FP8 (e4m3) cache format pins
+
+def test_round_e4m3_against_the_enumerated_format():
+    """All 256 codes of the 8-bit format decoded from its definition (sign, 4 exponent bits with bias 7, 3 mantissa bits,
+    0x7F / 0xFF are NaN, no infinities); rounding must return the nearest of the finite ones, ties to the even code."""
+    vals = []
+    for code in range(128):
+        e, m = code >> 3, code & 7
+        if code == 0x7F:
+            continue
+        vals.append((m / 8.0) * 2.0 ** -6 if e == 0 else (1 + m / 8.0) * 2.0 ** (e - 7))
+    vals = np.asarray(vals)
+    assert vals.max() == 448.0 and vals[1] == 2.0 ** -9 and len(vals) == 127
+    assert np.array_equal(O.round_e4m3(vals), vals) and np.array_equal(O.round_e4m3(-vals), -vals)
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.standard_normal(4000) * 3, rng.standard_normal(2000) * 200, rng.standard_normal(2000) * 0.01, [1000.0, -1e9]])
+    got = O.round_e4m3(x)
+    for xi, gi in zip(x, got):
+        a = min(abs(xi), 448.0)
+        d = np.abs(vals - a)
+        best = vals[np.flatnonzero(d == d.min())]
+        if len(best) == 2:                                  # a tie: the code with an even mantissa wins
+            codes = [int(np.flatnonzero(vals == b)[0]) for b in best]
+            best = [b for b, c in zip(best, codes) if (c + (1 if c >= 0x7F else 0)) % 2 == 0]
+        assert abs(gi) == best[0] and (gi == 0 or np.sign(gi) == np.sign(xi))
+
+
+def test_fp8_cache_oracle_reduces_to_the_plain_one():
+    """With K and V already e4m3-representable at the given scales, the FP8 oracle equals the plain one; in general it is
+    the plain oracle evaluated on the quantised cache; and its distance from the unquantised result stays within the
+    format's unit roundoff (2^-4) in relative L2."""
+    wl = synth.config2(n_req=1, prefix=70, branches=2, branch_len=20)
+    b = batch_dict(wl.batch)
+    vals = synth.request_values(wl, 0)
+    ks, vs = np.full(8, 0.01), np.full(8, 0.02)
+    o8 = O.decode_request_fp8(b, 0, vals["q"], vals["k"], vals["v"], ks, vs)
+    o = O.decode_request(b, 0, vals["q"], vals["k"], vals["v"])
+    rel = np.linalg.norm(o8 - o) / np.linalg.norm(o)
+    assert 1e-4 < rel < 2.0 ** -4
+    vq = O.quantise_kv_e4m3(vals["v"], vs)
+    assert np.array_equal(O.quantise_kv_e4m3(vq, vs), vq)                      # idempotent
+    # values only: quantising V by hand and giving a scale under which K is untouched (K = 0 here) is the same thing
+    k0 = np.zeros_like(vals["k"])
+    assert np.array_equal(O.decode_request_fp8(b, 0, vals["q"], k0, vals["v"], ks, vs), O.decode_request(b, 0, vals["q"], k0, vq))

@@ -152,3 +152,30 @@ def test_tensor_map_cache_is_keyed_by_device_pointers_and_extent():
     assert probe(0, v, k, 0, 4096, 128) is False                  # K and V swapped: fifth key, evicts the oldest entry
     assert probe(0, k, v, 0, 4096, 128) is False                  # ... which was the first one
     assert probe(0, k, v, k, 4096, 128) is False                  # a third pointer is part of the key
+
+
+def test_plan_without_geometry_then_bind_any_geometry():
+    """A plan made from the paper-level description alone has the canonical tables; the decode work lists are cut when a
+    geometry is bound, and can be cut again for another one; the canonical tables never change."""
+    wl = synth.config2(n_req=2, prefix=300, branches=5, branch_len=40)
+    plan = B.Plan(wl.batch)                                   # no geometry
+    st = plan.stats()
+    assert st["decode_ready"] == 1 and st["sched_kv_heads"] == 0 and st["n_items"] == 0 and st["n_partials"] == 0
+    want = O.plan_tables(batch_dict(wl.batch))
+    tabs = {k: plan.table(k) for k in want}
+    assert all(np.array_equal(tabs[k], want[k]) for k in want)
+    for hq, hkv in ((32, 8), (8, 8), (6, 2)):
+        plan.bind_geometry(B.make_geom(hq, hkv, 128, wl.batch.num_pages, "bf16"))
+        st = plan.stats()
+        assert (st["sched_kv_heads"], st["sched_group"]) == (hkv, hq // hkv) and st["n_items"] > 0
+        assert all(np.array_equal(plan.table(k), tabs[k]) for k in tabs)
+        same = B.Plan(wl.batch, geom=B.make_geom(hq, hkv, 128, wl.batch.num_pages, "bf16"))
+        for name in ("stages", "units", "item_rows", "cta_unit_off", "rowkv_part_off"):
+            assert np.array_equal(plan.work_table(name), same.work_table(name)), name
+    made_with = B.Plan(wl.batch, geom=B.make_geom(32, 8, 128, wl.batch.num_pages, "bf16"))
+    import pytest
+    with pytest.raises(B.MvError) as e:                       # it kept no copy of the batch
+        made_with.bind_geometry(B.make_geom(8, 8, 128, wl.batch.num_pages, "bf16"))
+    assert e.value.status == 4
+    with pytest.raises(B.MvError):                            # 6 query heads over 4 KV heads
+        B.Plan(wl.batch, geom=B.make_geom(6, 4, 128, wl.batch.num_pages, "bf16"))

@@ -88,10 +88,10 @@ def test_scheduler_steps_feed_the_attention_planner():
         b = s.step()
         if b is None:
             break
-        # the struct the scheduler filled goes to the planner as it is (the caller only adds its scheduling hints)
-        s.c_batch.n_kv_heads, s.c_batch.group_size = 8, 4
+        # the struct the scheduler filled goes to the planner as it is, next to the geometry the step will run with
+        geom = B.make_geom(32, 8, 128, 256, "bf16")
         h = C.c_void_p(None)
-        assert B.lib.mv_plan_dag(C.byref(s.c_batch), C.byref(h)) == 0
+        assert B.lib.mv_plan_dag(C.byref(s.c_batch), C.byref(geom), None, C.byref(h)) == 0
         B.lib.mv_plan_destroy(h)
         # and the same arrays through the binding's own batch type, to read the tables back
         batch = synth.DagBatch(b["n_req"], b["node_off"], b["node_len"], b["node_new"], b["parent_off"], b["parent_idx"],
