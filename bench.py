@@ -610,12 +610,59 @@ def _legs(torch, B, runtime, synth, dev, peaks, region, barrier, args, headline_
                 legs["rope_write_kv_config2"] = leg.rope_leg(peaks)
         del leg
         torch.cuda.empty_cache()
+    for name in ("config2", "config3"):
+        with region:
+            legs["decode_fp8_" + name], parity["decode_fp8_" + name] = _fp8_leg(torch, B, runtime, synth, dev, peaks, name)
+        torch.cuda.empty_cache()
     with region:
         legs["prefill"], legs["rope_write_kv_config4"], p4, (legs["prefill_backward"], pb) = _prefill_leg(torch, B, runtime, synth, dev, peaks)
         legs["append"], pa = _append_leg(torch, B, runtime, synth, dev, peaks)
         legs["prefill_config1_f32"], p1 = _config1_leg(torch, B, runtime, synth, dev)
     parity["prefill_config4"], parity["append"], parity["prefill_config1"], parity["prefill_backward_config4"] = p4, pa, p1, pb
     return legs, parity
+
+
+def _fp8_leg(torch, B, runtime, synth, dev, peaks, name):
+    """mv_dag_decode_attn_fp8: the same decode step with the KV history in 8-bit-float pools (one byte per element: half the
+    stream).  Algorithmic bytes: unique visible KV tokens x KV heads x head_dim x 2 (K, V) x 1 B, plus q and out in bf16."""
+    from oracle import medverse_oracle as O
+    wl = _workload(name)
+    g, b = wl.geom, wl.batch
+    pool_bytes = 2 * b.num_pages * g.n_kv_heads * g.page_size * g.head_dim
+    n_pools = max(2, min(8, int(np.ceil(1.0e9 / pool_bytes))))
+    st = runtime.DecodeStateFP8(wl, dev, n_pool_copies=n_pools)
+    stats = st.plan.stats()
+    rows = stats["n_new_tokens"]
+    algo = stats["unique_kv_tokens"] * g.n_kv_heads * g.head_dim * 2 + 2 * rows * g.n_q_heads * g.head_dim * 2
+    for i in range(n_pools):
+        st.step(i)
+
+    def call(i):
+        kp, vp = st.pools[i % n_pools]
+        B.mv_dag_decode_attn_fp8(st.plan, st.geom, st.q_rot, kp, vp, st.kv_scale, st.out, st.workspace)
+    ms, ms_min, launches, _ = _median_launch_ms(torch, call)
+    gbs = algo / (ms * 1e-3) / 1e9
+    leg = {"workload": wl.name + ", FP8 (e4m3) KV cache", "rows": int(rows), "ms": ms, "ms_min": ms_min, "launches": launches,
+           "algorithmic_bytes": int(algo), "GBs": gbs, "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0,
+           "query_tokens_per_s": rows / (ms * 1e-3), "l2": f"{n_pools} pool copies, {n_pools * pool_bytes / 1e9:.2f} GB"}
+    torch.cuda.synchronize()
+    got = st.out.float().cpu().numpy()
+    reqs = _parity_requests(wl, 8)
+    ks, vs = synth.fp8_scales(g)
+    bd = _batch_dict(b)
+    first, acc = [], 0
+    for r in range(b.n_req):
+        first.append(acc)
+        acc += int(sum(int(b.node_new[n]) for n in b.request_nodes(r)))
+    gs, ws = [], []
+    for r in reqs:
+        vals = synth.request_values(wl, r)
+        o = O.decode_request_fp8(bd, r, vals["q"], vals["k"], vals["v"], ks, vs, base=g.rope_base)
+        ws.append(o)
+        gs.append(got[first[r]:first[r] + o.shape[0]])
+    err, rel = _bf16_err(np.concatenate(gs), np.concatenate(ws))
+    return leg, {"max_abs": err, "rel_l2": rel, "rows": int(sum(x.shape[0] for x in gs)), "requests": len(reqs),
+                 "ok": bool(err <= BF16_TOL[0] and rel <= BF16_TOL[1]), "oracle": "cache quantised with the same per-head scales"}
 
 
 def _prefill_leg(torch, B, runtime, synth, dev, peaks):

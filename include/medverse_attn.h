@@ -238,6 +238,27 @@ mv_status mv_dag_decode_attn(const mv_plan* plan, const mv_attn_geom* geom, cons
                              const void* k_pages, const void* v_pages, void* out, void* workspace,
                              size_t workspace_bytes, void* cuda_stream);
 
+/* FP8 KV cache variant of the decode step (no counterpart in the paper: a storage format that halves the bytes a decode
+ * step streams).  The pools hold 8-bit floats with 4 exponent and 3 mantissa bits (largest finite value 448, no
+ * infinities), one scale per KV head: value = stored * scale[head].  kv_scale is a DEVICE array of 2 * n_kv_heads floats:
+ * the K scales of all heads, then the V scales (positive; chosen by the caller, e.g. from calibration).
+ * Pool layout: [num_pages][n_kv_heads][page_size][head_dim] bytes, K and V separate: the block of one (page, KV head) is
+ * 2 KB, contiguous, one token per 128-byte row.
+ *
+ * mv_rope_write_kv_fp8 is mv_rope_write_kv writing such pools: k_pages8[slot[t]] = round(RoPE(k[t], pos_id[t]) / K scale),
+ * v_pages8[slot[t]] = round(v[t] / V scale), rounding to nearest even and saturating at +-448; q_rot as before (bf16).
+ * mv_dag_decode_attn_fp8 is mv_dag_decode_attn reading them: same plan, same work lists, same workspace, same result up
+ * to the format's rounding.  Inside the kernel the queries and the softmax weights are 8-bit floats as well (one scale
+ * per q-vector; each as a rounded value plus a rounded remainder, about seven bits of mantissa), so that both products
+ * run on the tensor cores' 8-bit path straight on the pool bytes.
+ * MV_BF16 queries and outputs, head_dim 128, single-token steps only (max one new token per node); anything else is
+ * MV_ERR_UNSUPPORTED.  Other errors as for mv_rope_write_kv and mv_dag_decode_attn. */
+mv_status mv_rope_write_kv_fp8(const mv_plan* plan, const mv_attn_geom* geom, const void* q, const void* k, const void* v,
+                               void* q_rot, void* k_pages8, void* v_pages8, const float* kv_scale, void* cuda_stream);
+mv_status mv_dag_decode_attn_fp8(const mv_plan* plan, const mv_attn_geom* geom, const void* q_rot, const void* k_pages8,
+                                 const void* v_pages8, const float* kv_scale, void* out, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream);
+
 /* Decode attention for callers that cannot allocate device memory.  (The paper has no counterpart: this is
  * a packaging variant of mv_dag_decode_attn, same arithmetic, same kernels.)
  *

@@ -29,7 +29,7 @@ EXPORTS = ["mv_plan_dag", "mv_plan_bind_geometry", "mv_plan_table", "mv_plan_get
            "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
            "mv_dag_prefill_attn", "mv_dag_prefill_attn_bwd", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_decode_step_host_batch", "mv_status_string",
            "mv_launch_count", "mv_plan_read_status", "mv_dag_decode_attn_static",
-           "mv_static_workspace_bytes", "mv_selftest_bounded_wait", "mv_selftest_tmap_cache",
+           "mv_static_workspace_bytes", "mv_rope_write_kv_fp8", "mv_dag_decode_attn_fp8", "mv_selftest_bounded_wait", "mv_selftest_tmap_cache",
            "mv_sched_create", "mv_sched_destroy", "mv_sched_add_request", "mv_sched_step", "mv_sched_rows",
            "mv_sched_commit", "mv_sched_page_refs", "mv_sched_get_stats"]
 
@@ -91,6 +91,8 @@ def _load():
     lib.mv_dag_prefill_attn.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp, sz, vp]
     lib.mv_dag_prefill_attn_bwd.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 10 + [sz, vp]
     lib.mv_dag_decode_attn_static.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp]
+    lib.mv_rope_write_kv_fp8.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 8
+    lib.mv_dag_decode_attn_fp8.argtypes = [vp, C.POINTER(_Geom), vp, vp, vp, vp, vp, vp, sz, vp]
     lib.mv_static_workspace_bytes.argtypes = []
     lib.mv_static_workspace_bytes.restype = sz
     lib.mv_decode_step_staging_bytes.argtypes = [vp, C.POINTER(_Geom)]
@@ -274,6 +276,17 @@ def mv_dag_decode_attn_static(plan: Plan, geom: _Geom, q_rot, k_pages, v_pages, 
     raise MV_ERR_WORKSPACE).  Calls on one device share that array, so they must not overlap on the GPU."""
     _check(lib.mv_dag_decode_attn_static(plan.handle, C.byref(geom), _ptr(q_rot), _ptr(k_pages), _ptr(v_pages),
                                          _ptr(out), _stream_ptr(stream)), "mv_dag_decode_attn_static")
+
+
+def mv_rope_write_kv_fp8(plan: Plan, geom: _Geom, q, k, v, q_rot, k_pages8, v_pages8, kv_scale, stream=None):
+    _check(lib.mv_rope_write_kv_fp8(plan.handle, C.byref(geom), _ptr(q), _ptr(k), _ptr(v), _ptr(q_rot), _ptr(k_pages8), _ptr(v_pages8),
+                                    _ptr(kv_scale), _stream_ptr(stream)), "mv_rope_write_kv_fp8")
+
+
+def mv_dag_decode_attn_fp8(plan: Plan, geom: _Geom, q_rot, k_pages8, v_pages8, kv_scale, out, workspace, stream=None):
+    _check(lib.mv_dag_decode_attn_fp8(plan.handle, C.byref(geom), _ptr(q_rot), _ptr(k_pages8), _ptr(v_pages8), _ptr(kv_scale), _ptr(out),
+                                      _ptr(workspace), workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
+           "mv_dag_decode_attn_fp8")
 
 
 def mv_static_workspace_bytes() -> int:

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libmedverse_attn.so")
-SOURCES = ["planner.cpp", "scheduler.cpp", "plan_runtime.cu", "rope_write_kv.cu", "decode_attn.cu", "decode_attn_tc.cu", "prefill_attn_f32.cu",
+SOURCES = ["planner.cpp", "scheduler.cpp", "plan_runtime.cu", "rope_write_kv.cu", "decode_attn.cu", "decode_attn_tc.cu", "decode_attn_fp8.cu", "prefill_attn_f32.cu",
            "prefill_attn_bf16.cu", "prefill_attn_tc.cu", "prefill_bwd_tc.cu", "decode_step_host.cu", "tma_util.cu", "selftest.cu"]
 
 

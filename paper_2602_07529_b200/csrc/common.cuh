@@ -1,6 +1,7 @@
 // Shared device / launcher helpers of the library (sm_100a only).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <atomic>
@@ -115,6 +116,18 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
+// Two floats -> two 8-bit floats (4 exponent bits, 3 mantissa bits, round to nearest even, saturating at +-448): `lo` in
+// bits 0..7 of the result, `hi` in bits 8..15.  And back (exact: every such value is a half-precision value).
+__device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;\n" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float2 unpack_e4m3x2(uint32_t v) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;\n" : "=r"(h2) : "h"(uint16_t(v)));
+  return __half22float2(*reinterpret_cast<__half2*>(&h2));
+}
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
@@ -131,6 +144,8 @@ namespace mv {
 // Builds a 2-D tiled tensor map over a row-major bf16 matrix [rows][cols] with a [box_rows][64] box and the
 // 128-byte shared-memory swizzle.  Host call, no CUDA context state; false if the driver entry is missing.
 bool make_tmap_bf16_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// The same over a byte matrix [rows][128] (one 8-bit element per byte) with a [box_rows][128] box.
+bool make_tmap_u8_2d(CUtensorMap* map, const void* base, uint64_t rows, uint32_t box_rows);
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");

@@ -32,6 +32,8 @@ mv_status append_tc(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, 
                     cudaStream_t st);
 mv_status decode_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* kp, const void* vp, void* ws,
                     cudaStream_t st);
+mv_status decode_fp8(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* kp, const void* vp, const float* kv_scale,
+                     void* ws, cudaStream_t st);
 }
 
 namespace {
@@ -616,6 +618,36 @@ struct KvMaps {
   CUtensorMap tm_k, tm_v;
 };
 
+// The merge kernel is launched with programmatic stream serialisation: it may become resident while the attention kernel
+// is still running and waits (griddepcontrol.wait) for that grid to complete.
+template <int D>
+mv_status launch_merge(const mv_plan* P, const mv_attn_geom* g, void* ws, void* out, cudaStream_t st) {
+  const int G = g->n_q_heads / g->n_kv_heads;
+  const size_t vecs = size_t(P->stats.n_partials) * size_t(G);
+  const size_t o_bytes = (vecs * D * sizeof(float) + 255) & ~size_t(255);
+  const int n_rows = int(P->stats.n_new_tokens);
+  const int n_warps = n_rows * g->n_q_heads;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(unsigned((n_warps + 3) / 4), 1, 1);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, decode_merge_kernel<D>, static_cast<const float*>(ws),
+                                           reinterpret_cast<const float*>(static_cast<char*>(ws) + o_bytes),
+                                           mv::table<int32_t>(P, P->layout.rowkv_part_off), static_cast<bf16*>(out), n_rows, int(g->n_q_heads), G);
+  mv::g_launches++;
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return MV_ERR_CUDA;
+  }
+  return MV_OK;
+}
+
 template <int D>
 mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* kp, const void* vp, void* out,
                  void* ws, cudaStream_t st) {
@@ -661,29 +693,7 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
     mv::g_launches++;
     if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
   }
-  // the merge kernel is launched with programmatic stream serialisation: it may become resident while the
-  // attention kernel is still running and waits (griddepcontrol.wait) for that grid to complete
-  const int n_rows = int(P->stats.n_new_tokens);
-  const int n_warps = n_rows * g->n_q_heads;
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(unsigned((n_warps + 3) / 4), 1, 1);
-  cfg.blockDim = dim3(128, 1, 1);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, decode_merge_kernel<D>, static_cast<const float*>(a.part_o),
-                                           static_cast<const float*>(a.part_ml), mv::table<int32_t>(P, P->layout.rowkv_part_off),
-                                           static_cast<bf16*>(out), n_rows, int(g->n_q_heads), G);
-  mv::g_launches++;
-  if (e != cudaSuccess) {
-    (void)cudaGetLastError();
-    return MV_ERR_CUDA;
-  }
-  return MV_OK;
+  return launch_merge<D>(P, g, ws, out, st);
 }
 
 }  // namespace
@@ -713,6 +723,31 @@ extern "C" mv_status mv_dag_decode_attn(const mv_plan* P, const mv_attn_geom* g,
     return mv::append_tc(P, g, q_rot, k_pages, v_pages, out, s);
   return g->head_dim == 128 ? launch<128>(P, g, q_rot, k_pages, v_pages, out, workspace, s)
                             : launch<64>(P, g, q_rot, k_pages, v_pages, out, workspace, s);
+}
+
+// ---- decode attention over an FP8 KV cache -----------------------------------------------------------------------
+extern "C" mv_status mv_dag_decode_attn_fp8(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_pages8,
+                                            const void* v_pages8, const float* kv_scale, void* out, void* workspace,
+                                            size_t workspace_bytes, void* cuda_stream) {
+  if (!P || !P->valid) return MV_ERR_INVALID_ARG;
+  mv_status st = mv::check_geom(g);
+  if (st != MV_OK) return st;
+  if (P->stats.n_new_tokens == 0) return MV_OK;
+  if (g->dtype != MV_BF16 || g->head_dim != 128 || !P->stats.decode_ready) return MV_ERR_UNSUPPORTED;
+  if (P->stats.max_node_new > 1) return MV_ERR_UNSUPPORTED;  // single-token steps only: node append keeps the bf16 cache
+  if (!q_rot || !k_pages8 || !v_pages8 || !kv_scale || !out) return MV_ERR_INVALID_ARG;
+  if (!P->device_buf) return MV_ERR_WORKSPACE;
+  if (g->n_kv_heads != P->stats.sched_kv_heads || g->n_q_heads / g->n_kv_heads != P->stats.sched_group) return MV_ERR_UNSUPPORTED;
+  if (P->stats.max_item_rows * P->stats.sched_group > MAXQV) return MV_ERR_UNSUPPORTED;
+  if (P->stats.max_page_id >= g->num_pages) return MV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k_pages8) & 15) || (reinterpret_cast<uintptr_t>(v_pages8) & 15) || (reinterpret_cast<uintptr_t>(q_rot) & 15))
+    return MV_ERR_INVALID_ARG;
+  const size_t need = mv_workspace_bytes(P, g, MV_OP_DECODE_ATTN);
+  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return MV_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  st = mv::decode_fp8(P, g, q_rot, k_pages8, v_pages8, kv_scale, workspace, s);
+  if (st != MV_OK) return st;
+  return launch_merge<128>(P, g, workspace, out, s);
 }
 
 // ---- decode attention for callers that cannot allocate device memory -------------------------------------

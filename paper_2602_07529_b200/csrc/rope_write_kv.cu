@@ -48,6 +48,17 @@ struct Vec16<__nv_bfloat16> {
   }
 };
 
+// N floats times inv -> N bytes of 8-bit floats (N = 4 or 8), one vector store
+template <int N>
+__device__ __forceinline__ void store_e4m3(unsigned char* dst, const float (&x)[N], float inv) {
+  uint32_t w[N / 4];
+#pragma unroll
+  for (int i = 0; i < N / 4; ++i)
+    w[i] = mv::pack_e4m3x2(x[4 * i] * inv, x[4 * i + 1] * inv) | (mv::pack_e4m3x2(x[4 * i + 2] * inv, x[4 * i + 3] * inv) << 16);
+  if (N == 8) *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[N / 4 - 1]);
+  else *reinterpret_cast<uint32_t*>(dst) = w[0];
+}
+
 // theta_i = base^(-2i/d) for i < d/2, evaluated once per launch on the host in double precision
 struct ThetaTable {
   double theta[64];
@@ -77,12 +88,14 @@ __device__ __forceinline__ void rope_cos_sin(int pos, double theta, float& c, fl
 
 // TPC tokens per CTA.  Phase 1: the CTA's (token, i) pairs get their cos / sin, one pair per thread, while the first
 // loads of phase 2 are already in flight; phase 2: 16-byte units of q, k (rotated) and v (copied) stream through.
-template <typename T, int D, int TPC>
+// FP8: the pools hold 8-bit floats (4 exponent, 3 mantissa bits), [pages][KV heads][16 tokens][head_dim bytes]; a value is
+// stored as round(x / scale[head]), saturating (kv_scale = the K scales of all heads, then the V scales).
+template <typename T, int D, int TPC, bool FP8 = false>
 __global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                                                             T* __restrict__ q_rot, T* __restrict__ k_rot, T* __restrict__ k_pages,
                                                             T* __restrict__ v_pages, const int32_t* __restrict__ pos_id,
                                                             const int64_t* __restrict__ slot, int n_tok, int Hq, int Hkv,
-                                                            const __grid_constant__ ThetaTable tt) {
+                                                            const __grid_constant__ ThetaTable tt, const float* __restrict__ kv_scale = nullptr) {
   constexpr int HALF = D / 2;
   constexpr int N = Vec16<T>::N;
   constexpr int CH = HALF / N;  // 16-byte chunks per half head
@@ -116,8 +129,16 @@ __global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* __restrict_
     if (u >= n_q_units + n_k_units) {  // v is stored unrotated
       const int uu = u - n_q_units - n_k_units;
       const int h = uu / VCH, c = uu % VCH;
-      const uint4 val = *reinterpret_cast<const uint4*>(v + (t * Hkv + h) * D + c * N);
       const int e = c * N;
+      if (FP8) {
+        float x[N];
+        Vec16<T>::load(v + (t * Hkv + h) * D + e, x);
+        const float inv = 1.f / __ldg(kv_scale + Hkv + h);
+        unsigned char* dst = reinterpret_cast<unsigned char*>(v_pages) + (page * Hkv + h) * (16 * D) + off * D + e;
+        store_e4m3<N>(dst, x, inv);
+        continue;
+      }
+      const uint4 val = *reinterpret_cast<const uint4*>(v + (t * Hkv + h) * D + e);
       *reinterpret_cast<uint4*>(v_pages + (page * Hkv + h) * (16 * D) + (e >> 6) * 1024 + off * 64 + (e & 63)) = val;
       continue;
     }
@@ -140,7 +161,12 @@ __global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* __restrict_
       Vec16<T>::store(dst + HALF + c * N, ohi);
       continue;
     }
-    if (k_pages != nullptr) {
+    if (FP8) {
+      const float inv = 1.f / __ldg(kv_scale + h);
+      unsigned char* dst = reinterpret_cast<unsigned char*>(k_pages) + (page * Hkv + h) * (16 * D) + off * D;
+      store_e4m3<N>(dst + c * N, olo, inv);
+      store_e4m3<N>(dst + HALF + c * N, ohi, inv);
+    } else if (k_pages != nullptr) {
       // pool element (page, head, token, e) lives in 64-element column block e / 64 of the (page, head) block
       T* dst = k_pages + (page * Hkv + h) * (16 * D) + off * 64;
       const int e0 = c * N, e1 = HALF + c * N;
@@ -185,7 +211,39 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
                             : launch_d<T, 64>(P, g, q, k, v, q_rot, k_rot, k_pages, v_pages, st);
 }
 
+template <int TPC>
+void launch_fp8(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* q_rot, void* k_pages8,
+                void* v_pages8, const float* kv_scale, int n, cudaStream_t st) {
+  using T = __nv_bfloat16;
+  constexpr int D = 128;
+  ThetaTable tt{};
+  const double c = -2.0 * log2(g->rope_base) / double(D);
+  for (int i = 0; i < D / 2; ++i) tt.theta[i] = exp2(double(i) * c);
+  rope_write_kv_kernel<T, D, TPC, true><<<(n + TPC - 1) / TPC, 256, 0, st>>>(
+      (const T*)q, (const T*)k, (const T*)v, (T*)q_rot, nullptr, (T*)k_pages8, (T*)v_pages8, mv::table<int32_t>(P, P->layout.pos_id),
+      mv::table<int64_t>(P, P->layout.slot), n, g->n_q_heads, g->n_kv_heads, tt, kv_scale);
+}
+
 }  // namespace
+
+extern "C" mv_status mv_rope_write_kv_fp8(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v,
+                                          void* q_rot, void* k_pages8, void* v_pages8, const float* kv_scale, void* cuda_stream) {
+  if (!P || !P->valid) return MV_ERR_INVALID_ARG;
+  mv_status st = mv::check_geom(g);
+  if (st != MV_OK) return st;
+  if (g->dtype != MV_BF16 || g->head_dim != 128) return MV_ERR_UNSUPPORTED;
+  if (!P->device_buf) return MV_ERR_WORKSPACE;
+  if (P->stats.n_new_tokens == 0) return MV_OK;
+  if (!k || !v || !k_pages8 || !v_pages8 || !kv_scale) return MV_ERR_INVALID_ARG;
+  if ((q == nullptr) != (q_rot == nullptr)) return MV_ERR_INVALID_ARG;
+  if (P->stats.max_page_id >= g->num_pages || g->rope_base <= 0.0) return MV_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const int n = int(P->stats.n_new_tokens);
+  if (n < 2048) launch_fp8<1>(P, g, q, k, v, q_rot, k_pages8, v_pages8, kv_scale, n, s);
+  else launch_fp8<4>(P, g, q, k, v, q_rot, k_pages8, v_pages8, kv_scale, n, s);
+  mv::g_launches++;
+  return cudaGetLastError() == cudaSuccess ? MV_OK : MV_ERR_CUDA;
+}
 
 extern "C" mv_status mv_rope_write_kv(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k,
                                       const void* v, void* q_rot, void* k_rot, void* k_pages, void* v_pages,

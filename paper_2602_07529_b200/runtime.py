@@ -126,6 +126,42 @@ class DecodeState:
         return self.out
 
 
+class DecodeStateFP8(DecodeState):
+    """The same decode workload with the KV history in FP8 pools (8-bit floats, one scale per KV head)."""
+
+    def __init__(self, wl: synth.Workload, device="cuda", n_pool_copies: int = 1):
+        assert wl.kind == "decode" and wl.geom.dtype == "bf16" and wl.geom.head_dim == 128
+        self.wl, self.device = wl, device
+        g, b = wl.geom, wl.batch
+        self.local_geom = g
+        self.geom = B.make_geom(g.n_q_heads, g.n_kv_heads, g.head_dim, b.num_pages, g.dtype, g.page_size, 0.0, g.rope_base)
+        ks, vs = synth.fp8_scales(g)
+        self.kv_scale = torch.from_numpy(np.concatenate([ks, vs])).to(device)
+        shape = (b.num_pages, g.n_kv_heads, g.page_size, g.head_dim)
+        self.pools = [(torch.zeros(shape, dtype=torch.uint8, device=device), torch.zeros(shape, dtype=torch.uint8, device=device))
+                      for _ in range(n_pool_copies)]
+        hist = synth.DagBatch(b.n_req, b.node_off, np.zeros_like(b.node_len), b.node_len, b.parent_off, b.parent_idx,
+                              b.page_off, b.page_idx, b.page_size, b.num_pages, b.vis_mode, b.pos_mode)
+        _, kh, vh = _stack_values(wl, "history", device)
+        hp = PlanOnDevice(hist, device, geom=g)
+        for kp, vp in self.pools:
+            B.mv_rope_write_kv_fp8(hp.plan, self.geom, None, kh, vh, None, kp, vp, self.kv_scale)
+        torch.cuda.synchronize()
+        del kh, vh, hp
+        self.q, self.k, self.v = _stack_values(wl, "new", device)
+        self.pod = PlanOnDevice(b, device, 0, geom=g)
+        self.plan = self.pod.plan
+        self.q_rot = torch.empty_like(self.q)
+        self.out = torch.empty_like(self.q)
+        self.workspace = _dev_bytes(self.plan.workspace_bytes(self.geom, B.OP_DECODE_ATTN), device)
+
+    def step(self, pool: int = 0, stream=None):
+        kp, vp = self.pools[pool]
+        B.mv_rope_write_kv_fp8(self.plan, self.geom, self.q, self.k, self.v, self.q_rot, kp, vp, self.kv_scale, stream)
+        B.mv_dag_decode_attn_fp8(self.plan, self.geom, self.q_rot, kp, vp, self.kv_scale, self.out, self.workspace, stream)
+        return self.out
+
+
 class PrefillState:
     def __init__(self, wl: synth.Workload, device="cuda", with_pool: bool = True):
         assert wl.kind == "prefill"

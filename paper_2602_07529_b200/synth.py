@@ -308,6 +308,15 @@ def request_values(wl: Workload, r: int) -> dict:
             "node_q_off": np.asarray(q_off, dtype=np.int64)}
 
 
+def fp8_scales(geom: Geometry):
+    """Per-KV-head scales of the FP8 cache variant for this module's N(0, 1) * value_scale draws, as a calibration run
+    would fix them: the format's largest value (448) is put at 8 (keys, whose rotation can grow an element by sqrt 2) and
+    6 (values) standard deviations.  Returns (k_scale[Hkv], v_scale[Hkv]) float32."""
+    k = np.full(geom.n_kv_heads, 8.0 * geom.value_scale / 448.0, np.float32)
+    v = np.full(geom.n_kv_heads, 6.0 * geom.value_scale / 448.0, np.float32)
+    return k, v
+
+
 def unique_visible_tokens(batch: DagBatch, visible_nodes_per_row) -> int:
     """Tokens of every node that at least one row sees, each counted once
     (``visible_nodes_per_row``: iterable of iterables of global node ids)."""

@@ -27,7 +27,7 @@ def _compare(batch):
 def test_library_exports_every_declared_symbol():
     inc = os.path.join(ROOT, "include")
     hdr = "".join(open(os.path.join(inc, f)).read() for f in sorted(os.listdir(inc)) if f.endswith(".h"))
-    declared = set(re.findall(r"\b(mv_[a-z_]+)\s*\(", hdr))
+    declared = set(re.findall(r"\b(mv_[a-z0-9_]+)\s*\(", hdr))
     assert declared, "no declarations parsed"
     assert declared == set(B.EXPORTS)
     lib = ctypes.CDLL(B.LIB_PATH)
