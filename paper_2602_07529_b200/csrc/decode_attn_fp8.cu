@@ -185,9 +185,9 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
     };
     // Between units the first stages go out before the q tile is staged: they do not depend on it, and this keeps the ring
     // full while the producer waits for the previous unit to let go of the q tile (each stage still waits for its own
-    // buffer to come free).  At the start of the share the q tile goes first: every half of the grid asks for its first
-    // three stages at once (28 MB), and a q tile requested behind that burst arrives after it (measured: q ready 5.7 us
-    // after kernel entry, first stage long there), while the few KB of q requested first cost the stages nothing.
+    // buffer to come free).  At the start of the share the q-vectors go first: every half of the grid asks for its first
+    // stages at once, and q-vectors requested behind that burst arrive after it, while the softmax thread, which paces
+    // this kernel, cannot start before they are there.
     int s_next = 0;
     if (ui != 0)
       for (const int pre = min(wu.n_stages, NSTAGES); s_next < pre && ok; ++s_next) ok = issue_stage(s_next);
@@ -446,15 +446,16 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
         mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         mx = mx == -INFINITY ? -INFINITY : mx * mult;  // (a padding q-vector has mult = 0)
       }
-      if (s > 0) {  // O holds stages 0 .. s-1 of the unit once the previous product is done
-        ok = warp_wait(h, bar(&meta->o_done), (g - 1) & 1);
-        if (!ok) break;
-        mv::um::fence_after();
-      }
       if (warp_active) {
         // the reference maximum moves only when it would otherwise let P grow past 2^8
         const bool move = mx > m + RESCALE_THRESHOLD || (m == -INFINITY && mx > -INFINITY);
         if (s > 0 && __any_sync(0xffffffffu, move)) {
+          // O holds stages 0 .. s-1 of the unit once the previous product is done.  Only a warp that rescales waits for it:
+          // here the softmax thread, not the stream, paces a stage.  (The previous product cannot be more than one phase
+          // behind this wait: the product after it needs this very thread's P.)
+          ok = warp_wait(h, bar(&meta->o_done), (g - 1) & 1);
+          if (!ok) break;
+          mv::um::fence_after();
           const float f = (move && m != -INFINITY) ? mv::fast_exp2(m - mx) : 1.f;
 #pragma unroll 1
           for (int c = 0; c < D / 16; ++c) {  // sixteen columns at a time: the scores of the stage are live in registers
