@@ -273,7 +273,10 @@ mv_status mv_dag_decode_attn_fp8(const mv_plan* plan, const mv_attn_geom* geom, 
  *   - Limit: plans with mv_workspace_bytes(plan, geom, MV_OP_DECODE_ATTN) > MV_STATIC_WORKSPACE_BYTES are
  *     refused with MV_ERR_WORKSPACE before anything is launched (query it with mv_static_workspace_bytes()).
  *   - Set-up: the first call on each device looks up the array's device address (one cudaGetSymbolAddress,
- *     with the calling thread's current device); make that first call outside any stream capture.
+ *     with the calling thread's current device).  That first call is a set-up call: with lazy module loading it is
+ *     also the moment the driver brings the array into being on that device (and may synchronise).  Make it at
+ *     start-up, outside any stream capture and outside the region in which nothing may be allocated; every later
+ *     call on that device allocates and frees nothing.
  *   - Sharing: every call on a device uses the same array and finds the previous call's contents in it.
  *     The kernels write each partial result before they read it, so nothing needs clearing; but two calls
  *     whose kernels overlap on the GPU (different streams, no ordering between them) race on it.  Order such

@@ -25,6 +25,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "trace.h"
 #include "tmap_cache.h"
 
 namespace mv {
@@ -701,6 +702,7 @@ mv_status launch(const mv_plan* P, const mv_attn_geom* g, const void* q, const v
 extern "C" mv_status mv_dag_decode_attn(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_pages,
                                         const void* v_pages, void* out, void* workspace, size_t workspace_bytes,
                                         void* cuda_stream) {
+  mv::NvtxRange nvtx_range("mv_dag_decode_attn");
   if (!P || !P->valid) return MV_ERR_INVALID_ARG;
   mv_status st = mv::check_geom(g);
   if (st != MV_OK) return st;
@@ -729,6 +731,7 @@ extern "C" mv_status mv_dag_decode_attn(const mv_plan* P, const mv_attn_geom* g,
 extern "C" mv_status mv_dag_decode_attn_fp8(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_pages8,
                                             const void* v_pages8, const float* kv_scale, void* out, void* workspace,
                                             size_t workspace_bytes, void* cuda_stream) {
+  mv::NvtxRange nvtx_range("mv_dag_decode_attn_fp8");
   if (!P || !P->valid) return MV_ERR_INVALID_ARG;
   mv_status st = mv::check_geom(g);
   if (st != MV_OK) return st;

@@ -12,6 +12,7 @@
 #include <numeric>
 
 #include "plan_internal.h"
+#include "trace.h"
 
 namespace {
 
@@ -650,6 +651,7 @@ mv_status heads_of(const mv_attn_geom* g, int* kv_heads, int* group) {
 }  // namespace
 
 extern "C" mv_status mv_plan_dag(const mv_dag_batch* b, const mv_attn_geom* geom, const mv_plan_tuning* tuning, mv_plan** out) {
+  mv::NvtxRange nvtx_range("mv_plan_dag");
   int kv_heads = 0, group = 0;
   if (geom) {
     const mv_status st = heads_of(geom, &kv_heads, &group);

@@ -7,6 +7,7 @@
 // are double-buffered with cp.async into XOR-swizzled shared memory; QK^T and PV run on m16n8k16 MMAs,
 // softmax is online in log2 units.
 #include "common.cuh"
+#include "trace.h"
 
 namespace {
 
@@ -235,6 +236,7 @@ mv_status prefill_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, con
 extern "C" mv_status mv_dag_prefill_attn(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_rot,
                                          const void* v, void* out, void* workspace, size_t workspace_bytes,
                                          void* cuda_stream) {
+  mv::NvtxRange nvtx_range("mv_dag_prefill_attn");
   if (!P || !P->valid) return MV_ERR_INVALID_ARG;
   mv_status st = mv::check_geom(g);
   if (st != MV_OK) return st;

@@ -20,6 +20,7 @@
 // Every mbarrier wait is bounded; after one ran out a role issues nothing further, the producer and the issuer wait
 // for what they have in flight, and the status word of the plan reads MV_ERR_TIMEOUT.
 #include "common.cuh"
+#include "trace.h"
 #include "tmap_cache.h"
 #include "umma.cuh"
 
@@ -496,6 +497,7 @@ struct BwdMaps {
 extern "C" mv_status mv_dag_prefill_attn_bwd(const mv_plan* P, const mv_attn_geom* g, const void* q_rot, const void* k_rot, const void* v,
                                              const void* out, const void* dout, const void* lse, void* dq_rot, void* dk_rot, void* dv,
                                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  mv::NvtxRange nvtx_range("mv_dag_prefill_attn_bwd");
   if (!P || !P->valid) return MV_ERR_INVALID_ARG;
   mv_status st = mv::check_geom(g);
   if (st != MV_OK) return st;

@@ -10,6 +10,7 @@
 // HBM-bound elementwise kernel: one or four tokens per CTA, 16-byte vector loads and stores, the cos/sin
 // rows of the CTA's tokens are computed once into shared memory and reused by all heads.
 #include "common.cuh"
+#include "trace.h"
 
 namespace {
 
@@ -248,6 +249,7 @@ extern "C" mv_status mv_rope_write_kv_fp8(const mv_plan* P, const mv_attn_geom* 
 extern "C" mv_status mv_rope_write_kv(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k,
                                       const void* v, void* q_rot, void* k_rot, void* k_pages, void* v_pages,
                                       void* cuda_stream) {
+  mv::NvtxRange nvtx_range("mv_rope_write_kv");
   if (!P || !P->valid) return MV_ERR_INVALID_ARG;
   mv_status st = mv::check_geom(g);
   if (st != MV_OK) return st;

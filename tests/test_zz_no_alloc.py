@@ -30,14 +30,18 @@ def test_static_scratch_matches_workspace_entry_point_twice():
     second = runtime.DecodeState(synth.config3(n_req=4, prefix=500))
     want2 = second.step().clone()
     torch.cuda.synchronize()
-    for st, want in ((first, want1), (second, want2)):      # two calls in a row on the shared scratch
+    for i, (st, want) in enumerate(((first, want1), (second, want2))):      # two calls in a row on the shared scratch
         assert st.plan.workspace_bytes(st.geom, B.OP_DECODE_ATTN) <= B.mv_static_workspace_bytes()
         st.out.fill_(float("nan"))
         kp, vp = st.pools[0]
+        free_before = torch.cuda.mem_get_info()[0]
         B.mv_dag_decode_attn_static(st.plan, st.geom, st.q_rot, kp, vp, st.out)
         torch.cuda.synchronize()
+        if i > 0:   # past the set-up call of this device, the entry point leaves the device's free memory as it found it
+            assert torch.cuda.mem_get_info()[0] == free_before
         assert st.plan.read_status() == 0
         _same(st.out, want)
+        assert torch.equal(st.out, want)      # same kernels, same merge order as the workspace entry point: same bits
 
 
 def test_static_scratch_rejects_oversized_plans():
