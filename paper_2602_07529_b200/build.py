@@ -29,8 +29,10 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """``debug``: compile with -DMV_DEBUG (device-side bounds checks that set the plan's status word and skip the access
+    instead of touching memory out of range)."""
+    if not force and not debug and not _stale():
         return LIB
     build_dir = os.path.join(PKG, "_build")
     os.makedirs(build_dir, exist_ok=True)
@@ -39,6 +41,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         common += ["-Xptxas", "-v"]
+    if debug:
+        common += ["-DMV_DEBUG"]
     objs = []
     procs = []
     for src in SOURCES:
@@ -59,4 +63,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -63,6 +63,8 @@ struct TcArgs {
   int32_t* status;
   int Hq, Hkv, G;
   float scale_log2;
+  int n_rows;      // rows of q and out, partial vectors of the workspace: read only by the bounds checks of a debug build
+  int64_t n_vecs;  // (compile with -DMV_DEBUG: an index out of range sets the status word and the access is skipped)
 };
 
 struct Half {  // what every role of one half needs
@@ -218,7 +220,13 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
       const int r = min(x / a.G, MAXQV - 1);
       const int r_lo = __shfl_sync(0xffffffffu, ir0.row, r & 31), r_hi = __shfl_sync(0xffffffffu, ir1.row, r & 31);
       const int row = r < 32 ? r_lo : r_hi;
-      const bool okq = x < n_qv;
+      bool okq = x < n_qv;
+#ifdef MV_DEBUG
+      if (okq && (row < 0 || row >= a.n_rows)) {
+        atomicExch(h.status, int(MV_ERR_INVALID_ARG));
+        okq = false;
+      }
+#endif
       const bf16* src = a.q + (okq ? (int64_t(row) * a.Hq + wu.kvh * a.G + x % a.G) * D + c * 8 : 0);
       const uint32_t dst = h.q_smem + (c >> 3) * (Q_BYTES / 2) + x * 128 + (((c & 7) ^ (x & 7)) << 4);
       mv::cp_async_16(dst, src, okq ? 16 : 0);
@@ -467,6 +475,11 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
     ok = warp_wait(h, bar(&meta->o_done), (g - 1) & 1);
     if (!ok) break;
     mv::um::fence_after();
+#ifdef MV_DEBUG
+    if (pv >= a.n_vecs) atomicExch(h.status, int(MV_ERR_INVALID_ARG));
+    const int pv_checked = pv < a.n_vecs ? pv : -1;
+#define pv pv_checked
+#endif
     if (warp_active) {
       float* po = a.part_o + int64_t(pv >= 0 ? pv : 0) * D;
 #pragma unroll
@@ -483,6 +496,9 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
       }
       if (pv >= 0) *reinterpret_cast<float2*>(a.part_ml + int64_t(pv) * 2) = make_float2(m, l);
     }
+#ifdef MV_DEBUG
+#undef pv
+#endif
     mv::um::fence_before();
     mv::mbar_arrive(bar(&meta->o_free));  // O may be overwritten by the next unit's first product
   }
@@ -591,6 +607,8 @@ mv_status decode_tc(const mv_plan* P, const mv_attn_geom* g, const void* q, cons
   a.Hkv = g->n_kv_heads;
   a.G = G;
   a.scale_log2 = mv::softmax_scale(g) * 1.4426950408889634f;
+  a.n_rows = int(P->stats.n_new_tokens);
+  a.n_vecs = int64_t(vecs);
   const int n_shares = int(P->stats.n_ctas);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(unsigned((n_shares + 1) / 2), 1, 1);

@@ -96,7 +96,8 @@ __global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* __restrict_
                                                             T* __restrict__ q_rot, T* __restrict__ k_rot, T* __restrict__ k_pages,
                                                             T* __restrict__ v_pages, const int32_t* __restrict__ pos_id,
                                                             const int64_t* __restrict__ slot, int n_tok, int Hq, int Hkv,
-                                                            const __grid_constant__ ThetaTable tt, const float* __restrict__ kv_scale = nullptr) {
+                                                            const __grid_constant__ ThetaTable tt, const float* __restrict__ kv_scale = nullptr,
+                                                            int64_t num_pages_dbg = 0, int32_t* status_dbg = nullptr) {
   constexpr int HALF = D / 2;
   constexpr int N = Vec16<T>::N;
   constexpr int CH = HALF / N;  // 16-byte chunks per half head
@@ -115,7 +116,17 @@ __global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* __restrict_
     rope_cos_sin(__ldg(pos_id + t0 + tl), tt.theta[i], c, s);
     cs[tl][i] = c;
     sn[tl][i] = s;
-    if (i == 0) s_slot[tl] = __ldg(slot + t0 + tl);
+    if (i == 0) {
+      int64_t sl = __ldg(slot + t0 + tl);
+#ifdef MV_DEBUG
+      // debug build: a slot outside the pool sets the status word and the token's cache write is skipped
+      if ((k_pages != nullptr || v_pages != nullptr) && (sl < 0 || (sl >> 4) >= num_pages_dbg)) {
+        atomicExch(status_dbg, int(MV_ERR_INVALID_ARG));
+        sl = -1;
+      }
+#endif
+      s_slot[tl] = sl;
+    }
   }
   __syncthreads();
   const int n_q_units = q ? Hq * CH : 0;
@@ -126,11 +137,17 @@ __global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* __restrict_
     const int tl = x / per_tok, u = x % per_tok;
     const int64_t t = t0 + tl;
     const int64_t sl = s_slot[tl];
+#ifdef MV_DEBUG
+    const bool pool_ok = sl >= 0;
+#else
+    constexpr bool pool_ok = true;
+#endif
     const int64_t page = sl >> 4, off = sl & 15;
     if (u >= n_q_units + n_k_units) {  // v is stored unrotated
       const int uu = u - n_q_units - n_k_units;
       const int h = uu / VCH, c = uu % VCH;
       const int e = c * N;
+      if (!pool_ok) continue;
       if (FP8) {
         float x[N];
         Vec16<T>::load(v + (t * Hkv + h) * D + e, x);
@@ -162,12 +179,12 @@ __global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* __restrict_
       Vec16<T>::store(dst + HALF + c * N, ohi);
       continue;
     }
-    if (FP8) {
+    if (FP8 && pool_ok) {
       const float inv = 1.f / __ldg(kv_scale + h);
       unsigned char* dst = reinterpret_cast<unsigned char*>(k_pages) + (page * Hkv + h) * (16 * D) + off * D;
       store_e4m3<N>(dst + c * N, olo, inv);
       store_e4m3<N>(dst + HALF + c * N, ohi, inv);
-    } else if (k_pages != nullptr) {
+    } else if (!FP8 && k_pages != nullptr && pool_ok) {
       // pool element (page, head, token, e) lives in 64-element column block e / 64 of the (page, head) block
       T* dst = k_pages + (page * Hkv + h) * (16 * D) + off * 64;
       const int e0 = c * N, e1 = HALF + c * N;
@@ -182,6 +199,8 @@ __global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* __restrict_
   }
 }
 
+inline int32_t* dbg_status(const mv_plan* P) { return const_cast<int32_t*>(mv::table<int32_t>(P, P->layout.sched)) + 2; }
+
 template <typename T, int D>
 mv_status launch_d(const mv_plan* P, const mv_attn_geom* g, const void* q, const void* k, const void* v, void* q_rot,
                    void* k_rot, void* k_pages, void* v_pages, cudaStream_t st) {
@@ -195,11 +214,11 @@ mv_status launch_d(const mv_plan* P, const mv_attn_geom* g, const void* q, const
   // amortise the set-up and keep more 16-byte units in flight per thread
   if (n < 2048)
     rope_write_kv_kernel<T, D, 1><<<n, 256, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_rot, (T*)k_pages,
-                                                     (T*)v_pages, pos, slot, n, g->n_q_heads, g->n_kv_heads, tt);
+                                                     (T*)v_pages, pos, slot, n, g->n_q_heads, g->n_kv_heads, tt, nullptr, g->num_pages, dbg_status(P));
   else
     rope_write_kv_kernel<T, D, 4><<<(n + 3) / 4, 256, 0, st>>>((const T*)q, (const T*)k, (const T*)v, (T*)q_rot, (T*)k_rot,
                                                                (T*)k_pages, (T*)v_pages, pos, slot, n, g->n_q_heads,
-                                                               g->n_kv_heads, tt);
+                                                               g->n_kv_heads, tt, nullptr, g->num_pages, dbg_status(P));
   mv::g_launches++;
   if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
   return MV_OK;
@@ -222,7 +241,7 @@ void launch_fp8(const mv_plan* P, const mv_attn_geom* g, const void* q, const vo
   for (int i = 0; i < D / 2; ++i) tt.theta[i] = exp2(double(i) * c);
   rope_write_kv_kernel<T, D, TPC, true><<<(n + TPC - 1) / TPC, 256, 0, st>>>(
       (const T*)q, (const T*)k, (const T*)v, (T*)q_rot, nullptr, (T*)k_pages8, (T*)v_pages8, mv::table<int32_t>(P, P->layout.pos_id),
-      mv::table<int64_t>(P, P->layout.slot), n, g->n_q_heads, g->n_kv_heads, tt, kv_scale);
+      mv::table<int64_t>(P, P->layout.slot), n, g->n_q_heads, g->n_kv_heads, tt, kv_scale, g->num_pages, dbg_status(P));
 }
 
 }  // namespace
