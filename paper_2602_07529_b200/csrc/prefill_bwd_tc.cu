@@ -30,13 +30,18 @@ using bf16 = __nv_bfloat16;
 constexpr int D = 128;
 constexpr int BT = 128;                 // rows of every tile (queries or keys)
 constexpr int TILE_BYTES = BT * D * 2;  // 32 KB: [2 column blocks][128 rows][128 B]
-constexpr int NTHREADS = 192;           // warp 0 producer, warp 1 issuer, warps 2..5 one thread per tensor-memory lane
-constexpr int OFF_FIXED = 0;            // two tiles that stay for the whole CTA (dq: Q, dO; dkv: K, V)
-constexpr int OFF_RING = 2 * TILE_BYTES;  // two stages of two tiles (dq: K, V; dkv: Q, dO)
-constexpr int NSTAGE = 2;
-constexpr int OFF_VEC = OFF_RING + NSTAGE * 2 * TILE_BYTES;  // dkv: per stage lse[128], delta[128] of the stage's queries
-constexpr int OFF_BAR = OFF_VEC + NSTAGE * 2 * BT * 4;
-constexpr int SMEM_BYTES = OFF_BAR + 128;
+constexpr int HB = 64;                  // a step is one 64-column half of a 128 x 128 score tile
+constexpr int HALF_BYTES = HB * D * 2;  // 16 KB: [2 column blocks][64 rows][128 B]
+constexpr int NTHREADS = 320;           // warp 0 producer, warp 1 issuer, warps 2..9: two threads per tensor-memory lane,
+                                        // each taking 32 of a step's 64 columns
+constexpr int OFF_FIXED = 0;            // two 128-row tiles that stay for the whole CTA (dq: Q, dO; dkv: K, V)
+constexpr int OFF_RING = 2 * TILE_BYTES;  // stages of two 64-row halves (dq: K, V; dkv: Q, dO), one stage per step
+constexpr int NSTAGE = 4;
+constexpr int STAGE_BYTES = 2 * HALF_BYTES;
+constexpr int OFF_VEC = OFF_RING + NSTAGE * STAGE_BYTES;  // dkv: per stage lse[64], delta[64] of the step's queries
+constexpr int OFF_BAR = OFF_VEC + NSTAGE * 2 * HB * 4;
+constexpr int N_BARS = 2 + 2 * NSTAGE + 6;
+constexpr int SMEM_BYTES = OFF_BAR + N_BARS * 8 + 16;
 
 struct BwdArgs {
   const mv::QTile* tiles;     // dq: query tiles; dkv: key tiles
@@ -52,7 +57,8 @@ struct BwdArgs {
 };
 
 struct Bars {
-  uint32_t fixed_full, full, empty, s_full, p_full, acc_done, drained;  // full / empty: NSTAGE consecutive barriers
+  // full / empty: NSTAGE consecutive barriers; s_full / p_full / acc_done: one per score buffer (two)
+  uint32_t fixed_full, full, empty, s_full, p_full, acc_done, drained;
 };
 
 struct Waiter {
@@ -71,7 +77,7 @@ struct Waiter {
   __device__ __forceinline__ bool aborted() const { return *abort != 0; }
 };
 
-// 128-row sub-tiles of a tile's ranges, in table order.  FWD walk (dq): a causal range ends after the tile's last query.
+// 64-row steps of a tile's ranges, in table order.  FWD walk (dq): a causal range ends after the tile's last query.
 // Transposed walk (dkv): a causal range starts at the tile's first key and is not cut.
 struct Walk {
   const mv::KvRange* rg;
@@ -88,38 +94,45 @@ struct Walk {
       if (causal) end = min(end, last_causal + 1);
     }
     start = pos;
-    n = min(BT, end - pos);
+    n = min(HB, end - pos);
     c = causal;
-    pos += BT;
+    pos += HB;
     return true;
   }
 };
 
+// every tensor map's box is 64 columns x 64 rows (8 KB)
 __device__ __forceinline__ void load_tile(uint32_t dst, const CUtensorMap* tm, int col, int row, uint32_t bar) {
-  for (int h = 0; h < 2; ++h) mv::tma_load_2d(dst + h * (TILE_BYTES / 2), tm, col + h * 64, row, bar);
+  for (int cb = 0; cb < 2; ++cb)
+    for (int rh = 0; rh < 2; ++rh) mv::tma_load_2d(dst + cb * (TILE_BYTES / 2) + rh * (HALF_BYTES / 2), tm, col + cb * 64, row + rh * HB, bar);
+}
+__device__ __forceinline__ void load_half(uint32_t dst, const CUtensorMap* tm, int col, int row, uint32_t bar) {
+  for (int cb = 0; cb < 2; ++cb) mv::tma_load_2d(dst + cb * (HALF_BYTES / 2), tm, col + cb * 64, row, bar);
 }
 
-// D[tmem] = A B^T with both operands K-major tiles ([128 rows][128 elements of the contraction]): eight k-steps
-__device__ __forceinline__ void issue_nt(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc) {
-  constexpr uint32_t idesc = mv::um::idesc_bf16(BT, BT, 0, 0);
+// D[tmem, 128 x 64] = A B^T, A a K-major 128-row tile, B a K-major 64-row half: eight k-steps over head_dim
+__device__ __forceinline__ void issue_nt(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr) {
+  constexpr uint32_t idesc = mv::um::idesc_bf16(BT, HB, 0, 0);
+  const uint64_t a_desc = mv::um::smem_desc(a_addr, 16, 1024), b_desc = mv::um::smem_desc(b_addr, 16, 1024);
   mv::um::mma_ss<false>(d_tmem, a_desc, b_desc, idesc);
 #pragma unroll
   for (int k = 1; k < D / 16; ++k) {
-    const uint32_t off = ((k >> 2) * (TILE_BYTES / 2) + (k & 3) * 32) >> 4;
-    mv::um::mma_ss<true>(d_tmem, a_desc + off, b_desc + off, idesc);
+    const uint32_t a_off = ((k >> 2) * (TILE_BYTES / 2) + (k & 3) * 32) >> 4, b_off = ((k >> 2) * (HALF_BYTES / 2) + (k & 3) * 32) >> 4;
+    mv::um::mma_ss<true>(d_tmem, a_desc + a_off, b_desc + b_off, idesc);
   }
 }
-// D[tmem] (+)= A[tmem, 128 x 128 bf16 pairs] B with B an MN-major tile ([128 contraction rows][128 columns]): eight k-steps
-__device__ __forceinline__ void issue_tn(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, bool accumulate) {
+// D[tmem, 128 x 128] (+)= A[tmem, 128 x 64 as bf16 pairs] B with B a 64-row half read as the MN-major operand
+// ([64 contraction rows][128 columns]): four k-steps.  The lane threads leave A in two pieces, the pairs of a step's
+// columns 0..31 at a_tmem + 0..15 and those of columns 32..63 at a_tmem + 32..47.
+__device__ __forceinline__ void issue_tn(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_addr, bool accumulate) {
   constexpr uint32_t idesc = mv::um::idesc_bf16(BT, D, 0, 1);
+  const uint64_t b_desc = mv::um::smem_desc(b_addr, HALF_BYTES / 2, 1024);
   if (accumulate) mv::um::mma_ts<true>(d_tmem, a_tmem, b_desc, idesc);
   else mv::um::mma_ts<false>(d_tmem, a_tmem, b_desc, idesc);
 #pragma unroll
-  for (int k = 1; k < BT / 16; ++k) mv::um::mma_ts<true>(d_tmem, a_tmem + k * 8, b_desc + uint32_t((k * 2048) >> 4), idesc);
+  for (int k = 1; k < HB / 16; ++k)
+    mv::um::mma_ts<true>(d_tmem, a_tmem + (k >> 1) * 32 + (k & 1) * 8, b_desc + uint32_t((k * 2048) >> 4), idesc);
 }
-
-__device__ __forceinline__ uint64_t kmajor_desc(uint32_t addr) { return mv::um::smem_desc(addr, 16, 1024); }
-__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t addr) { return mv::um::smem_desc(addr, TILE_BYTES / 2, 1024); }
 
 struct Ctx {
   unsigned char* smem;
@@ -133,15 +146,16 @@ __device__ __forceinline__ bool setup(Ctx& c, unsigned char* smem, int32_t* stat
   c.smem = smem;
   c.smem_base = mv::smem_u32(smem);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 96);
-  int* abort_flag = reinterpret_cast<int*>(smem + OFF_BAR + 104);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + N_BARS * 8);
+  int* abort_flag = reinterpret_cast<int*>(smem + OFF_BAR + N_BARS * 8 + 8);
   c.br.fixed_full = mv::smem_u32(&bars[0]);
   c.br.full = mv::smem_u32(&bars[1]);
   c.br.empty = mv::smem_u32(&bars[1 + NSTAGE]);
   c.br.s_full = mv::smem_u32(&bars[1 + 2 * NSTAGE]);
-  c.br.p_full = mv::smem_u32(&bars[2 + 2 * NSTAGE]);
-  c.br.acc_done = mv::smem_u32(&bars[3 + 2 * NSTAGE]);
-  c.br.drained = mv::smem_u32(&bars[4 + 2 * NSTAGE]);
+  c.br.p_full = mv::smem_u32(&bars[3 + 2 * NSTAGE]);
+  c.br.acc_done = mv::smem_u32(&bars[5 + 2 * NSTAGE]);
+  c.br.drained = mv::smem_u32(&bars[7 + 2 * NSTAGE]);
+  static_assert(8 + 2 * NSTAGE <= N_BARS, "barrier table too small");
   if ((c.smem_base & 1023u) != 0) {  // the swizzle pattern is anchored at 1024-byte boundaries
     if (tid == 0) atomicExch(status, int(MV_ERR_UNSUPPORTED));
     return false;
@@ -153,9 +167,11 @@ __device__ __forceinline__ bool setup(Ctx& c, unsigned char* smem, int32_t* stat
       mv::mbar_init(c.br.full + 8 * i, 1);
       mv::mbar_init(c.br.empty + 8 * i, 1);  // one tcgen05.commit
     }
-    mv::mbar_init(c.br.s_full, 1);     // one tcgen05.commit
-    mv::mbar_init(c.br.p_full, 128);   // the 128 lane threads
-    mv::mbar_init(c.br.acc_done, 1);   // one tcgen05.commit
+    for (int b = 0; b < 2; ++b) {
+      mv::mbar_init(c.br.s_full + 8 * b, 1);     // one tcgen05.commit
+      mv::mbar_init(c.br.p_full + 8 * b, 256);   // the 256 lane threads
+      mv::mbar_init(c.br.acc_done + 8 * b, 1);   // one tcgen05.commit
+    }
     mv::mbar_init(c.br.drained, 1);
     mv::mbar_fence_init();
     mv::fence_proxy_async();
@@ -206,7 +222,11 @@ __global__ void __launch_bounds__(128) delta_kernel(const bf16* __restrict__ out
 }
 
 // ---- dQ ------------------------------------------------------------------------------------------------------
-// tensor memory: S at +0 (dS written back over its first 64 columns), dP at +128, dQ accumulator at +256
+// The visible keys are taken in steps of 64, one ring stage (K, V halves) per step, alternating between two score
+// buffers in tensor memory, so that the tensor cores compute the next step's S and dP while the lane threads turn this
+// one's into dS.  Buffer b: S at 128 b (dS written back over its columns 0..15 and 32..47), dP at 128 b + 64; the dQ
+// accumulator at +256.
+
 __global__ void __launch_bounds__(NTHREADS, 1) dq_kernel(const BwdArgs a, const __grid_constant__ CUtensorMap tm_q,
                                                          const __grid_constant__ CUtensorMap tm_do, const __grid_constant__ CUtensorMap tm_k,
                                                          const __grid_constant__ CUtensorMap tm_v) {
@@ -231,91 +251,98 @@ __global__ void __launch_bounds__(NTHREADS, 1) dq_kernel(const BwdArgs a, const 
         const int st = e % NSTAGE;
         ok = w.wait(br.empty + 8 * st, ((e / NSTAGE) & 1) ^ 1);
         if (!ok) break;
-        mv::mbar_arrive_expect_tx(br.full + 8 * st, 2 * TILE_BYTES);
-        load_tile(c.smem_base + OFF_RING + st * 2 * TILE_BYTES, &tm_k, kvh * D, start, br.full + 8 * st);
-        load_tile(c.smem_base + OFF_RING + st * 2 * TILE_BYTES + TILE_BYTES, &tm_v, kvh * D, start, br.full + 8 * st);
+        mv::mbar_arrive_expect_tx(br.full + 8 * st, STAGE_BYTES);
+        load_half(c.smem_base + OFF_RING + st * STAGE_BYTES, &tm_k, kvh * D, start, br.full + 8 * st);
+        load_half(c.smem_base + OFF_RING + st * STAGE_BYTES + HALF_BYTES, &tm_v, kvh * D, start, br.full + 8 * st);
         ++e;
       }
       if (!ok) drain_producer(c, e);
     }
   } else if (warp == 1) {
-    // issuer: the whole warp walks, one elected lane issues
+    // issuer: the whole warp walks, one elected lane issues.  The dQ product of a step is issued after the scores of
+    // the step behind it, so the tensor cores always have the next scores queued while the lane threads work.
     const bool lead = mv::um::elect_one();
     Walk it(a.ranges + qt.range_begin, qt.range_count, q_last);
-    const uint64_t q_desc = kmajor_desc(c.smem_base + OFF_FIXED), do_desc = kmajor_desc(c.smem_base + OFF_FIXED + TILE_BYTES);
+    const uint32_t q_addr = c.smem_base + OFF_FIXED, do_addr = q_addr + TILE_BYTES;
     int start, n, cz, e = 0;
+    // step f's dQ product: after the lane threads have left dS in buffer f & 1; it frees the buffer and the stage
+    auto finish = [&](int f) -> bool {
+      const int b = f & 1;
+      if (!w.wait(br.p_full + 8 * b, (f >> 1) & 1)) return false;
+      mv::um::fence_after();
+      if (lead) {
+        issue_tn(c.tmem + 256, c.tmem + 128 * b, c.smem_base + OFF_RING + (f % NSTAGE) * STAGE_BYTES, f > 0);  // dQ += dS K
+        mv::um::commit(br.acc_done + 8 * b);
+        mv::um::commit(br.empty + 8 * (f % NSTAGE));
+      }
+      __syncwarp();
+      return true;
+    };
     bool ok = w.wait(br.fixed_full, 0);
     while (ok && it.next(start, n, cz)) {
-      const int st = e % NSTAGE;
-      const uint32_t kt = c.smem_base + OFF_RING + st * 2 * TILE_BYTES, vt = kt + TILE_BYTES;
+      const int st = e % NSTAGE, b = e & 1;
+      const uint32_t kh = c.smem_base + OFF_RING + st * STAGE_BYTES, vh = kh + HALF_BYTES;
       ok = w.wait(br.full + 8 * st, (e / NSTAGE) & 1);
-      // the previous tile's dQ product has read dS (the S columns) before they are overwritten
-      if (ok && e > 0) ok = w.wait(br.acc_done, (e - 1) & 1);
+      // the dQ product two steps back has read dS from this buffer before the new scores overwrite it
+      if (ok && e >= 2) ok = w.wait(br.acc_done + 8 * b, ((e >> 1) - 1) & 1);
       if (!ok) break;
       mv::um::fence_after();
       if (lead) {
-        issue_nt(c.tmem, q_desc, kmajor_desc(kt));          // S = Q K^T
-        issue_nt(c.tmem + 128, do_desc, kmajor_desc(vt));   // dP = dO V^T
-        mv::um::commit(br.s_full);
+        issue_nt(c.tmem + 128 * b, q_addr, kh);         // S = Q K^T
+        issue_nt(c.tmem + 128 * b + HB, do_addr, vh);   // dP = dO V^T
+        mv::um::commit(br.s_full + 8 * b);
       }
-      ok = w.wait(br.p_full, e & 1);
-      if (!ok) break;
-      mv::um::fence_after();
-      if (lead) {
-        issue_tn(c.tmem + 256, c.tmem, mnmajor_desc(kt), e > 0);  // dQ += dS K
-        mv::um::commit(br.acc_done);
-        mv::um::commit(br.empty + 8 * st);
-      }
+      __syncwarp();
+      if (e > 0) ok = finish(e - 1);
       ++e;
     }
+    if (ok && e > 0) ok = finish(e - 1);
     if (w.aborted()) drain_issuer(c, lead);
   } else {
-    // lane threads: thread on tensor-memory lane r owns query row r of the tile
-    const int r = (warp & 3) * 32 + lane;
+    // lane threads: the two threads on tensor-memory lane r own query row r of the tile, 32 columns of a step each
+    const int r = (warp & 3) * 32 + lane, ch = (warp - 2) >> 2;
     const uint32_t lane_base = c.tmem + (uint32_t((warp & 3) * 32) << 16);
     const int qi = qt.q_start + r, qc = qt.causal_base + r;
     const bool row_ok = r < qt.q_len;
     const float lse = row_ok ? a.lse[int64_t(qi) * a.Hq + head] : 0.f;
-    const float dl = row_ok ? a.delta[int64_t(qi) * a.Hq + head] : 0.f;
+    const float dl = row_ok ? a.delta[int64_t(qi) * a.Hq + head] * a.scale : 0.f;
     Walk it(a.ranges + qt.range_begin, qt.range_count, q_last);
     int start, n, cz, e = 0;
     bool ok = true;
     while (it.next(start, n, cz)) {
-      ok = w.warp_wait(br.s_full, e & 1);
+      const int b = e & 1;
+      const int lim = row_ok ? (cz ? min(n, qc - start + 1) : n) : 0;  // keys [0, lim) of the step are visible to this row
+      ok = w.warp_wait(br.s_full + 8 * b, (e >> 1) & 1);
       if (!ok) break;
       mv::um::fence_after();
-      const int lim = row_ok ? (cz ? min(n, qc - start + 1) : n) : 0;  // keys [0, lim) of the tile are visible to this row
-#pragma unroll 1
-      for (int cb = 0; cb < BT / 32; ++cb) {
-        uint32_t s[32], dp[32], ds[16];
-        mv::um::ld32(lane_base + cb * 32, s);
-        mv::um::ld32(lane_base + 128 + cb * 32, dp);
-        mv::um::wait_ld();
+      const uint32_t base = lane_base + 128 * b + ch * 32;
+      const int j0 = ch * 32;
+      uint32_t s[32], dp[32], ds[16];
+      mv::um::ld32(base, s);
+      mv::um::ld32(base + HB, dp);
+      mv::um::wait_ld();
 #pragma unroll
-        for (int k = 0; k < 32; k += 2) {
-          const int j = cb * 32 + k;
-          const float p0 = j < lim ? mv::fast_exp2(fmaf(__uint_as_float(s[k]), a.scale_log2, -lse)) : 0.f;
-          const float p1 = j + 1 < lim ? mv::fast_exp2(fmaf(__uint_as_float(s[k + 1]), a.scale_log2, -lse)) : 0.f;
-          const float d0 = j < lim ? p0 * (__uint_as_float(dp[k]) - dl) * a.scale : 0.f;
-          const float d1 = j + 1 < lim ? p1 * (__uint_as_float(dp[k + 1]) - dl) * a.scale : 0.f;
-          ds[k >> 1] = mv::pack_bf16(d0, d1);
-        }
-        // dS over S in place: columns 2c, 2c+1 -> packed column c (chunk cb fills packed columns 16 cb .. 16 cb + 15, which
-        // lie inside the S columns already read: 16 cb + 15 < 32 cb + 32)
-        mv::um::st16(lane_base + cb * 16, ds);
+      for (int k = 0; k < 32; k += 2) {
+        // a masked pair has P = 0, and with it dS = 0: dP and delta are finite whatever the padding holds
+        const float p0 = j0 + k < lim ? mv::fast_exp2(fmaf(__uint_as_float(s[k]), a.scale_log2, -lse)) : 0.f;
+        const float p1 = j0 + k + 1 < lim ? mv::fast_exp2(fmaf(__uint_as_float(s[k + 1]), a.scale_log2, -lse)) : 0.f;
+        const float d0 = p0 * fmaf(__uint_as_float(dp[k]), a.scale, -dl);
+        const float d1 = p1 * fmaf(__uint_as_float(dp[k + 1]), a.scale, -dl);
+        ds[k >> 1] = mv::pack_bf16(d0, d1);
       }
+      mv::um::st16(base, ds);  // over the thread's own S columns, which it has read
       mv::um::wait_st();
       mv::um::fence_before();
-      mv::mbar_arrive(br.p_full);
+      mv::mbar_arrive(br.p_full + 8 * b);
       ++e;
     }
-    if (ok && e > 0 && w.warp_wait(br.acc_done, (e - 1) & 1)) {
+    if (ok && e > 0 && w.warp_wait(br.acc_done + 8 * ((e - 1) & 1), ((e - 1) >> 1) & 1)) {
       mv::um::fence_after();
-      bf16* dst = a.dq + (int64_t(qi) * a.Hq + head) * D;
+      bf16* dst = a.dq + (int64_t(qi) * a.Hq + head) * D + ch * 64;
 #pragma unroll 1
-      for (int cb = 0; cb < D / 32; ++cb) {
+      for (int cb = 0; cb < 2; ++cb) {
         uint32_t o[32];
-        mv::um::ld32(lane_base + 256 + cb * 32, o);
+        mv::um::ld32(lane_base + 256 + ch * 64 + cb * 32, o);
         mv::um::wait_ld();
         if (row_ok) {
 #pragma unroll
@@ -335,9 +362,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) dq_kernel(const BwdArgs a, const 
 }
 
 // ---- dK, dV --------------------------------------------------------------------------------------------------
-// tensor memory: S^T at +0 (P^T written back over its first 64 columns), dP^T at +128 (dS^T over its first 64 columns),
-// dV accumulator at +256, dK accumulator at +384.  A stage of the ring is one (128-query sub-tile, query head): Q, dO
-// and the queries' lse and delta.
+// A step is (64 queries that see the tile's node, one query head of the group): one ring stage holds the Q and dO
+// halves and the queries' lse and delta.  Two score buffers as in dq_kernel.  Buffer b: S^T at 128 b (P^T written
+// back over its columns 0..15 and 32..47), dP^T at 128 b + 64 (dS^T likewise); the dV accumulator at +256, dK at +384.
 __global__ void __launch_bounds__(NTHREADS, 1) dkv_kernel(const BwdArgs a, const __grid_constant__ CUtensorMap tm_q,
                                                           const __grid_constant__ CUtensorMap tm_do, const __grid_constant__ CUtensorMap tm_k,
                                                           const __grid_constant__ CUtensorMap tm_v) {
@@ -350,7 +377,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) dkv_kernel(const BwdArgs a, const
   const Bars& br = c.br;
   const Waiter& w = c.w;
   constexpr int NO_CUT = 0x3fffffff;
-  float* vec = reinterpret_cast<float*>(smem + OFF_VEC);  // [stage][lse 128 | delta 128]
+  float* vec = reinterpret_cast<float*>(smem + OFF_VEC);  // [stage][lse 64 | delta * scale 64]
   if (warp == 0) {
     // producer: lane 0 issues the tile copies; all lanes fetch the stage's lse / delta vectors with plain loads
     if (lane == 0) {
@@ -368,17 +395,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) dkv_kernel(const BwdArgs a, const
         if (lane == 0) go = w.wait(br.empty + 8 * st, ((e / NSTAGE) & 1) ^ 1) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, go, 0) != 0;
         if (!ok) break;
-        float* vs = vec + st * 2 * BT;
-        for (int x = lane; x < BT; x += 32) {
+        float* vs = vec + st * 2 * HB;
+        for (int x = lane; x < HB; x += 32) {
           const bool in = x < n;
           vs[x] = in ? a.lse[int64_t(start + x) * a.Hq + head] : 0.f;
-          vs[BT + x] = in ? a.delta[int64_t(start + x) * a.Hq + head] : 0.f;
+          vs[HB + x] = in ? a.delta[int64_t(start + x) * a.Hq + head] * a.scale : 0.f;
         }
         __syncwarp();
         if (lane == 0) {
-          mv::mbar_arrive_expect_tx(br.full + 8 * st, 2 * TILE_BYTES);  // releases the vector stores above
-          load_tile(c.smem_base + OFF_RING + st * 2 * TILE_BYTES, &tm_q, head * D, start, br.full + 8 * st);
-          load_tile(c.smem_base + OFF_RING + st * 2 * TILE_BYTES + TILE_BYTES, &tm_do, head * D, start, br.full + 8 * st);
+          mv::mbar_arrive_expect_tx(br.full + 8 * st, STAGE_BYTES);  // releases the vector stores above
+          load_half(c.smem_base + OFF_RING + st * STAGE_BYTES, &tm_q, head * D, start, br.full + 8 * st);
+          load_half(c.smem_base + OFF_RING + st * STAGE_BYTES + HALF_BYTES, &tm_do, head * D, start, br.full + 8 * st);
         }
       }
     }
@@ -387,37 +414,47 @@ __global__ void __launch_bounds__(NTHREADS, 1) dkv_kernel(const BwdArgs a, const
   } else if (warp == 1) {
     const bool lead = mv::um::elect_one();
     Walk it(a.ranges + kt.range_begin, kt.range_count, NO_CUT);
-    const uint64_t k_desc = kmajor_desc(c.smem_base + OFF_FIXED), v_desc = kmajor_desc(c.smem_base + OFF_FIXED + TILE_BYTES);
+    const uint32_t k_addr = c.smem_base + OFF_FIXED, v_addr = k_addr + TILE_BYTES;
     int start, n, cz, e = 0;
+    // step f's accumulating products: after the lane threads have left P^T and dS^T in buffer f & 1
+    auto finish = [&](int f) -> bool {
+      const int b = f & 1;
+      if (!w.wait(br.p_full + 8 * b, (f >> 1) & 1)) return false;
+      mv::um::fence_after();
+      if (lead) {
+        const uint32_t qh = c.smem_base + OFF_RING + (f % NSTAGE) * STAGE_BYTES, doh = qh + HALF_BYTES;
+        issue_tn(c.tmem + 256, c.tmem + 128 * b, doh, f > 0);      // dV += P^T dO
+        issue_tn(c.tmem + 384, c.tmem + 128 * b + HB, qh, f > 0);  // dK += dS^T Q
+        mv::um::commit(br.acc_done + 8 * b);
+        mv::um::commit(br.empty + 8 * (f % NSTAGE));
+      }
+      __syncwarp();
+      return true;
+    };
     bool ok = w.wait(br.fixed_full, 0);
     while (ok && it.next(start, n, cz)) {
       for (int hg = 0; hg < a.G && ok; ++hg, ++e) {
-        const int st = e % NSTAGE;
-        const uint32_t qtile = c.smem_base + OFF_RING + st * 2 * TILE_BYTES, dotile = qtile + TILE_BYTES;
+        const int st = e % NSTAGE, b = e & 1;
+        const uint32_t qh = c.smem_base + OFF_RING + st * STAGE_BYTES, doh = qh + HALF_BYTES;
         ok = w.wait(br.full + 8 * st, (e / NSTAGE) & 1);
-        if (ok && e > 0) ok = w.wait(br.acc_done, (e - 1) & 1);  // the previous products have read P^T and dS^T
+        // the products two steps back have read P^T and dS^T from this buffer before the new scores overwrite them
+        if (ok && e >= 2) ok = w.wait(br.acc_done + 8 * b, ((e >> 1) - 1) & 1);
         if (!ok) break;
         mv::um::fence_after();
         if (lead) {
-          issue_nt(c.tmem, k_desc, kmajor_desc(qtile));          // S^T = K Q^T
-          issue_nt(c.tmem + 128, v_desc, kmajor_desc(dotile));   // dP^T = V dO^T
-          mv::um::commit(br.s_full);
+          issue_nt(c.tmem + 128 * b, k_addr, qh);         // S^T = K Q^T
+          issue_nt(c.tmem + 128 * b + HB, v_addr, doh);   // dP^T = V dO^T
+          mv::um::commit(br.s_full + 8 * b);
         }
-        ok = w.wait(br.p_full, e & 1);
-        if (!ok) break;
-        mv::um::fence_after();
-        if (lead) {
-          issue_tn(c.tmem + 256, c.tmem, mnmajor_desc(dotile), e > 0);       // dV += P^T dO
-          issue_tn(c.tmem + 384, c.tmem + 128, mnmajor_desc(qtile), e > 0);  // dK += dS^T Q
-          mv::um::commit(br.acc_done);
-          mv::um::commit(br.empty + 8 * st);
-        }
+        __syncwarp();
+        if (e > 0) ok = finish(e - 1);
       }
     }
+    if (ok && e > 0) ok = finish(e - 1);
     if (w.aborted()) drain_issuer(c, lead);
   } else {
-    // lane threads: thread on tensor-memory lane r owns key r of the tile
-    const int r = (warp & 3) * 32 + lane;
+    // lane threads: the two threads on tensor-memory lane r own key r of the tile, 32 queries of a step each
+    const int r = (warp & 3) * 32 + lane, ch = (warp - 2) >> 2;
     const uint32_t lane_base = c.tmem + (uint32_t((warp & 3) * 32) << 16);
     const bool key_ok = r < kt.q_len;
     const int kc = kt.causal_base + r;  // the key's flattened index
@@ -425,50 +462,56 @@ __global__ void __launch_bounds__(NTHREADS, 1) dkv_kernel(const BwdArgs a, const
     int start, n, cz, e = 0;
     bool ok = true;
     while (ok && it.next(start, n, cz)) {
+      // queries [first, n) of the step see this key: all valid ones, or (own node) those not before the key
+      const int first = key_ok ? (cz ? max(0, kc - start) : 0) : n;
       for (int hg = 0; hg < a.G && ok; ++hg, ++e) {
-        const int st = e % NSTAGE;
+        const int st = e % NSTAGE, b = e & 1;
         ok = w.warp_wait(br.full + 8 * st, (e / NSTAGE) & 1);  // the stage's lse / delta vectors are visible
-        if (ok) ok = w.warp_wait(br.s_full, e & 1);
+        if (ok) ok = w.warp_wait(br.s_full + 8 * b, (e >> 1) & 1);
         if (!ok) break;
         mv::um::fence_after();
-        const float* vs = vec + st * 2 * BT;
-        // queries [first, n) of the sub-tile see this key: all valid ones, or (own node) those not before the key
-        const int first = key_ok ? (cz ? max(0, kc - start) : 0) : n;
-#pragma unroll 1
-        for (int cb = 0; cb < BT / 32; ++cb) {
-          uint32_t s[32], dp[32], pt[16], ds[16];
-          mv::um::ld32(lane_base + cb * 32, s);
-          mv::um::ld32(lane_base + 128 + cb * 32, dp);
-          mv::um::wait_ld();
+        const float4* vl = reinterpret_cast<const float4*>(vec + st * 2 * HB + ch * 32);
+        const float4* vd = reinterpret_cast<const float4*>(vec + st * 2 * HB + HB + ch * 32);
+        const uint32_t base = lane_base + 128 * b + ch * 32;
+        const int j0 = ch * 32;
+        uint32_t s[32], dp[32], pt[16], ds[16];
+        mv::um::ld32(base, s);
+        mv::um::ld32(base + HB, dp);
+        mv::um::wait_ld();
 #pragma unroll
-          for (int k = 0; k < 32; k += 2) {
-            const int j = cb * 32 + k;
-            const bool v0 = j >= first && j < n, v1 = j + 1 >= first && j + 1 < n;
-            const float p0 = v0 ? mv::fast_exp2(fmaf(__uint_as_float(s[k]), a.scale_log2, -vs[j])) : 0.f;
-            const float p1 = v1 ? mv::fast_exp2(fmaf(__uint_as_float(s[k + 1]), a.scale_log2, -vs[j + 1])) : 0.f;
-            const float d0 = v0 ? p0 * (__uint_as_float(dp[k]) - vs[BT + j]) * a.scale : 0.f;
-            const float d1 = v1 ? p1 * (__uint_as_float(dp[k + 1]) - vs[BT + j + 1]) * a.scale : 0.f;
-            pt[k >> 1] = mv::pack_bf16(p0, p1);
-            ds[k >> 1] = mv::pack_bf16(d0, d1);
+        for (int k = 0; k < 32; k += 4) {
+          const float4 l4 = vl[k >> 2], d4 = vd[k >> 2];
+          const float ls[4] = {l4.x, l4.y, l4.z, l4.w}, dl[4] = {d4.x, d4.y, d4.z, d4.w};
+          float p[4], d[4];
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            const int j = j0 + k + x;
+            // a masked pair has P = 0, and with it dS = 0: dP and delta are finite whatever the padding holds
+            p[x] = (j >= first && j < n) ? mv::fast_exp2(fmaf(__uint_as_float(s[k + x]), a.scale_log2, -ls[x])) : 0.f;
+            d[x] = p[x] * fmaf(__uint_as_float(dp[k + x]), a.scale, -dl[x]);
           }
-          mv::um::st16(lane_base + cb * 16, pt);
-          mv::um::st16(lane_base + 128 + cb * 16, ds);
+          pt[k >> 1] = mv::pack_bf16(p[0], p[1]);
+          pt[(k >> 1) + 1] = mv::pack_bf16(p[2], p[3]);
+          ds[k >> 1] = mv::pack_bf16(d[0], d[1]);
+          ds[(k >> 1) + 1] = mv::pack_bf16(d[2], d[3]);
         }
+        mv::um::st16(base, pt);       // over the thread's own S^T columns, which it has read
+        mv::um::st16(base + HB, ds);  // and over its own dP^T columns
         mv::um::wait_st();
         mv::um::fence_before();
-        mv::mbar_arrive(br.p_full);
+        mv::mbar_arrive(br.p_full + 8 * b);
       }
     }
-    if (ok && e > 0 && w.warp_wait(br.acc_done, (e - 1) & 1)) {
+    if (ok && e > 0 && w.warp_wait(br.acc_done + 8 * ((e - 1) & 1), ((e - 1) >> 1) & 1)) {
       mv::um::fence_after();
       const int64_t tok = int64_t(kt.q_start + r);
 #pragma unroll 1
       for (int which = 0; which < 2; ++which) {
-        bf16* dst = (which == 0 ? a.dv : a.dk) + (tok * a.Hkv + kvh) * D;
+        bf16* dst = (which == 0 ? a.dv : a.dk) + (tok * a.Hkv + kvh) * D + ch * 64;
 #pragma unroll 1
-        for (int cb = 0; cb < D / 32; ++cb) {
+        for (int cb = 0; cb < 2; ++cb) {
           uint32_t o[32];
-          mv::um::ld32(lane_base + 256 + which * 128 + cb * 32, o);
+          mv::um::ld32(lane_base + 256 + which * 128 + ch * 64 + cb * 32, o);
           mv::um::wait_ld();
           if (key_ok) {
 #pragma unroll
@@ -523,10 +566,10 @@ extern "C" mv_status mv_dag_prefill_attn_bwd(const mv_plan* P, const mv_attn_geo
   BwdMaps* tm = cache.find(key);
   if (!tm) {
     tm = cache.claim(key);
-    if (!mv::make_tmap_bf16_2d(&tm->tm_q, q_rot, uint64_t(T), uint64_t(g->n_q_heads) * D, BT) ||
-        !mv::make_tmap_bf16_2d(&tm->tm_do, dout, uint64_t(T), uint64_t(g->n_q_heads) * D, BT) ||
-        !mv::make_tmap_bf16_2d(&tm->tm_k, k_rot, uint64_t(T), uint64_t(g->n_kv_heads) * D, BT) ||
-        !mv::make_tmap_bf16_2d(&tm->tm_v, v, uint64_t(T), uint64_t(g->n_kv_heads) * D, BT)) {
+    if (!mv::make_tmap_bf16_2d(&tm->tm_q, q_rot, uint64_t(T), uint64_t(g->n_q_heads) * D, HB) ||
+        !mv::make_tmap_bf16_2d(&tm->tm_do, dout, uint64_t(T), uint64_t(g->n_q_heads) * D, HB) ||
+        !mv::make_tmap_bf16_2d(&tm->tm_k, k_rot, uint64_t(T), uint64_t(g->n_kv_heads) * D, HB) ||
+        !mv::make_tmap_bf16_2d(&tm->tm_v, v, uint64_t(T), uint64_t(g->n_kv_heads) * D, HB)) {
       cache.drop();
       return MV_ERR_CUDA;
     }
