@@ -6,15 +6,22 @@
 //   dV = P^T dO,  dP = dO V^T,  dS = P o (dP - delta),  delta_i = sum_j P_ij dP_ij = <dO_i, O_i>,
 //   dQ = scale * dS K,  dK = scale * dS^T Q,
 // a KV head collecting dK and dV from every query head of its group.  P is rebuilt from the scores and the row's
-// log-sum-exp that the forward kernel leaves (no second softmax pass).  Three kernels:
-//   delta_kernel     delta[i][h] = <dO[i][h], O[i][h]>                                   (elementwise, one warp per row-head)
-//   dq_kernel        one CTA per (query tile, query head): walks the KV tiles the tile's node may see, exactly the
-//                    forward's walk: S = Q K^T and dP = dO V^T into tensor memory, one thread per query row turns them
-//                    into dS (bf16, written back over S), dQ += dS K with K as the MN-major operand.
-//   dkv_kernel       one CTA per (key tile, KV head): walks the transposed lists (the runs of queries that see the tile's
-//                    node; its own node causally) for every query head of the group: S^T = K Q^T and dP^T = V dO^T into
-//                    tensor memory (a lane is a key, a column a query), one thread per key builds P^T and dS^T (bf16,
-//                    written back in place), dV += P^T dO and dK += dS^T Q with dO and Q as MN-major operands.
+// log-sum-exp that the forward kernel leaves (no second softmax pass).  The kernels:
+//   delta_kernel   delta[i][h] = <dO[i][h], O[i][h]>                                   (elementwise, one warp per row-head)
+//   bwd_kernel<DQ> one CTA per (query tile, query head): walks the KV tiles the tile's node may see, exactly the
+//                  forward's walk: S = Q K^T and dP = dO V^T into tensor memory, the lane threads turn them into dS
+//                  (bf16, written back over S), dQ += dS K with K as the MN-major operand.
+//   bwd_kernel<DK> one CTA per (key tile, KV head): walks the transposed lists (the runs of queries that see the tile's
+//                  node; its own node causally) for every query head of the group: S^T = K Q^T and dP^T = V dO^T (a
+//                  lane is a key, a column a query), dS^T written back over S^T, dK += dS^T Q with Q MN-major.
+//   bwd_kernel<DV> the same walk: S^T = K Q^T, P^T written back over S^T, dV += P^T dO with dO MN-major.
+// Every product is 128 x 128 x 16 per instruction, the shape at which the tensor cores run at their full rate
+// (measured: a 128 x 64 x 16 instruction takes three quarters of the time of a 128 x 128 x 16 one).  Tensor memory
+// holds two score buffers (three in DV), one dP buffer and the accumulator: while the lane threads work on step e the
+// tensor cores run the accumulating product of step e - 1 and the scores of step e + 1.  The lane threads copy their
+// part of dP to registers first and hand the dP buffer back at once, which is what lets one dP buffer do.  dK and dV
+// come from separate CTAs because two accumulators would leave tensor memory for one score buffer only, and the
+// products and the elementwise work would then run in turn.
 // Masked pairs get P = 0 by selection, so nothing depends on what the padding rows or columns of a ragged tile hold.
 // No atomics: every output element is written by exactly one CTA, and the result is deterministic.
 // Every mbarrier wait is bounded; after one ran out a role issues nothing further, the producer and the issuer wait
@@ -30,26 +37,34 @@ using bf16 = __nv_bfloat16;
 constexpr int D = 128;
 constexpr int BT = 128;                 // rows of every tile (queries or keys)
 constexpr int TILE_BYTES = BT * D * 2;  // 32 KB: [2 column blocks][128 rows][128 B]
-constexpr int HB = 64;                  // a step is one 64-column half of a 128 x 128 score tile
-constexpr int HALF_BYTES = HB * D * 2;  // 16 KB: [2 column blocks][64 rows][128 B]
-constexpr int NTHREADS = 320;           // warp 0 producer, warp 1 issuer, warps 2..9: two threads per tensor-memory lane,
-                                        // each taking 32 of a step's 64 columns
-constexpr int OFF_FIXED = 0;            // two 128-row tiles that stay for the whole CTA (dq: Q, dO; dkv: K, V)
-constexpr int OFF_RING = 2 * TILE_BYTES;  // stages of two 64-row halves (dq: K, V; dkv: Q, dO), one stage per step
-constexpr int NSTAGE = 4;
-constexpr int STAGE_BYTES = 2 * HALF_BYTES;
-constexpr int OFF_VEC = OFF_RING + NSTAGE * STAGE_BYTES;  // dkv: per stage lse[64], delta[64] of the step's queries
-constexpr int OFF_BAR = OFF_VEC + NSTAGE * 2 * HB * 4;
-constexpr int N_BARS = 2 + 2 * NSTAGE + 6;
+constexpr int NTHREADS = 384;           // warp 0 producer, warp 1 issuer of the scores, warp 2 issuer of the accumulating
+                                        // products, warp 3 idle, warps 4..11: two threads per tensor-memory lane, each
+                                        // taking 64 of a step's 128 columns
+constexpr int NLANE_THREADS = 256;
+enum Mode { DQ = 0, DK = 1, DV = 2 };
+constexpr int NLONG = 3, NSHORT = 2;    // ring slots: tiles needed until the accumulating product / only for the scores
+constexpr int OFF_FIXED = 0;            // two tiles that stay for the whole CTA (DQ: Q, dO; DK: K, V; DV: K)
+constexpr int OFF_LONG = 2 * TILE_BYTES;                   // DQ: K; DK: Q; DV: dO
+constexpr int OFF_SHORT = OFF_LONG + NLONG * TILE_BYTES;   // DQ: V; DK: dO; DV: Q
+constexpr int OFF_VEC = OFF_SHORT + NSHORT * TILE_BYTES;   // DK, DV: two slots of -lse[128], -scale * delta[128] of a step's queries
+constexpr int OFF_BAR = OFF_VEC + 2 * 2 * BT * 4;
+constexpr int N_BARS = 1 + 2 * NLONG + 2 * NSHORT + 3 + 1 + 3 + 3 + 2 + 1;
 constexpr int SMEM_BYTES = OFF_BAR + N_BARS * 8 + 16;
+static_assert(SMEM_BYTES <= 232448, "over the shared memory of a CTA");
+// tensor memory columns
+constexpr uint32_t TM_S = 0;      // score buffers at 0, 128 (and 256 in DV)
+constexpr uint32_t TM_DP = 256;   // dP (DQ, DK)
+constexpr uint32_t TM_ACC = 384;  // dQ / dK / dV accumulator
 
 struct BwdArgs {
-  const mv::QTile* tiles;     // dq: query tiles; dkv: key tiles
-  const mv::KvRange* ranges;  // dq: key ranges;  dkv: query ranges
-  const float* lse;           // [T][Hq] log2-domain log-sum-exp of the forward
-  const float* delta;         // [T][Hq]
-  bf16* dq;                   // [T][Hq][D]
-  bf16* dk;                   // [T][Hkv][D]
+  const mv::QTile* q_tiles;    // query tiles and their key ranges (DQ)
+  const mv::KvRange* kv_ranges;
+  const mv::QTile* k_tiles;    // key tiles and the query ranges that see them (DK, DV)
+  const mv::KvRange* q_ranges;
+  const float* lse;            // [T][Hq] log2-domain log-sum-exp of the forward
+  const float* delta;          // [T][Hq]
+  bf16* dq;                    // [T][Hq][D]
+  bf16* dk;                    // [T][Hkv][D]
   bf16* dv;
   int32_t* status;
   int Hq, Hkv, G, T;
@@ -57,14 +72,15 @@ struct BwdArgs {
 };
 
 struct Bars {
-  // full / empty: NSTAGE consecutive barriers; s_full / p_full / acc_done: one per score buffer (two)
-  uint32_t fixed_full, full, empty, s_full, p_full, acc_done, drained;
+  // lfull / lempty: NLONG consecutive barriers; sfull / sempty: NSHORT; s_full / p_full / acc_done: one per score buffer
+  uint32_t fixed_full, lfull, lempty, sfull, sempty, s_full, dp_free, p_full, acc_done, drained, vec_ready;  // drained: two, one per issuer
 };
 
 struct Waiter {
   volatile int* abort;
   int32_t* status;
   __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
+    if (mv::mbar_try_wait(bar, parity)) return !*abort;
     if (*abort) return false;
     if (!mv::mbar_wait_bounded(bar, parity, 2000000000ull, abort)) {
       if (!*abort) atomicExch(status, int(MV_ERR_TIMEOUT));
@@ -77,61 +93,66 @@ struct Waiter {
   __device__ __forceinline__ bool aborted() const { return *abort != 0; }
 };
 
-// 64-row steps of a tile's ranges, in table order.  FWD walk (dq): a causal range ends after the tile's last query.
-// Transposed walk (dkv): a causal range starts at the tile's first key and is not cut.
-struct Walk {
+// The steps of a CTA, in table order.  DQ: the 128-key sub-tiles of the query tile's ranges, a causal range ending
+// after the tile's last query.  DK, DV: the 128-query sub-tiles of the key tile's transposed ranges (a causal range
+// starts at the tile's first key and is not cut), each taken once per query head of the group.
+struct Steps {
   const mv::KvRange* rg;
-  int n_ranges, last_causal;  // last_causal: last index a causal range may reach (dq), or a very large number (dkv)
-  int ri = 0, pos = 0, end = 0, causal = 0;
-  __device__ Walk(const mv::KvRange* r, int n, int lc) : rg(r), n_ranges(n), last_causal(lc) {}
-  __device__ bool next(int& start, int& n, int& c) {
-    while (pos >= end) {
-      if (ri >= n_ranges) return false;
-      const mv::KvRange r = rg[ri++];
-      pos = r.kv_start;
-      end = r.kv_start + r.kv_len;
-      causal = r.causal;
-      if (causal) end = min(end, last_causal + 1);
+  int n_ranges, last_causal, heads;
+  int ri = 0, pos = 0, end = 0, causal = 0, hg = 0, cur_start = 0, cur_n = 0;
+  __device__ Steps(const mv::KvRange* r, int n, int lc, int h) : rg(r), n_ranges(n), last_causal(lc), heads(h), hg(h) {}
+  __device__ bool next(int& start, int& n, int& c, int& head_in_group) {
+    if (hg + 1 < heads) {
+      ++hg;
+    } else {
+      while (pos >= end) {
+        if (ri >= n_ranges) return false;
+        const mv::KvRange r = rg[ri++];
+        pos = r.kv_start;
+        end = r.kv_start + r.kv_len;
+        causal = r.causal;
+        if (causal) end = min(end, last_causal + 1);
+      }
+      cur_start = pos;
+      cur_n = min(BT, end - pos);
+      pos += BT;
+      hg = 0;
     }
-    start = pos;
-    n = min(HB, end - pos);
+    start = cur_start;
+    n = cur_n;
     c = causal;
-    pos += HB;
+    head_in_group = hg;
     return true;
   }
 };
 
-// every tensor map's box is 64 columns x 64 rows (8 KB)
+// every tensor map's box is 64 columns x 128 rows (16 KB)
 __device__ __forceinline__ void load_tile(uint32_t dst, const CUtensorMap* tm, int col, int row, uint32_t bar) {
-  for (int cb = 0; cb < 2; ++cb)
-    for (int rh = 0; rh < 2; ++rh) mv::tma_load_2d(dst + cb * (TILE_BYTES / 2) + rh * (HALF_BYTES / 2), tm, col + cb * 64, row + rh * HB, bar);
-}
-__device__ __forceinline__ void load_half(uint32_t dst, const CUtensorMap* tm, int col, int row, uint32_t bar) {
-  for (int cb = 0; cb < 2; ++cb) mv::tma_load_2d(dst + cb * (HALF_BYTES / 2), tm, col + cb * 64, row, bar);
+  for (int cb = 0; cb < 2; ++cb) mv::tma_load_2d(dst + cb * (TILE_BYTES / 2), tm, col + cb * 64, row, bar);
 }
 
-// D[tmem, 128 x 64] = A B^T, A a K-major 128-row tile, B a K-major 64-row half: eight k-steps over head_dim
+// D[tmem, 128 x 128] = A B^T with both operands K-major tiles ([128 rows][128 elements of the contraction]): eight k-steps
 __device__ __forceinline__ void issue_nt(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr) {
-  constexpr uint32_t idesc = mv::um::idesc_bf16(BT, HB, 0, 0);
+  constexpr uint32_t idesc = mv::um::idesc_bf16(BT, BT, 0, 0);
   const uint64_t a_desc = mv::um::smem_desc(a_addr, 16, 1024), b_desc = mv::um::smem_desc(b_addr, 16, 1024);
   mv::um::mma_ss<false>(d_tmem, a_desc, b_desc, idesc);
 #pragma unroll
   for (int k = 1; k < D / 16; ++k) {
-    const uint32_t a_off = ((k >> 2) * (TILE_BYTES / 2) + (k & 3) * 32) >> 4, b_off = ((k >> 2) * (HALF_BYTES / 2) + (k & 3) * 32) >> 4;
-    mv::um::mma_ss<true>(d_tmem, a_desc + a_off, b_desc + b_off, idesc);
+    const uint32_t off = ((k >> 2) * (TILE_BYTES / 2) + (k & 3) * 32) >> 4;
+    mv::um::mma_ss<true>(d_tmem, a_desc + off, b_desc + off, idesc);
   }
 }
-// D[tmem, 128 x 128] (+)= A[tmem, 128 x 64 as bf16 pairs] B with B a 64-row half read as the MN-major operand
-// ([64 contraction rows][128 columns]): four k-steps.  The lane threads leave A in two pieces, the pairs of a step's
-// columns 0..31 at a_tmem + 0..15 and those of columns 32..63 at a_tmem + 32..47.
+// D[tmem, 128 x 128] (+)= A[tmem, 128 x 128 as bf16 pairs] B with B an MN-major tile ([128 contraction rows][128
+// columns]): eight k-steps.  The lane threads leave A in two pieces, the pairs of a step's columns 0..63 at
+// a_tmem + 0..31 and those of columns 64..127 at a_tmem + 64..95.
 __device__ __forceinline__ void issue_tn(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_addr, bool accumulate) {
   constexpr uint32_t idesc = mv::um::idesc_bf16(BT, D, 0, 1);
-  const uint64_t b_desc = mv::um::smem_desc(b_addr, HALF_BYTES / 2, 1024);
+  const uint64_t b_desc = mv::um::smem_desc(b_addr, TILE_BYTES / 2, 1024);
   if (accumulate) mv::um::mma_ts<true>(d_tmem, a_tmem, b_desc, idesc);
   else mv::um::mma_ts<false>(d_tmem, a_tmem, b_desc, idesc);
 #pragma unroll
-  for (int k = 1; k < HB / 16; ++k)
-    mv::um::mma_ts<true>(d_tmem, a_tmem + (k >> 1) * 32 + (k & 1) * 8, b_desc + uint32_t((k * 2048) >> 4), idesc);
+  for (int k = 1; k < BT / 16; ++k)
+    mv::um::mma_ts<true>(d_tmem, a_tmem + (k >> 2) * 64 + (k & 3) * 8, b_desc + uint32_t((k * 2048) >> 4), idesc);
 }
 
 struct Ctx {
@@ -148,31 +169,30 @@ __device__ __forceinline__ bool setup(Ctx& c, unsigned char* smem, int32_t* stat
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + N_BARS * 8);
   int* abort_flag = reinterpret_cast<int*>(smem + OFF_BAR + N_BARS * 8 + 8);
-  c.br.fixed_full = mv::smem_u32(&bars[0]);
-  c.br.full = mv::smem_u32(&bars[1]);
-  c.br.empty = mv::smem_u32(&bars[1 + NSTAGE]);
-  c.br.s_full = mv::smem_u32(&bars[1 + 2 * NSTAGE]);
-  c.br.p_full = mv::smem_u32(&bars[3 + 2 * NSTAGE]);
-  c.br.acc_done = mv::smem_u32(&bars[5 + 2 * NSTAGE]);
-  c.br.drained = mv::smem_u32(&bars[7 + 2 * NSTAGE]);
-  static_assert(8 + 2 * NSTAGE <= N_BARS, "barrier table too small");
+  int i = 0;
+  c.br.fixed_full = mv::smem_u32(&bars[i]); i += 1;
+  c.br.lfull = mv::smem_u32(&bars[i]); i += NLONG;
+  c.br.lempty = mv::smem_u32(&bars[i]); i += NLONG;
+  c.br.sfull = mv::smem_u32(&bars[i]); i += NSHORT;
+  c.br.sempty = mv::smem_u32(&bars[i]); i += NSHORT;
+  c.br.s_full = mv::smem_u32(&bars[i]); i += 3;
+  c.br.dp_free = mv::smem_u32(&bars[i]); i += 1;
+  c.br.p_full = mv::smem_u32(&bars[i]); i += 3;
+  c.br.acc_done = mv::smem_u32(&bars[i]); i += 3;
+  c.br.drained = mv::smem_u32(&bars[i]); i += 2;
+  c.br.vec_ready = mv::smem_u32(&bars[i]); i += 1;
   if ((c.smem_base & 1023u) != 0) {  // the swizzle pattern is anchored at 1024-byte boundaries
     if (tid == 0) atomicExch(status, int(MV_ERR_UNSUPPORTED));
     return false;
   }
   if (tid == 0) {
     *abort_flag = 0;
-    mv::mbar_init(c.br.fixed_full, 1);
-    for (int i = 0; i < NSTAGE; ++i) {
-      mv::mbar_init(c.br.full + 8 * i, 1);
-      mv::mbar_init(c.br.empty + 8 * i, 1);  // one tcgen05.commit
+    for (int b = 0; b < N_BARS; ++b) {
+      // one tcgen05.commit or one arrive of the producer, except the barriers on which the 256 lane threads arrive
+      const uint32_t addr = mv::smem_u32(&bars[b]);
+      const bool lanes = addr == c.br.dp_free || addr == c.br.vec_ready || (addr >= c.br.p_full && addr < c.br.p_full + 24);
+      mv::mbar_init(addr, lanes ? NLANE_THREADS : 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mv::mbar_init(c.br.s_full + 8 * b, 1);     // one tcgen05.commit
-      mv::mbar_init(c.br.p_full + 8 * b, 256);   // the 256 lane threads
-      mv::mbar_init(c.br.acc_done + 8 * b, 1);   // one tcgen05.commit
-    }
-    mv::mbar_init(c.br.drained, 1);
     mv::mbar_fence_init();
     mv::fence_proxy_async();
   }
@@ -195,15 +215,14 @@ __device__ __forceinline__ void teardown(const Ctx& c) {
 }
 
 // after a wait ran out: the producer's copies in flight must land before the CTA may return
-__device__ __forceinline__ void drain_producer(const Ctx& c, int e) {
-  (void)mv::mbar_wait_bounded(c.br.fixed_full, 0, 20000000ull);
-  for (int k = 1; k <= min(e, NSTAGE); ++k)
-    (void)mv::mbar_wait_bounded(c.br.full + 8 * ((e - k) % NSTAGE), ((e - k) / NSTAGE) & 1, 20000000ull);
+__device__ __forceinline__ void drain_ring(uint32_t full, int nslots, int issued) {
+  for (int k = 1; k <= min(issued, nslots); ++k)
+    (void)mv::mbar_wait_bounded(full + 8 * ((issued - k) % nslots), ((issued - k) / nslots) & 1, 20000000ull);
 }
-__device__ __forceinline__ void drain_issuer(const Ctx& c, bool lead) {
+__device__ __forceinline__ void drain_issuer(uint32_t drained, bool lead) {
   __syncwarp();
-  if (lead) mv::um::commit(c.br.drained);
-  (void)mv::mbar_wait_bounded(c.br.drained, 0, 20000000ull);
+  if (lead) mv::um::commit(drained);
+  (void)mv::mbar_wait_bounded(drained, 0, 20000000ull);
 }
 
 // ---- delta[i][h] = <dO[i][h], O[i][h]> ------------------------------------------------------------------------
@@ -221,137 +240,245 @@ __global__ void __launch_bounds__(128) delta_kernel(const bf16* __restrict__ out
   if (lane == 0) delta[w] = s;
 }
 
-// ---- dQ ------------------------------------------------------------------------------------------------------
-// The visible keys are taken in steps of 64, one ring stage (K, V halves) per step, alternating between two score
-// buffers in tensor memory, so that the tensor cores compute the next step's S and dP while the lane threads turn this
-// one's into dS.  Buffer b: S at 128 b (dS written back over its columns 0..15 and 32..47), dP at 128 b + 64; the dQ
-// accumulator at +256.
+// ---- the three tensor-core kernels -----------------------------------------------------------------------------
+// One step of the lane threads' arithmetic over 32 columns: s (scores, fp32 bits) and dp (dP, fp32 bits) -> packed bf16
+// pairs.  nl2 / nd2: per pair of columns, (-lse, -lse) and (-scale * delta, -scale * delta) of the row (DQ) or of the
+// two columns (DK, DV).  Columns outside [lo, hi) are masked; `all` says that no column of the warp's 32 is.
+template <int MODE, bool ALL, typename NL, typename ND>
+__device__ __forceinline__ void lane_math(const uint32_t (&s)[32], const uint32_t* dp, uint32_t (&o)[16], float scale_log2, float scale,
+                                          int j0, int lo, int hi, NL nl2, ND nd2) {
+  const uint64_t sl2 = mv::pack_f32x2(scale_log2, scale_log2), sc2 = mv::pack_f32x2(scale, scale);
+#pragma unroll
+  for (int k = 0; k < 32; k += 2) {
+    float x0, x1;
+    mv::unpack_f32x2(mv::fma_f32x2(mv::pack_u32x2(s[k], s[k + 1]), sl2, nl2(k)), x0, x1);
+    float p0 = mv::fast_exp2(x0), p1 = mv::fast_exp2(x1);
+    if (!ALL) {
+      // a masked pair has P = 0, and with it dS = 0: dP and delta are finite whatever the padding holds
+      p0 = (j0 + k >= lo && j0 + k < hi) ? p0 : 0.f;
+      p1 = (j0 + k + 1 >= lo && j0 + k + 1 < hi) ? p1 : 0.f;
+    }
+    if (MODE == DV) {
+      o[k >> 1] = mv::pack_bf16(p0, p1);
+    } else {
+      float d0, d1;
+      mv::unpack_f32x2(mv::mul_f32x2(mv::pack_f32x2(p0, p1), mv::fma_f32x2(mv::pack_u32x2(dp[k], dp[k + 1]), sc2, nd2(k))), d0, d1);
+      o[k >> 1] = mv::pack_bf16(d0, d1);
+    }
+  }
+}
 
-__global__ void __launch_bounds__(NTHREADS, 1) dq_kernel(const BwdArgs a, const __grid_constant__ CUtensorMap tm_q,
-                                                         const __grid_constant__ CUtensorMap tm_do, const __grid_constant__ CUtensorMap tm_k,
-                                                         const __grid_constant__ CUtensorMap tm_v) {
-  extern __shared__ __align__(1024) unsigned char smem[];
+template <int MODE>
+__device__ __forceinline__ void bwd_body(const BwdArgs& a, const CUtensorMap* tm_q, const CUtensorMap* tm_do, const CUtensorMap* tm_k,
+                                         const CUtensorMap* tm_v, unsigned char* smem) {
+  constexpr int NBUF = MODE == DV ? 3 : 2;  // score buffers
   Ctx c;
   if (!setup(c, smem, a.status)) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const mv::QTile qt = a.tiles[blockIdx.y];
-  const int head = blockIdx.x, kvh = head / a.G;
+  const mv::QTile tile = MODE == DQ ? a.q_tiles[blockIdx.y] : a.k_tiles[blockIdx.y];  // DK, DV: q_start / q_len are keys
+  const mv::KvRange* ranges = (MODE == DQ ? a.kv_ranges : a.q_ranges) + tile.range_begin;
+  // DQ: blockIdx.x is the query head.  DK, DV: the KV head, and a step's query head is kvh * G + its index in the group.
+  const int kvh = MODE == DQ ? blockIdx.x / a.G : blockIdx.x;
+  const int heads = MODE == DQ ? 1 : a.G;
+  const int cut = MODE == DQ ? tile.causal_base + tile.q_len - 1 : 0x3fffffff;
   const Bars& br = c.br;
   const Waiter& w = c.w;
-  const int q_last = qt.causal_base + qt.q_len - 1;
+  const uint32_t fixed0 = c.smem_base + OFF_FIXED, fixed1 = fixed0 + TILE_BYTES;
+  const uint32_t ring_long = c.smem_base + OFF_LONG, ring_short = c.smem_base + OFF_SHORT;
   if (warp == 0) {
     if (lane == 0) {  // producer
-      mv::mbar_arrive_expect_tx(br.fixed_full, 2 * TILE_BYTES);
-      load_tile(c.smem_base + OFF_FIXED, &tm_q, head * D, qt.q_start, br.fixed_full);
-      load_tile(c.smem_base + OFF_FIXED + TILE_BYTES, &tm_do, head * D, qt.q_start, br.fixed_full);
-      Walk it(a.ranges + qt.range_begin, qt.range_count, q_last);
-      int start, n, cz, e = 0;
+      const CUtensorMap* tm_f0 = MODE == DQ ? tm_q : tm_k;
+      const CUtensorMap* tm_f1 = MODE == DQ ? tm_do : tm_v;
+      const CUtensorMap* tm_long = MODE == DQ ? tm_k : (MODE == DK ? tm_q : tm_do);
+      const CUtensorMap* tm_short = MODE == DQ ? tm_v : (MODE == DK ? tm_do : tm_q);
+      const int fixed_col = (MODE == DQ ? int(blockIdx.x) : kvh) * D;
+      mv::mbar_arrive_expect_tx(br.fixed_full, (MODE == DV ? 1 : 2) * TILE_BYTES);
+      load_tile(fixed0, tm_f0, fixed_col, tile.q_start, br.fixed_full);
+      if (MODE != DV) load_tile(fixed1, tm_f1, fixed_col, tile.q_start, br.fixed_full);
+      Steps it(ranges, tile.range_count, cut, heads);
+      int start, n, cz, hg, es = 0, el = 0;  // short / long tiles issued
       bool ok = true;
-      while (ok && it.next(start, n, cz)) {
-        const int st = e % NSTAGE;
-        ok = w.wait(br.empty + 8 * st, ((e / NSTAGE) & 1) ^ 1);
+      while (ok && it.next(start, n, cz, hg)) {
+        const int col = (MODE == DQ ? kvh : kvh * a.G + hg) * D;
+        const int ss = es % NSHORT, ls = el % NLONG;
+        ok = w.wait(br.sempty + 8 * ss, ((es / NSHORT) & 1) ^ 1);
         if (!ok) break;
-        mv::mbar_arrive_expect_tx(br.full + 8 * st, STAGE_BYTES);
-        load_half(c.smem_base + OFF_RING + st * STAGE_BYTES, &tm_k, kvh * D, start, br.full + 8 * st);
-        load_half(c.smem_base + OFF_RING + st * STAGE_BYTES + HALF_BYTES, &tm_v, kvh * D, start, br.full + 8 * st);
-        ++e;
+        mv::mbar_arrive_expect_tx(br.sfull + 8 * ss, TILE_BYTES);
+        load_tile(ring_short + ss * TILE_BYTES, tm_short, col, start, br.sfull + 8 * ss);
+        ++es;
+        ok = w.wait(br.lempty + 8 * ls, ((el / NLONG) & 1) ^ 1);
+        if (!ok) break;
+        mv::mbar_arrive_expect_tx(br.lfull + 8 * ls, TILE_BYTES);
+        load_tile(ring_long + ls * TILE_BYTES, tm_long, col, start, br.lfull + 8 * ls);
+        ++el;
       }
-      if (!ok) drain_producer(c, e);
+      if (!ok) {
+        (void)mv::mbar_wait_bounded(br.fixed_full, 0, 20000000ull);
+        drain_ring(br.sfull, NSHORT, es);
+        drain_ring(br.lfull, NLONG, el);
+      }
     }
-  } else if (warp == 1) {
-    // issuer: the whole warp walks, one elected lane issues.  The dQ product of a step is issued after the scores of
-    // the step behind it, so the tensor cores always have the next scores queued while the lane threads work.
+  } else if (warp == 1 || warp == 2) {
+    // Two issuers, because a thread that issues products is held until the tensor cores take them: warp 1 issues dP
+    // and the scores, warp 2 the accumulating products, and the barrier waits of one fall into the products of the
+    // other.  While the lane threads work on step e, warp 2 issues the accumulating product of step e - 1 and warp 1
+    // dP of step e + 1 (the lane threads have copied dP of step e to registers by then), then the scores of step e + 1,
+    // whose buffer the accumulating product of step e + 1 - NBUF has read.  The whole warp walks, one elected lane issues.
     const bool lead = mv::um::elect_one();
-    Walk it(a.ranges + qt.range_begin, qt.range_count, q_last);
-    const uint32_t q_addr = c.smem_base + OFF_FIXED, do_addr = q_addr + TILE_BYTES;
-    int start, n, cz, e = 0;
-    // step f's dQ product: after the lane threads have left dS in buffer f & 1; it frees the buffer and the stage
-    auto finish = [&](int f) -> bool {
-      const int b = f & 1;
-      if (!w.wait(br.p_full + 8 * b, (f >> 1) & 1)) return false;
-      mv::um::fence_after();
-      if (lead) {
-        issue_tn(c.tmem + 256, c.tmem + 128 * b, c.smem_base + OFF_RING + (f % NSTAGE) * STAGE_BYTES, f > 0);  // dQ += dS K
-        mv::um::commit(br.acc_done + 8 * b);
-        mv::um::commit(br.empty + 8 * (f % NSTAGE));
-      }
-      __syncwarp();
-      return true;
-    };
+    Steps it(ranges, tile.range_count, cut, heads);
+    int start, n, cz, hg, f = 0;
     bool ok = w.wait(br.fixed_full, 0);
-    while (ok && it.next(start, n, cz)) {
-      const int st = e % NSTAGE, b = e & 1;
-      const uint32_t kh = c.smem_base + OFF_RING + st * STAGE_BYTES, vh = kh + HALF_BYTES;
-      ok = w.wait(br.full + 8 * st, (e / NSTAGE) & 1);
-      // the dQ product two steps back has read dS from this buffer before the new scores overwrite it
-      if (ok && e >= 2) ok = w.wait(br.acc_done + 8 * b, ((e >> 1) - 1) & 1);
-      if (!ok) break;
-      mv::um::fence_after();
-      if (lead) {
-        issue_nt(c.tmem + 128 * b, q_addr, kh);         // S = Q K^T
-        issue_nt(c.tmem + 128 * b + HB, do_addr, vh);   // dP = dO V^T
-        mv::um::commit(br.s_full + 8 * b);
+    if (warp == 1) {
+      for (; ok && it.next(start, n, cz, hg); ++f) {
+        const int b = f % NBUF, u = f / NBUF, ss = f % NSHORT, ls = f % NLONG;
+        ok = w.wait(br.sfull + 8 * ss, (f / NSHORT) & 1);
+        if (MODE != DV) {
+          if (ok && f >= 1) ok = w.wait(br.dp_free, (f - 1) & 1);  // the lane threads hold dP of step f - 1 in registers
+          if (!ok) break;
+          mv::um::fence_after();
+          if (lead) {
+            issue_nt(c.tmem + TM_DP, fixed1, ring_short + ss * TILE_BYTES);  // dP = dO V^T  /  dP^T = V dO^T
+            mv::um::commit(br.sempty + 8 * ss);
+          }
+          __syncwarp();
+          ok = w.wait(br.lfull + 8 * ls, (f / NLONG) & 1);
+        }
+        if (ok && f >= NBUF) ok = w.wait(br.acc_done + 8 * b, (u - 1) & 1);
+        if (!ok) break;
+        mv::um::fence_after();
+        if (lead) {
+          // S = Q K^T  /  S^T = K Q^T
+          issue_nt(c.tmem + TM_S + 128 * b, fixed0, MODE == DV ? ring_short + ss * TILE_BYTES : ring_long + ls * TILE_BYTES);
+          if (MODE == DV) mv::um::commit(br.sempty + 8 * ss);
+          mv::um::commit(br.s_full + 8 * b);
+        }
+        __syncwarp();
       }
-      __syncwarp();
-      if (e > 0) ok = finish(e - 1);
-      ++e;
+    } else {
+      for (; ok && it.next(start, n, cz, hg); ++f) {
+        const int b = f % NBUF, ls = f % NLONG;
+        ok = w.wait(br.p_full + 8 * b, (f / NBUF) & 1);  // the lane threads have left dS (P^T in DV) in the buffer
+        if (ok && MODE == DV) ok = w.wait(br.lfull + 8 * ls, (f / NLONG) & 1);
+        if (!ok) break;
+        mv::um::fence_after();
+        if (lead) {
+          issue_tn(c.tmem + TM_ACC, c.tmem + TM_S + 128 * b, ring_long + ls * TILE_BYTES, f > 0);  // dQ += dS K, dK += dS^T Q, dV += P^T dO
+          mv::um::commit(br.acc_done + 8 * b);
+          mv::um::commit(br.lempty + 8 * ls);
+        }
+        __syncwarp();
+      }
     }
-    if (ok && e > 0) ok = finish(e - 1);
-    if (w.aborted()) drain_issuer(c, lead);
-  } else {
-    // lane threads: the two threads on tensor-memory lane r own query row r of the tile, 32 columns of a step each
-    const int r = (warp & 3) * 32 + lane, ch = (warp - 2) >> 2;
+    if (w.aborted()) drain_issuer(br.drained + 8 * (warp - 1), lead);
+  } else if (warp >= 4) {
+    // lane threads: the two threads on tensor-memory lane r own row r of the tile (a query in DQ, a key in DK and DV),
+    // 64 columns of a step each
+    const int tl = threadIdx.x - 128;
+    const int r = (warp & 3) * 32 + lane, ch = (warp - 4) >> 2;
     const uint32_t lane_base = c.tmem + (uint32_t((warp & 3) * 32) << 16);
-    const int qi = qt.q_start + r, qc = qt.causal_base + r;
-    const bool row_ok = r < qt.q_len;
-    const float lse = row_ok ? a.lse[int64_t(qi) * a.Hq + head] : 0.f;
-    const float dl = row_ok ? a.delta[int64_t(qi) * a.Hq + head] * a.scale : 0.f;
-    Walk it(a.ranges + qt.range_begin, qt.range_count, q_last);
-    int start, n, cz, e = 0;
-    bool ok = true;
-    while (it.next(start, n, cz)) {
-      const int b = e & 1;
-      const int lim = row_ok ? (cz ? min(n, qc - start + 1) : n) : 0;  // keys [0, lim) of the step are visible to this row
-      ok = w.warp_wait(br.s_full + 8 * b, (e >> 1) & 1);
+    const bool row_ok = r < tile.q_len;
+    const int tok = tile.q_start + r, rc = tile.causal_base + r;  // the row's token, and its index in the causal numbering
+    float* vec = reinterpret_cast<float*>(smem + OFF_VEC);
+    uint64_t row_nl2 = 0, row_nd2 = 0;
+    if (MODE == DQ) {
+      const float nl = row_ok ? -a.lse[int64_t(tok) * a.Hq + blockIdx.x] : 0.f;
+      const float nd = row_ok ? -a.delta[int64_t(tok) * a.Hq + blockIdx.x] * a.scale : 0.f;
+      row_nl2 = mv::pack_f32x2(nl, nl);
+      row_nd2 = mv::pack_f32x2(nd, nd);
+    }
+    // DK, DV: the step's -lse and -scale * delta per query, fetched one step ahead by the lane threads themselves
+    // (thread t < 128: lse of query t; t >= 128: delta of query t - 128) into the slot of the step's parity
+    auto fetch = [&](int start, int n, int hg) -> float {
+      const int x = tl & (BT - 1);
+      if (x >= n) return 0.f;
+      const int64_t at = int64_t(start + x) * a.Hq + kvh * a.G + hg;
+      return tl < BT ? a.lse[at] : a.delta[at];
+    };
+    const float vec_mul = tl < BT ? -1.f : -a.scale;  // applied when the value is stored, a step after it was fetched
+    Steps it(ranges, tile.range_count, cut, heads), ahead(ranges, tile.range_count, cut, heads);
+    int start, n, cz, hg, e = 0;
+    int a_start = 0, a_n = 0, a_cz = 0, a_hg = 0;
+    bool a_ok = false, ok = true;
+    if (MODE != DQ) {
+      if (ahead.next(a_start, a_n, a_cz, a_hg)) vec[tl] = fetch(a_start, a_n, a_hg) * vec_mul;
+      mv::mbar_arrive(br.vec_ready);
+      a_ok = ahead.next(a_start, a_n, a_cz, a_hg);
+    }
+    while (it.next(start, n, cz, hg)) {
+      const int b = e % NBUF;
+      float pre = 0.f;
+      if (MODE != DQ && a_ok) pre = fetch(a_start, a_n, a_hg);
+      if (MODE != DQ) ok = w.warp_wait(br.vec_ready, e & 1);
+      if (ok) ok = w.warp_wait(br.s_full + 8 * b, (e / NBUF) & 1);
       if (!ok) break;
       mv::um::fence_after();
-      const uint32_t base = lane_base + 128 * b + ch * 32;
-      const int j0 = ch * 32;
-      uint32_t s[32], dp[32], ds[16];
-      mv::um::ld32(base, s);
-      mv::um::ld32(base + HB, dp);
-      mv::um::wait_ld();
-#pragma unroll
-      for (int k = 0; k < 32; k += 2) {
-        // a masked pair has P = 0, and with it dS = 0: dP and delta are finite whatever the padding holds
-        const float p0 = j0 + k < lim ? mv::fast_exp2(fmaf(__uint_as_float(s[k]), a.scale_log2, -lse)) : 0.f;
-        const float p1 = j0 + k + 1 < lim ? mv::fast_exp2(fmaf(__uint_as_float(s[k + 1]), a.scale_log2, -lse)) : 0.f;
-        const float d0 = p0 * fmaf(__uint_as_float(dp[k]), a.scale, -dl);
-        const float d1 = p1 * fmaf(__uint_as_float(dp[k + 1]), a.scale, -dl);
-        ds[k >> 1] = mv::pack_bf16(d0, d1);
+      // columns [lo, hi) of the step are visible to this row.  DQ: the keys up to the query's own (causal range) or all
+      // n; DK, DV: the queries from the key's own on (own node) or all n.
+      int lo, hi;
+      if (MODE == DQ) {
+        lo = 0;
+        hi = row_ok ? (cz ? min(n, rc - start + 1) : n) : 0;
+      } else {
+        lo = row_ok ? (cz ? max(0, rc - start) : 0) : n;
+        hi = n;
       }
-      mv::um::st16(base, ds);  // over the thread's own S columns, which it has read
+      const uint32_t sbuf = lane_base + TM_S + 128 * b + ch * 64;
+      const float* vs = vec + (e & 1) * 2 * BT + ch * 64;
+      uint32_t s0[32], s1[32], dp0[32], dp1[32], o[16];
+      mv::um::ld32(sbuf, s0);
+      mv::um::ld32(sbuf + 32, s1);
+      if (MODE != DV) {
+        mv::um::ld32(lane_base + TM_DP + ch * 64, dp0);
+        mv::um::ld32(lane_base + TM_DP + ch * 64 + 32, dp1);
+      }
+      mv::um::wait_ld();
+      if (MODE != DV) {
+        mv::um::fence_before();
+        mv::mbar_arrive(br.dp_free);  // dP is in registers: the tensor cores may write the next step's
+      }
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        const int j0 = ch * 64 + cc * 32;
+        const uint32_t(&s)[32] = cc == 0 ? s0 : s1;
+        const uint32_t* dp = cc == 0 ? dp0 : dp1;
+        const bool all = __all_sync(0xffffffffu, lo <= j0 && hi >= j0 + 32);
+        auto nl2 = [&](int k) -> uint64_t { return MODE == DQ ? row_nl2 : *reinterpret_cast<const uint64_t*>(vs + cc * 32 + k); };
+        auto nd2 = [&](int k) -> uint64_t { return MODE == DQ ? row_nd2 : *reinterpret_cast<const uint64_t*>(vs + BT + cc * 32 + k); };
+        if (all) lane_math<MODE, true>(s, dp, o, a.scale_log2, a.scale, j0, lo, hi, nl2, nd2);
+        else lane_math<MODE, false>(s, dp, o, a.scale_log2, a.scale, j0, lo, hi, nl2, nd2);
+        // over the thread's own score columns, all of which it has read: 16 packed columns per 32
+        mv::um::st16(sbuf + cc * 16, o);
+      }
       mv::um::wait_st();
       mv::um::fence_before();
       mv::mbar_arrive(br.p_full + 8 * b);
+      if (MODE != DQ) {
+        // every lane thread has passed this step's vec_ready wait, so none still reads the other slot (step e - 1's)
+        if (a_ok) vec[((e + 1) & 1) * 2 * BT + tl] = pre * vec_mul;
+        mv::mbar_arrive(br.vec_ready);
+        a_ok = ahead.next(a_start, a_n, a_cz, a_hg);
+      }
       ++e;
     }
-    if (ok && e > 0 && w.warp_wait(br.acc_done + 8 * ((e - 1) & 1), ((e - 1) >> 1) & 1)) {
+    if (ok && e > 0 && w.warp_wait(br.acc_done + 8 * ((e - 1) % NBUF), ((e - 1) / NBUF) & 1)) {
       mv::um::fence_after();
-      bf16* dst = a.dq + (int64_t(qi) * a.Hq + head) * D + ch * 64;
+      bf16* dst;
+      if (MODE == DQ) dst = a.dq + (int64_t(tok) * a.Hq + blockIdx.x) * D;
+      else dst = (MODE == DK ? a.dk : a.dv) + (int64_t(tok) * a.Hkv + kvh) * D;
+      dst += ch * 64;
 #pragma unroll 1
       for (int cb = 0; cb < 2; ++cb) {
-        uint32_t o[32];
-        mv::um::ld32(lane_base + 256 + ch * 64 + cb * 32, o);
+        uint32_t acc[32];
+        mv::um::ld32(lane_base + TM_ACC + ch * 64 + cb * 32, acc);
         mv::um::wait_ld();
         if (row_ok) {
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             uint4 v;
-            v.x = mv::pack_bf16(__uint_as_float(o[8 * k]), __uint_as_float(o[8 * k + 1]));
-            v.y = mv::pack_bf16(__uint_as_float(o[8 * k + 2]), __uint_as_float(o[8 * k + 3]));
-            v.z = mv::pack_bf16(__uint_as_float(o[8 * k + 4]), __uint_as_float(o[8 * k + 5]));
-            v.w = mv::pack_bf16(__uint_as_float(o[8 * k + 6]), __uint_as_float(o[8 * k + 7]));
+            v.x = mv::pack_bf16(__uint_as_float(acc[8 * k]), __uint_as_float(acc[8 * k + 1]));
+            v.y = mv::pack_bf16(__uint_as_float(acc[8 * k + 2]), __uint_as_float(acc[8 * k + 3]));
+            v.z = mv::pack_bf16(__uint_as_float(acc[8 * k + 4]), __uint_as_float(acc[8 * k + 5]));
+            v.w = mv::pack_bf16(__uint_as_float(acc[8 * k + 6]), __uint_as_float(acc[8 * k + 7]));
             *reinterpret_cast<uint4*>(dst + cb * 32 + k * 8) = v;
           }
         }
@@ -361,174 +488,19 @@ __global__ void __launch_bounds__(NTHREADS, 1) dq_kernel(const BwdArgs a, const 
   teardown(c);
 }
 
-// ---- dK, dV --------------------------------------------------------------------------------------------------
-// A step is (64 queries that see the tile's node, one query head of the group): one ring stage holds the Q and dO
-// halves and the queries' lse and delta.  Two score buffers as in dq_kernel.  Buffer b: S^T at 128 b (P^T written
-// back over its columns 0..15 and 32..47), dP^T at 128 b + 64 (dS^T likewise); the dV accumulator at +256, dK at +384.
+__global__ void __launch_bounds__(NTHREADS, 1) dq_kernel(const BwdArgs a, const __grid_constant__ CUtensorMap tm_q,
+                                                         const __grid_constant__ CUtensorMap tm_do, const __grid_constant__ CUtensorMap tm_k,
+                                                         const __grid_constant__ CUtensorMap tm_v) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  bwd_body<DQ>(a, &tm_q, &tm_do, &tm_k, &tm_v, smem);
+}
+// blockIdx.z = 0: dK, 1: dV (the longer CTAs are scheduled first)
 __global__ void __launch_bounds__(NTHREADS, 1) dkv_kernel(const BwdArgs a, const __grid_constant__ CUtensorMap tm_q,
                                                           const __grid_constant__ CUtensorMap tm_do, const __grid_constant__ CUtensorMap tm_k,
                                                           const __grid_constant__ CUtensorMap tm_v) {
   extern __shared__ __align__(1024) unsigned char smem[];
-  Ctx c;
-  if (!setup(c, smem, a.status)) return;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const mv::QTile kt = a.tiles[blockIdx.y];  // q_start / q_len: the tile's first key and key count
-  const int kvh = blockIdx.x;
-  const Bars& br = c.br;
-  const Waiter& w = c.w;
-  constexpr int NO_CUT = 0x3fffffff;
-  float* vec = reinterpret_cast<float*>(smem + OFF_VEC);  // [stage][lse 64 | delta * scale 64]
-  if (warp == 0) {
-    // producer: lane 0 issues the tile copies; all lanes fetch the stage's lse / delta vectors with plain loads
-    if (lane == 0) {
-      mv::mbar_arrive_expect_tx(br.fixed_full, 2 * TILE_BYTES);
-      load_tile(c.smem_base + OFF_FIXED, &tm_k, kvh * D, kt.q_start, br.fixed_full);
-      load_tile(c.smem_base + OFF_FIXED + TILE_BYTES, &tm_v, kvh * D, kt.q_start, br.fixed_full);
-    }
-    Walk it(a.ranges + kt.range_begin, kt.range_count, NO_CUT);
-    int start, n, cz, e = 0;
-    bool ok = true;
-    while (ok && it.next(start, n, cz)) {
-      for (int hg = 0; hg < a.G && ok; ++hg, ++e) {
-        const int st = e % NSTAGE, head = kvh * a.G + hg;
-        int go = 1;
-        if (lane == 0) go = w.wait(br.empty + 8 * st, ((e / NSTAGE) & 1) ^ 1) ? 1 : 0;
-        ok = __shfl_sync(0xffffffffu, go, 0) != 0;
-        if (!ok) break;
-        float* vs = vec + st * 2 * HB;
-        for (int x = lane; x < HB; x += 32) {
-          const bool in = x < n;
-          vs[x] = in ? a.lse[int64_t(start + x) * a.Hq + head] : 0.f;
-          vs[HB + x] = in ? a.delta[int64_t(start + x) * a.Hq + head] * a.scale : 0.f;
-        }
-        __syncwarp();
-        if (lane == 0) {
-          mv::mbar_arrive_expect_tx(br.full + 8 * st, STAGE_BYTES);  // releases the vector stores above
-          load_half(c.smem_base + OFF_RING + st * STAGE_BYTES, &tm_q, head * D, start, br.full + 8 * st);
-          load_half(c.smem_base + OFF_RING + st * STAGE_BYTES + HALF_BYTES, &tm_do, head * D, start, br.full + 8 * st);
-        }
-      }
-    }
-    if (!ok && lane == 0) drain_producer(c, e);
-    __syncwarp();
-  } else if (warp == 1) {
-    const bool lead = mv::um::elect_one();
-    Walk it(a.ranges + kt.range_begin, kt.range_count, NO_CUT);
-    const uint32_t k_addr = c.smem_base + OFF_FIXED, v_addr = k_addr + TILE_BYTES;
-    int start, n, cz, e = 0;
-    // step f's accumulating products: after the lane threads have left P^T and dS^T in buffer f & 1
-    auto finish = [&](int f) -> bool {
-      const int b = f & 1;
-      if (!w.wait(br.p_full + 8 * b, (f >> 1) & 1)) return false;
-      mv::um::fence_after();
-      if (lead) {
-        const uint32_t qh = c.smem_base + OFF_RING + (f % NSTAGE) * STAGE_BYTES, doh = qh + HALF_BYTES;
-        issue_tn(c.tmem + 256, c.tmem + 128 * b, doh, f > 0);      // dV += P^T dO
-        issue_tn(c.tmem + 384, c.tmem + 128 * b + HB, qh, f > 0);  // dK += dS^T Q
-        mv::um::commit(br.acc_done + 8 * b);
-        mv::um::commit(br.empty + 8 * (f % NSTAGE));
-      }
-      __syncwarp();
-      return true;
-    };
-    bool ok = w.wait(br.fixed_full, 0);
-    while (ok && it.next(start, n, cz)) {
-      for (int hg = 0; hg < a.G && ok; ++hg, ++e) {
-        const int st = e % NSTAGE, b = e & 1;
-        const uint32_t qh = c.smem_base + OFF_RING + st * STAGE_BYTES, doh = qh + HALF_BYTES;
-        ok = w.wait(br.full + 8 * st, (e / NSTAGE) & 1);
-        // the products two steps back have read P^T and dS^T from this buffer before the new scores overwrite them
-        if (ok && e >= 2) ok = w.wait(br.acc_done + 8 * b, ((e >> 1) - 1) & 1);
-        if (!ok) break;
-        mv::um::fence_after();
-        if (lead) {
-          issue_nt(c.tmem + 128 * b, k_addr, qh);         // S^T = K Q^T
-          issue_nt(c.tmem + 128 * b + HB, v_addr, doh);   // dP^T = V dO^T
-          mv::um::commit(br.s_full + 8 * b);
-        }
-        __syncwarp();
-        if (e > 0) ok = finish(e - 1);
-      }
-    }
-    if (ok && e > 0) ok = finish(e - 1);
-    if (w.aborted()) drain_issuer(c, lead);
-  } else {
-    // lane threads: the two threads on tensor-memory lane r own key r of the tile, 32 queries of a step each
-    const int r = (warp & 3) * 32 + lane, ch = (warp - 2) >> 2;
-    const uint32_t lane_base = c.tmem + (uint32_t((warp & 3) * 32) << 16);
-    const bool key_ok = r < kt.q_len;
-    const int kc = kt.causal_base + r;  // the key's flattened index
-    Walk it(a.ranges + kt.range_begin, kt.range_count, NO_CUT);
-    int start, n, cz, e = 0;
-    bool ok = true;
-    while (ok && it.next(start, n, cz)) {
-      // queries [first, n) of the step see this key: all valid ones, or (own node) those not before the key
-      const int first = key_ok ? (cz ? max(0, kc - start) : 0) : n;
-      for (int hg = 0; hg < a.G && ok; ++hg, ++e) {
-        const int st = e % NSTAGE, b = e & 1;
-        ok = w.warp_wait(br.full + 8 * st, (e / NSTAGE) & 1);  // the stage's lse / delta vectors are visible
-        if (ok) ok = w.warp_wait(br.s_full + 8 * b, (e >> 1) & 1);
-        if (!ok) break;
-        mv::um::fence_after();
-        const float4* vl = reinterpret_cast<const float4*>(vec + st * 2 * HB + ch * 32);
-        const float4* vd = reinterpret_cast<const float4*>(vec + st * 2 * HB + HB + ch * 32);
-        const uint32_t base = lane_base + 128 * b + ch * 32;
-        const int j0 = ch * 32;
-        uint32_t s[32], dp[32], pt[16], ds[16];
-        mv::um::ld32(base, s);
-        mv::um::ld32(base + HB, dp);
-        mv::um::wait_ld();
-#pragma unroll
-        for (int k = 0; k < 32; k += 4) {
-          const float4 l4 = vl[k >> 2], d4 = vd[k >> 2];
-          const float ls[4] = {l4.x, l4.y, l4.z, l4.w}, dl[4] = {d4.x, d4.y, d4.z, d4.w};
-          float p[4], d[4];
-#pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            const int j = j0 + k + x;
-            // a masked pair has P = 0, and with it dS = 0: dP and delta are finite whatever the padding holds
-            p[x] = (j >= first && j < n) ? mv::fast_exp2(fmaf(__uint_as_float(s[k + x]), a.scale_log2, -ls[x])) : 0.f;
-            d[x] = p[x] * fmaf(__uint_as_float(dp[k + x]), a.scale, -dl[x]);
-          }
-          pt[k >> 1] = mv::pack_bf16(p[0], p[1]);
-          pt[(k >> 1) + 1] = mv::pack_bf16(p[2], p[3]);
-          ds[k >> 1] = mv::pack_bf16(d[0], d[1]);
-          ds[(k >> 1) + 1] = mv::pack_bf16(d[2], d[3]);
-        }
-        mv::um::st16(base, pt);       // over the thread's own S^T columns, which it has read
-        mv::um::st16(base + HB, ds);  // and over its own dP^T columns
-        mv::um::wait_st();
-        mv::um::fence_before();
-        mv::mbar_arrive(br.p_full + 8 * b);
-      }
-    }
-    if (ok && e > 0 && w.warp_wait(br.acc_done + 8 * ((e - 1) & 1), ((e - 1) >> 1) & 1)) {
-      mv::um::fence_after();
-      const int64_t tok = int64_t(kt.q_start + r);
-#pragma unroll 1
-      for (int which = 0; which < 2; ++which) {
-        bf16* dst = (which == 0 ? a.dv : a.dk) + (tok * a.Hkv + kvh) * D + ch * 64;
-#pragma unroll 1
-        for (int cb = 0; cb < 2; ++cb) {
-          uint32_t o[32];
-          mv::um::ld32(lane_base + 256 + which * 128 + ch * 64 + cb * 32, o);
-          mv::um::wait_ld();
-          if (key_ok) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              uint4 v;
-              v.x = mv::pack_bf16(__uint_as_float(o[8 * k]), __uint_as_float(o[8 * k + 1]));
-              v.y = mv::pack_bf16(__uint_as_float(o[8 * k + 2]), __uint_as_float(o[8 * k + 3]));
-              v.z = mv::pack_bf16(__uint_as_float(o[8 * k + 4]), __uint_as_float(o[8 * k + 5]));
-              v.w = mv::pack_bf16(__uint_as_float(o[8 * k + 6]), __uint_as_float(o[8 * k + 7]));
-              *reinterpret_cast<uint4*>(dst + cb * 32 + k * 8) = v;
-            }
-          }
-        }
-      }
-    }
-  }
-  teardown(c);
+  if (blockIdx.z == 0) bwd_body<DK>(a, &tm_q, &tm_do, &tm_k, &tm_v, smem);
+  else bwd_body<DV>(a, &tm_q, &tm_do, &tm_k, &tm_v, smem);
 }
 
 struct BwdMaps {
@@ -566,15 +538,19 @@ extern "C" mv_status mv_dag_prefill_attn_bwd(const mv_plan* P, const mv_attn_geo
   BwdMaps* tm = cache.find(key);
   if (!tm) {
     tm = cache.claim(key);
-    if (!mv::make_tmap_bf16_2d(&tm->tm_q, q_rot, uint64_t(T), uint64_t(g->n_q_heads) * D, HB) ||
-        !mv::make_tmap_bf16_2d(&tm->tm_do, dout, uint64_t(T), uint64_t(g->n_q_heads) * D, HB) ||
-        !mv::make_tmap_bf16_2d(&tm->tm_k, k_rot, uint64_t(T), uint64_t(g->n_kv_heads) * D, HB) ||
-        !mv::make_tmap_bf16_2d(&tm->tm_v, v, uint64_t(T), uint64_t(g->n_kv_heads) * D, HB)) {
+    if (!mv::make_tmap_bf16_2d(&tm->tm_q, q_rot, uint64_t(T), uint64_t(g->n_q_heads) * D, BT) ||
+        !mv::make_tmap_bf16_2d(&tm->tm_do, dout, uint64_t(T), uint64_t(g->n_q_heads) * D, BT) ||
+        !mv::make_tmap_bf16_2d(&tm->tm_k, k_rot, uint64_t(T), uint64_t(g->n_kv_heads) * D, BT) ||
+        !mv::make_tmap_bf16_2d(&tm->tm_v, v, uint64_t(T), uint64_t(g->n_kv_heads) * D, BT)) {
       cache.drop();
       return MV_ERR_CUDA;
     }
   }
   BwdArgs a;
+  a.q_tiles = mv::table<mv::QTile>(P, P->layout.q_tiles);
+  a.kv_ranges = mv::table<mv::KvRange>(P, P->layout.kv_ranges);
+  a.k_tiles = mv::table<mv::QTile>(P, P->layout.k_tiles);
+  a.q_ranges = mv::table<mv::KvRange>(P, P->layout.q_ranges);
   a.lse = static_cast<const float*>(lse);
   a.delta = static_cast<float*>(workspace);
   a.dq = static_cast<bf16*>(dq_rot);
@@ -592,14 +568,10 @@ extern "C" mv_status mv_dag_prefill_attn_bwd(const mv_plan* P, const mv_attn_geo
                                                               static_cast<float*>(workspace), n_row_heads);
   mv::g_launches++;
   if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
-  a.tiles = mv::table<mv::QTile>(P, P->layout.q_tiles);
-  a.ranges = mv::table<mv::KvRange>(P, P->layout.kv_ranges);
   dq_kernel<<<dim3(unsigned(g->n_q_heads), unsigned(P->q_tiles.size())), NTHREADS, SMEM_BYTES, s>>>(a, tm->tm_q, tm->tm_do, tm->tm_k, tm->tm_v);
   mv::g_launches++;
   if (cudaGetLastError() != cudaSuccess) return MV_ERR_CUDA;
-  a.tiles = mv::table<mv::QTile>(P, P->layout.k_tiles);
-  a.ranges = mv::table<mv::KvRange>(P, P->layout.q_ranges);
-  dkv_kernel<<<dim3(unsigned(g->n_kv_heads), unsigned(P->k_tiles.size())), NTHREADS, SMEM_BYTES, s>>>(a, tm->tm_q, tm->tm_do, tm->tm_k, tm->tm_v);
+  dkv_kernel<<<dim3(unsigned(g->n_kv_heads), unsigned(P->k_tiles.size()), 2), NTHREADS, SMEM_BYTES, s>>>(a, tm->tm_q, tm->tm_do, tm->tm_k, tm->tm_v);
   mv::g_launches++;
   return cudaGetLastError() == cudaSuccess ? MV_OK : MV_ERR_CUDA;
 }
