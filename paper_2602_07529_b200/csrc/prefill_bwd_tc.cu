@@ -132,9 +132,10 @@ __device__ __forceinline__ void load_tile(uint32_t dst, const CUtensorMap* tm, i
 }
 
 // D[tmem, 128 x 128] = A B^T with both operands K-major tiles ([128 rows][128 elements of the contraction]): eight k-steps
-__device__ __forceinline__ void issue_nt(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr) {
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t addr) { return mv::um::smem_desc(addr, 16, 1024); }
+__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t addr) { return mv::um::smem_desc(addr, TILE_BYTES / 2, 1024); }
+__device__ __forceinline__ void issue_nt(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc) {
   constexpr uint32_t idesc = mv::um::idesc_bf16(BT, BT, 0, 0);
-  const uint64_t a_desc = mv::um::smem_desc(a_addr, 16, 1024), b_desc = mv::um::smem_desc(b_addr, 16, 1024);
   mv::um::mma_ss<false>(d_tmem, a_desc, b_desc, idesc);
 #pragma unroll
   for (int k = 1; k < D / 16; ++k) {
@@ -145,9 +146,8 @@ __device__ __forceinline__ void issue_nt(uint32_t d_tmem, uint32_t a_addr, uint3
 // D[tmem, 128 x 128] (+)= A[tmem, 128 x 128 as bf16 pairs] B with B an MN-major tile ([128 contraction rows][128
 // columns]): eight k-steps.  The lane threads leave A in two pieces, the pairs of a step's columns 0..63 at
 // a_tmem + 0..31 and those of columns 64..127 at a_tmem + 64..95.
-__device__ __forceinline__ void issue_tn(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_addr, bool accumulate) {
+__device__ __forceinline__ void issue_tn(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, bool accumulate) {
   constexpr uint32_t idesc = mv::um::idesc_bf16(BT, D, 0, 1);
-  const uint64_t b_desc = mv::um::smem_desc(b_addr, TILE_BYTES / 2, 1024);
   if (accumulate) mv::um::mma_ts<true>(d_tmem, a_tmem, b_desc, idesc);
   else mv::um::mma_ts<false>(d_tmem, a_tmem, b_desc, idesc);
 #pragma unroll
@@ -241,29 +241,51 @@ __global__ void __launch_bounds__(128) delta_kernel(const bf16* __restrict__ out
 }
 
 // ---- the three tensor-core kernels -----------------------------------------------------------------------------
-// One step of the lane threads' arithmetic over 32 columns: s (scores, fp32 bits) and dp (dP, fp32 bits) -> packed bf16
-// pairs.  nl2 / nd2: per pair of columns, (-lse, -lse) and (-scale * delta, -scale * delta) of the row (DQ) or of the
-// two columns (DK, DV).  Columns outside [lo, hi) are masked; `all` says that no column of the warp's 32 is.
-template <int MODE, bool ALL, typename NL, typename ND>
-__device__ __forceinline__ void lane_math(const uint32_t (&s)[32], const uint32_t* dp, uint32_t (&o)[16], float scale_log2, float scale,
-                                          int j0, int lo, int hi, NL nl2, ND nd2) {
-  const uint64_t sl2 = mv::pack_f32x2(scale_log2, scale_log2), sc2 = mv::pack_f32x2(scale, scale);
+// The lane threads' arithmetic over 32 columns: s (scores, fp32 bits) and dp (dP, fp32 bits) -> packed bf16 pairs.
+// The per-pair constants (-lse, -lse) and (-scale * delta, -scale * delta) are the row's in DQ (row_nl2, row_nd2) and
+// the columns' in DK and DV, read from shared memory (vs: 32 values of -lse; vs + BT: of -scale * delta) eight
+// columns ahead of their use.  Columns outside [lo, hi) are masked; ALL says that none of the warp's 32 is.
+template <int MODE>
+__device__ __forceinline__ void lane_consts(const float* vs, int col, uint64_t (&nl)[4], uint64_t (&nd)[4], uint64_t row_nl2, uint64_t row_nd2) {
+  if (MODE == DQ) {
 #pragma unroll
-  for (int k = 0; k < 32; k += 2) {
-    float x0, x1;
-    mv::unpack_f32x2(mv::fma_f32x2(mv::pack_u32x2(s[k], s[k + 1]), sl2, nl2(k)), x0, x1);
-    float p0 = mv::fast_exp2(x0), p1 = mv::fast_exp2(x1);
-    if (!ALL) {
-      // a masked pair has P = 0, and with it dS = 0: dP and delta are finite whatever the padding holds
-      p0 = (j0 + k >= lo && j0 + k < hi) ? p0 : 0.f;
-      p1 = (j0 + k + 1 >= lo && j0 + k + 1 < hi) ? p1 : 0.f;
+    for (int i = 0; i < 4; ++i) nl[i] = row_nl2, nd[i] = row_nd2;
+  } else {
+    const float4 l0 = *reinterpret_cast<const float4*>(vs + col), l1 = *reinterpret_cast<const float4*>(vs + col + 4);
+    nl[0] = mv::pack_f32x2(l0.x, l0.y), nl[1] = mv::pack_f32x2(l0.z, l0.w), nl[2] = mv::pack_f32x2(l1.x, l1.y), nl[3] = mv::pack_f32x2(l1.z, l1.w);
+    if (MODE == DK) {
+      const float4 d0 = *reinterpret_cast<const float4*>(vs + BT + col), d1 = *reinterpret_cast<const float4*>(vs + BT + col + 4);
+      nd[0] = mv::pack_f32x2(d0.x, d0.y), nd[1] = mv::pack_f32x2(d0.z, d0.w), nd[2] = mv::pack_f32x2(d1.x, d1.y), nd[3] = mv::pack_f32x2(d1.z, d1.w);
     }
-    if (MODE == DV) {
-      o[k >> 1] = mv::pack_bf16(p0, p1);
-    } else {
-      float d0, d1;
-      mv::unpack_f32x2(mv::mul_f32x2(mv::pack_f32x2(p0, p1), mv::fma_f32x2(mv::pack_u32x2(dp[k], dp[k + 1]), sc2, nd2(k))), d0, d1);
-      o[k >> 1] = mv::pack_bf16(d0, d1);
+  }
+}
+template <int MODE, bool ALL>
+__device__ __forceinline__ void lane_math(const uint32_t (&s)[32], const uint32_t* dp, uint32_t (&o)[16], float scale_log2, float scale,
+                                          int j0, int lo, int hi, const float* vs, uint64_t row_nl2, uint64_t row_nd2) {
+  const uint64_t sl2 = mv::pack_f32x2(scale_log2, scale_log2), sc2 = mv::pack_f32x2(scale, scale);
+  uint64_t nl[2][4], nd[2][4];
+  lane_consts<MODE>(vs, 0, nl[0], nd[0], row_nl2, row_nd2);
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    if (g + 1 < 4) lane_consts<MODE>(vs, (g + 1) * 8, nl[(g + 1) & 1], nd[(g + 1) & 1], row_nl2, row_nd2);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int k = g * 8 + 2 * i;
+      float x0, x1;
+      mv::unpack_f32x2(mv::fma_f32x2(mv::pack_u32x2(s[k], s[k + 1]), sl2, nl[g & 1][i]), x0, x1);
+      float p0 = mv::fast_exp2(x0), p1 = mv::fast_exp2(x1);
+      if (!ALL) {
+        // a masked pair has P = 0, and with it dS = 0: dP and delta are finite whatever the padding holds
+        p0 = (j0 + k >= lo && j0 + k < hi) ? p0 : 0.f;
+        p1 = (j0 + k + 1 >= lo && j0 + k + 1 < hi) ? p1 : 0.f;
+      }
+      if (MODE == DV) {
+        o[k >> 1] = mv::pack_bf16(p0, p1);
+      } else {
+        float d0, d1;
+        mv::unpack_f32x2(mv::mul_f32x2(mv::pack_f32x2(p0, p1), mv::fma_f32x2(mv::pack_u32x2(dp[k], dp[k + 1]), sc2, nd[g & 1][i])), d0, d1);
+        o[k >> 1] = mv::pack_bf16(d0, d1);
+      }
     }
   }
 }
@@ -328,27 +350,26 @@ __device__ __forceinline__ void bwd_body(const BwdArgs& a, const CUtensorMap* tm
     Steps it(ranges, tile.range_count, cut, heads);
     int start, n, cz, hg, f = 0;
     bool ok = w.wait(br.fixed_full, 0);
+    // Descriptors are made before the waits, and the wait that is satisfied last comes last, so that little stands
+    // between a barrier's completion and the first product.
     if (warp == 1) {
+      const uint64_t f0_desc = kmajor_desc(fixed0), f1_desc = kmajor_desc(fixed1);
       for (; ok && it.next(start, n, cz, hg); ++f) {
         const int b = f % NBUF, u = f / NBUF, ss = f % NSHORT, ls = f % NLONG;
+        const uint64_t short_desc = kmajor_desc(ring_short + ss * TILE_BYTES), long_desc = kmajor_desc(ring_long + ls * TILE_BYTES);
+        const uint32_t s_tmem = c.tmem + TM_S + 128 * b;
         ok = w.wait(br.sfull + 8 * ss, (f / NSHORT) & 1);
-        if (MODE != DV) {
-          if (ok && f >= 1) ok = w.wait(br.dp_free, (f - 1) & 1);  // the lane threads hold dP of step f - 1 in registers
-          if (!ok) break;
-          mv::um::fence_after();
-          if (lead) {
-            issue_nt(c.tmem + TM_DP, fixed1, ring_short + ss * TILE_BYTES);  // dP = dO V^T  /  dP^T = V dO^T
-            mv::um::commit(br.sempty + 8 * ss);
-          }
-          __syncwarp();
-          ok = w.wait(br.lfull + 8 * ls, (f / NLONG) & 1);
-        }
+        if (ok && MODE != DV) ok = w.wait(br.lfull + 8 * ls, (f / NLONG) & 1);
         if (ok && f >= NBUF) ok = w.wait(br.acc_done + 8 * b, (u - 1) & 1);
+        if (ok && MODE != DV && f >= 1) ok = w.wait(br.dp_free, (f - 1) & 1);  // the lane threads hold dP of step f - 1 in registers
         if (!ok) break;
         mv::um::fence_after();
         if (lead) {
-          // S = Q K^T  /  S^T = K Q^T
-          issue_nt(c.tmem + TM_S + 128 * b, fixed0, MODE == DV ? ring_short + ss * TILE_BYTES : ring_long + ls * TILE_BYTES);
+          if (MODE != DV) {
+            issue_nt(c.tmem + TM_DP, f1_desc, short_desc);  // dP = dO V^T  /  dP^T = V dO^T
+            mv::um::commit(br.sempty + 8 * ss);
+          }
+          issue_nt(s_tmem, f0_desc, MODE == DV ? short_desc : long_desc);  // S = Q K^T  /  S^T = K Q^T
           if (MODE == DV) mv::um::commit(br.sempty + 8 * ss);
           mv::um::commit(br.s_full + 8 * b);
         }
@@ -357,12 +378,14 @@ __device__ __forceinline__ void bwd_body(const BwdArgs& a, const CUtensorMap* tm
     } else {
       for (; ok && it.next(start, n, cz, hg); ++f) {
         const int b = f % NBUF, ls = f % NLONG;
-        ok = w.wait(br.p_full + 8 * b, (f / NBUF) & 1);  // the lane threads have left dS (P^T in DV) in the buffer
-        if (ok && MODE == DV) ok = w.wait(br.lfull + 8 * ls, (f / NLONG) & 1);
+        const uint64_t long_desc = mnmajor_desc(ring_long + ls * TILE_BYTES);
+        const uint32_t s_tmem = c.tmem + TM_S + 128 * b;
+        if (MODE == DV) ok = w.wait(br.lfull + 8 * ls, (f / NLONG) & 1);
+        if (ok) ok = w.wait(br.p_full + 8 * b, (f / NBUF) & 1);  // the lane threads have left dS (P^T in DV) in the buffer
         if (!ok) break;
         mv::um::fence_after();
         if (lead) {
-          issue_tn(c.tmem + TM_ACC, c.tmem + TM_S + 128 * b, ring_long + ls * TILE_BYTES, f > 0);  // dQ += dS K, dK += dS^T Q, dV += P^T dO
+          issue_tn(c.tmem + TM_ACC, s_tmem, long_desc, f > 0);  // dQ += dS K, dK += dS^T Q, dV += P^T dO
           mv::um::commit(br.acc_done + 8 * b);
           mv::um::commit(br.lempty + 8 * ls);
         }
@@ -424,9 +447,12 @@ __device__ __forceinline__ void bwd_body(const BwdArgs& a, const CUtensorMap* tm
       }
       const uint32_t sbuf = lane_base + TM_S + 128 * b + ch * 64;
       const float* vs = vec + (e & 1) * 2 * BT + ch * 64;
+      // DK is short of registers (the column constants are prefetched beside dP): it reads the second half of its
+      // scores after the first half's arithmetic
+      constexpr bool S1_LATE = MODE == DK;
       uint32_t s0[32], s1[32], dp0[32], dp1[32], o[16];
       mv::um::ld32(sbuf, s0);
-      mv::um::ld32(sbuf + 32, s1);
+      if (!S1_LATE) mv::um::ld32(sbuf + 32, s1);
       if (MODE != DV) {
         mv::um::ld32(lane_base + TM_DP + ch * 64, dp0);
         mv::um::ld32(lane_base + TM_DP + ch * 64 + 32, dp1);
@@ -439,14 +465,16 @@ __device__ __forceinline__ void bwd_body(const BwdArgs& a, const CUtensorMap* tm
 #pragma unroll
       for (int cc = 0; cc < 2; ++cc) {
         const int j0 = ch * 64 + cc * 32;
+        if (S1_LATE && cc == 1) {
+          mv::um::ld32(sbuf + 32, s1);
+          mv::um::wait_ld();
+        }
         const uint32_t(&s)[32] = cc == 0 ? s0 : s1;
         const uint32_t* dp = cc == 0 ? dp0 : dp1;
         const bool all = __all_sync(0xffffffffu, lo <= j0 && hi >= j0 + 32);
-        auto nl2 = [&](int k) -> uint64_t { return MODE == DQ ? row_nl2 : *reinterpret_cast<const uint64_t*>(vs + cc * 32 + k); };
-        auto nd2 = [&](int k) -> uint64_t { return MODE == DQ ? row_nd2 : *reinterpret_cast<const uint64_t*>(vs + BT + cc * 32 + k); };
-        if (all) lane_math<MODE, true>(s, dp, o, a.scale_log2, a.scale, j0, lo, hi, nl2, nd2);
-        else lane_math<MODE, false>(s, dp, o, a.scale_log2, a.scale, j0, lo, hi, nl2, nd2);
-        // over the thread's own score columns, all of which it has read: 16 packed columns per 32
+        if (all) lane_math<MODE, true>(s, dp, o, a.scale_log2, a.scale, j0, lo, hi, vs + cc * 32, row_nl2, row_nd2);
+        else lane_math<MODE, false>(s, dp, o, a.scale_log2, a.scale, j0, lo, hi, vs + cc * 32, row_nl2, row_nd2);
+        // over the thread's own score columns that it has read: 16 packed columns per 32
         mv::um::st16(sbuf + cc * 16, o);
       }
       mv::um::wait_st();
@@ -454,6 +482,7 @@ __device__ __forceinline__ void bwd_body(const BwdArgs& a, const CUtensorMap* tm
       mv::mbar_arrive(br.p_full + 8 * b);
       if (MODE != DQ) {
         // every lane thread has passed this step's vec_ready wait, so none still reads the other slot (step e - 1's)
+        asm volatile("" : "+f"(pre));  // the value is consumed here, not where the load was issued
         if (a_ok) vec[((e + 1) & 1) * 2 * BT + tl] = pre * vec_mul;
         mv::mbar_arrive(br.vec_ready);
         a_ok = ahead.next(a_start, a_n, a_cz, a_hg);
