@@ -48,7 +48,7 @@ constexpr int OFF_LONG = 2 * TILE_BYTES;                   // DQ: K; DK: Q; DV: 
 constexpr int OFF_SHORT = OFF_LONG + NLONG * TILE_BYTES;   // DQ: V; DK: dO; DV: Q
 constexpr int OFF_VEC = OFF_SHORT + NSHORT * TILE_BYTES;   // DK, DV: two slots of -lse[128], -scale * delta[128] of a step's queries
 constexpr int OFF_BAR = OFF_VEC + 2 * 2 * BT * 4;
-constexpr int N_BARS = 1 + 2 * NLONG + 2 * NSHORT + 3 + 1 + 3 + 3 + 2 + 1;
+constexpr int N_BARS = 1 + 2 * NLONG + 2 * NSHORT + 3 + 2 + 3 + 3 + 2 + 1;
 constexpr int SMEM_BYTES = OFF_BAR + N_BARS * 8 + 16;
 static_assert(SMEM_BYTES <= 232448, "over the shared memory of a CTA");
 // tensor memory columns
@@ -73,7 +73,7 @@ struct BwdArgs {
 
 struct Bars {
   // lfull / lempty: NLONG consecutive barriers; sfull / sempty: NSHORT; s_full / p_full / acc_done: one per score buffer
-  uint32_t fixed_full, lfull, lempty, sfull, sempty, s_full, dp_free, p_full, acc_done, drained, vec_ready;  // drained: two, one per issuer
+  uint32_t fixed_full, lfull, lempty, sfull, sempty, s_full, dp_full, dp_free, p_full, acc_done, drained, vec_ready;  // drained: two, one per issuer
 };
 
 struct Waiter {
@@ -176,6 +176,7 @@ __device__ __forceinline__ bool setup(Ctx& c, unsigned char* smem, int32_t* stat
   c.br.sfull = mv::smem_u32(&bars[i]); i += NSHORT;
   c.br.sempty = mv::smem_u32(&bars[i]); i += NSHORT;
   c.br.s_full = mv::smem_u32(&bars[i]); i += 3;
+  c.br.dp_full = mv::smem_u32(&bars[i]); i += 1;
   c.br.dp_free = mv::smem_u32(&bars[i]); i += 1;
   c.br.p_full = mv::smem_u32(&bars[i]); i += 3;
   c.br.acc_done = mv::smem_u32(&bars[i]); i += 3;
@@ -359,16 +360,22 @@ __device__ __forceinline__ void bwd_body(const BwdArgs& a, const CUtensorMap* tm
         const uint64_t short_desc = kmajor_desc(ring_short + ss * TILE_BYTES), long_desc = kmajor_desc(ring_long + ls * TILE_BYTES);
         const uint32_t s_tmem = c.tmem + TM_S + 128 * b;
         ok = w.wait(br.sfull + 8 * ss, (f / NSHORT) & 1);
-        if (ok && MODE != DV) ok = w.wait(br.lfull + 8 * ls, (f / NLONG) & 1);
+        if (MODE != DV) {
+          if (ok && f >= 1) ok = w.wait(br.dp_free, (f - 1) & 1);  // the lane threads hold dP of step f - 1 in registers
+          if (!ok) break;
+          mv::um::fence_after();
+          if (lead) {
+            issue_nt(c.tmem + TM_DP, f1_desc, short_desc);  // dP = dO V^T  /  dP^T = V dO^T
+            mv::um::commit(br.sempty + 8 * ss);
+            mv::um::commit(br.dp_full);
+          }
+          __syncwarp();
+          ok = w.wait(br.lfull + 8 * ls, (f / NLONG) & 1);
+        }
         if (ok && f >= NBUF) ok = w.wait(br.acc_done + 8 * b, (u - 1) & 1);
-        if (ok && MODE != DV && f >= 1) ok = w.wait(br.dp_free, (f - 1) & 1);  // the lane threads hold dP of step f - 1 in registers
         if (!ok) break;
         mv::um::fence_after();
         if (lead) {
-          if (MODE != DV) {
-            issue_nt(c.tmem + TM_DP, f1_desc, short_desc);  // dP = dO V^T  /  dP^T = V dO^T
-            mv::um::commit(br.sempty + 8 * ss);
-          }
           issue_nt(s_tmem, f0_desc, MODE == DV ? short_desc : long_desc);  // S = Q K^T  /  S^T = K Q^T
           if (MODE == DV) mv::um::commit(br.sempty + 8 * ss);
           mv::um::commit(br.s_full + 8 * b);
@@ -431,6 +438,21 @@ __device__ __forceinline__ void bwd_body(const BwdArgs& a, const CUtensorMap* tm
       const int b = e % NBUF;
       float pre = 0.f;
       if (MODE != DQ && a_ok) pre = fetch(a_start, a_n, a_hg);
+      // dP is complete a product before the scores.  In DQ it goes to registers at once and the buffer back to the tensor
+      // cores (measured: 1.91 -> 1.83 ms); in DK, whose lane threads have more to wait for, the extra wait costs more
+      // than it gains (a step 2400 -> 2660 cycles), so dP is read together with the scores.
+      constexpr bool DP_EARLY = MODE == DQ;
+      uint32_t s0[32], s1[32], dp0[32], dp1[32], o[16];
+      if (MODE != DV && DP_EARLY) {
+        ok = w.warp_wait(br.dp_full, e & 1);
+        if (!ok) break;
+        mv::um::fence_after();
+        mv::um::ld32(lane_base + TM_DP + ch * 64, dp0);
+        mv::um::ld32(lane_base + TM_DP + ch * 64 + 32, dp1);
+        mv::um::wait_ld();
+        mv::um::fence_before();
+        mv::mbar_arrive(br.dp_free);
+      }
       if (MODE != DQ) ok = w.warp_wait(br.vec_ready, e & 1);
       if (ok) ok = w.warp_wait(br.s_full + 8 * b, (e / NBUF) & 1);
       if (!ok) break;
@@ -450,15 +472,14 @@ __device__ __forceinline__ void bwd_body(const BwdArgs& a, const CUtensorMap* tm
       // DK is short of registers (the column constants are prefetched beside dP): it reads the second half of its
       // scores after the first half's arithmetic
       constexpr bool S1_LATE = MODE == DK;
-      uint32_t s0[32], s1[32], dp0[32], dp1[32], o[16];
       mv::um::ld32(sbuf, s0);
       if (!S1_LATE) mv::um::ld32(sbuf + 32, s1);
-      if (MODE != DV) {
+      if (MODE != DV && !DP_EARLY) {
         mv::um::ld32(lane_base + TM_DP + ch * 64, dp0);
         mv::um::ld32(lane_base + TM_DP + ch * 64 + 32, dp1);
       }
       mv::um::wait_ld();
-      if (MODE != DV) {
+      if (MODE != DV && !DP_EARLY) {
         mv::um::fence_before();
         mv::mbar_arrive(br.dp_free);  // dP is in registers: the tensor cores may write the next step's
       }
