@@ -468,8 +468,19 @@ def run_ours(args):
     vp_ = C.c_void_p
     qh_p, kh_p, vh_p, oh_p, stg_p, stg_len = (vp_(qh.data_ptr()), vp_(kh.data_ptr()), vp_(vh.data_ptr()), vp_(oh.data_ptr()),
                                               vp_(staging.data_ptr()), staging.numel())
-    decode_step_host = B.lib.mv_decode_step_host_batch
     stream = leg.stream
+    # a step that moves megabytes is cut into two slices of requests whose copies overlap each other's kernels
+    e2e_slices = 2 if qh.numel() * qh.element_size() >= (2 << 20) and wl.batch.n_req >= 2 else 1
+    if e2e_slices > 1:
+        slices = B.PlanSlices(leg.plans[0], st.geom, e2e_slices)
+        staging = torch.empty(slices.staging_bytes(st.geom), dtype=torch.uint8, device=dev)
+        stg_p, stg_len = vp_(staging.data_ptr()), staging.numel()
+        pipelined = B.lib.mv_decode_step_host_pipelined
+
+        def decode_step_host(cb, _plan_ref, g, *rest):
+            return pipelined(cb, slices._hs, e2e_slices, g, *rest)
+    else:
+        decode_step_host = B.lib.mv_decode_step_host_batch
 
     def e2e_step(i):
         kp, vp = leg.pool_ptr[i % leg.n_pools]
@@ -512,7 +523,10 @@ def run_ours(args):
         gc.record(stream)
         barrier()
         gather_ms, _ = multirank.reduce_job(ga.elapsed_time(gc) / 20, 0, dist, dev)
-    same = bool(torch.equal(oh, st.out.cpu()))   # the e2e output equals the device-path output bit for bit
+    # the e2e output against the device path's: bit for bit when unsliced; a slice cuts its key ranges for its own share of
+    # the step, so the split-KV merge may round in another order (bf16 tolerance then)
+    e2e_dev_err = float((oh.float() - st.out.float().cpu()).abs().max())
+    same = bool(torch.equal(oh, st.out.cpu())) if e2e_slices == 1 else bool(e2e_dev_err <= BF16_TOL[0])
     h2d = int(leg.plans[0].device_bytes() + qh.numel() * 2 + kh.numel() * 2 + vh.numel() * 2)
     d2h = int(oh.numel() * 2)
 
@@ -559,8 +573,11 @@ def run_ours(args):
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_rows / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": Ke, "repeats": len(e2e_reps), "ms_per_step": e2e_ms / Ke, "wall_ms_per_step": e2e_med[1] / Ke,
-                "call": "mv_decode_step_host_batch (pinned host q/k/v in, planning inside the call while they travel, host out), stream synchronised every step",
-                "matches_device_path": same},
+                "call": ("mv_decode_step_host_pipelined (two slices of requests, each planned inside the call; pinned host q/k/v in, host out; "
+                         "a slice's copies overlap the other's kernels), stream synchronised every step" if e2e_slices > 1 else
+                         "mv_decode_step_host_batch (pinned host q/k/v in, planning inside the call while they travel, host out), "
+                         "stream synchronised every step"),
+                "matches_device_path": same, "max_abs_vs_device_path": e2e_dev_err, "slices": e2e_slices},
         "gpu_launches": int(3 * K),
         "gpu_launches_all_repeats": int(launches_all),
         "planner_us": planner_us,

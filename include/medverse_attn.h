@@ -353,6 +353,31 @@ mv_status mv_decode_step_host_batch(const mv_dag_batch* batch, mv_plan** plan, c
                                     void* k_pages, void* v_pages, void* staging, size_t staging_bytes,
                                     void* cuda_stream);
 
+/* The same step cut into slices that overlap (Sec. 4.3: the requests of a batch advance independently of one
+ * another, so a batch may be cut between requests).  The batch is split into n_slices runs of consecutive requests with
+ * about equal numbers of new tokens; every slice is planned on its own (plans[i], created when NULL, reused
+ * otherwise) and runs as mv_decode_step_host_batch does, on one of two streams that the library keeps per device
+ * (created by the first call on that device, with two event pairs, and kept until the process exits): slice i + 1's
+ * inputs travel while slice i computes, and slice i's output travels while slice i + 1 computes.  The work starts
+ * behind everything already enqueued on `cuda_stream`, and `cuda_stream` continues behind all of it: synchronise
+ * `cuda_stream` before reading out_host, as with the other forms.  Rows of q, k, v, out are those of the whole batch
+ * (a slice's rows are consecutive).  Results are those of the unsliced call up to the rounding order of the split-KV
+ * merge (a slice's key ranges are cut for its own share of the step).
+ *   plans    host array of n_slices plan pointers (in/out); none may have an upload in flight
+ *   n_slices 1 .. min(8, batch->n_req)
+ *   staging  device, 256-byte aligned; mv_decode_step_pipelined_staging_bytes(plans, n_slices, geom) bytes after
+ *            mv_decode_step_pipelined_plan on a batch of the same shape (0 if a plan is missing or invalid)
+ * mv_decode_step_pipelined_plan plans the slices only (host work; for sizing the staging buffer).
+ * Errors: MV_ERR_INVALID_ARG (n_slices out of range, a slice without a request, null pointers), MV_ERR_WORKSPACE,
+ * MV_ERR_CUDA, and those of mv_plan_dag; after an error, work of earlier slices may already be enqueued. */
+mv_status mv_decode_step_pipelined_plan(const mv_dag_batch* batch, mv_plan** plans, int32_t n_slices,
+                                        const mv_attn_geom* geom);
+size_t mv_decode_step_pipelined_staging_bytes(mv_plan* const* plans, int32_t n_slices, const mv_attn_geom* geom);
+mv_status mv_decode_step_host_pipelined(const mv_dag_batch* batch, mv_plan** plans, int32_t n_slices,
+                                        const mv_attn_geom* geom, const void* q_host, const void* k_host,
+                                        const void* v_host, void* out_host, void* k_pages, void* v_pages,
+                                        void* staging, size_t staging_bytes, void* cuda_stream);
+
 /* Reads the device-side status word of the kernels that last ran with this plan's uploaded tables: MV_OK, or
  * MV_ERR_TIMEOUT if a bounded wait inside a kernel ran out (the kernel then still terminated, with an
  * undefined result).  Copies 4 bytes device->host on `cuda_stream` and synchronises that stream.

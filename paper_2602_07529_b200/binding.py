@@ -27,7 +27,8 @@ WORK_TABLES = {"stages": 10, "units": 11, "item_rows": 12, "cta_unit_off": 13, "
 
 EXPORTS = ["mv_plan_dag", "mv_plan_bind_geometry", "mv_plan_table", "mv_plan_get_stats", "mv_plan_device_bytes", "mv_plan_upload",
            "mv_plan_destroy", "mv_workspace_bytes", "mv_rope_write_kv", "mv_dag_decode_attn",
-           "mv_dag_prefill_attn", "mv_dag_prefill_attn_bwd", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_decode_step_host_batch", "mv_status_string",
+           "mv_dag_prefill_attn", "mv_dag_prefill_attn_bwd", "mv_decode_step_staging_bytes", "mv_decode_step_host", "mv_decode_step_host_batch", "mv_decode_step_pipelined_plan", "mv_decode_step_pipelined_staging_bytes",
+           "mv_decode_step_host_pipelined", "mv_status_string",
            "mv_launch_count", "mv_plan_read_status", "mv_dag_decode_attn_static",
            "mv_static_workspace_bytes", "mv_rope_write_kv_fp8", "mv_dag_decode_attn_fp8", "mv_selftest_bounded_wait", "mv_selftest_tmap_cache",
            "mv_sched_create", "mv_sched_destroy", "mv_sched_add_request", "mv_sched_step", "mv_sched_rows",
@@ -99,6 +100,10 @@ def _load():
     lib.mv_decode_step_staging_bytes.restype = sz
     lib.mv_decode_step_host.argtypes = [vp, C.POINTER(_Geom)] + [vp] * 7 + [sz, vp]
     lib.mv_decode_step_host_batch.argtypes = [C.POINTER(_DagBatch), C.POINTER(vp), C.POINTER(_Geom)] + [vp] * 7 + [sz, vp]
+    lib.mv_decode_step_pipelined_plan.argtypes = [C.POINTER(_DagBatch), C.POINTER(vp), i32, C.POINTER(_Geom)]
+    lib.mv_decode_step_pipelined_staging_bytes.argtypes = [C.POINTER(vp), i32, C.POINTER(_Geom)]
+    lib.mv_decode_step_pipelined_staging_bytes.restype = sz
+    lib.mv_decode_step_host_pipelined.argtypes = [C.POINTER(_DagBatch), C.POINTER(vp), i32, C.POINTER(_Geom)] + [vp] * 7 + [sz, vp]
     lib.mv_status_string.argtypes = [C.c_int]
     lib.mv_status_string.restype = C.c_char_p
     lib.mv_plan_read_status.argtypes = [vp, vp, C.POINTER(i32)]
@@ -320,6 +325,45 @@ def mv_decode_step_host_batch(plan: Plan, geom: _Geom, q_host, k_host, v_host, o
     _check(lib.mv_decode_step_host_batch(C.byref(plan.c_batch), C.byref(plan._h), C.byref(geom), _ptr(q_host), _ptr(k_host),
                                          _ptr(v_host), _ptr(out_host), _ptr(k_pages), _ptr(v_pages), _ptr(staging),
                                          staging.numel() * staging.element_size(), _stream_ptr(stream)), "mv_decode_step_host_batch")
+
+
+class PlanSlices:
+    """Owner of the plans of a sliced step: ``PlanSlices(plan, geom, n)`` cuts ``plan``'s batch into ``n`` runs of requests
+    and plans each (host work)."""
+
+    def __init__(self, plan: Plan, geom: _Geom, n_slices: int):
+        self.n = int(n_slices)
+        self.batch_owner = plan  # keeps the batch arrays alive
+        self._hs = (C.c_void_p * self.n)()
+        _check(lib.mv_decode_step_pipelined_plan(C.byref(plan.c_batch), self._hs, self.n, C.byref(geom)), "mv_decode_step_pipelined_plan")
+
+    def staging_bytes(self, geom: _Geom) -> int:
+        return int(lib.mv_decode_step_pipelined_staging_bytes(self._hs, self.n, C.byref(geom)))
+
+    def table(self, i: int, name: str) -> np.ndarray:
+        """A canonical table of slice ``i``'s plan (a copy)."""
+        view = Plan.__new__(Plan)
+        view._h, view._keep = C.c_void_p(self._hs[i]), None
+        try:
+            return view.table(name)
+        finally:
+            view._h = C.c_void_p(None)   # borrowed: the slices own the plan
+
+    def __del__(self):
+        try:
+            for i in range(getattr(self, "n", 0)):
+                if self._hs[i]:
+                    lib.mv_plan_destroy(C.c_void_p(self._hs[i]))
+                    self._hs[i] = None
+        except Exception:   # interpreter shutdown: the module's globals may be gone
+            pass
+
+
+def mv_decode_step_host_pipelined(slices: PlanSlices, geom: _Geom, q_host, k_host, v_host, out_host, k_pages, v_pages, staging, stream=None):
+    """The host-to-host step in overlapping slices (each slice planned again inside the call)."""
+    _check(lib.mv_decode_step_host_pipelined(C.byref(slices.batch_owner.c_batch), slices._hs, slices.n, C.byref(geom), _ptr(q_host),
+                                             _ptr(k_host), _ptr(v_host), _ptr(out_host), _ptr(k_pages), _ptr(v_pages), _ptr(staging),
+                                             staging.numel() * staging.element_size(), _stream_ptr(stream)), "mv_decode_step_host_pipelined")
 
 
 def mv_selftest_bounded_wait(plan: Plan, limit_ns: int, stream=None):

@@ -409,6 +409,37 @@ def test_decode_step_host_matches_device_calls():
     st.plan.upload(st.pod.tables)
 
 
+def test_decode_step_host_pipelined_matches_unsliced():
+    """The sliced host-to-host step (slices planned on their own, two internal streams) against the device calls on the
+    whole batch: a slice cuts its key ranges for its own share of the step, so the split-KV merge may round in another
+    order; everything else is the same arithmetic."""
+    B, rt = _B(), _rt()
+    wl = synth.config2(n_req=7, prefix=300, branches=3, branch_len=40)
+    st = rt.DecodeState(wl)
+    want = st.step().float().cpu()
+    qh, kh, vh = (t.cpu().pin_memory() for t in (st.q, st.k, st.v))
+    kp, vp = st.pools[0]
+    for n_slices in (1, 2, 3, 7):
+        slices = B.PlanSlices(st.plan, st.geom, n_slices)
+        nbytes = slices.staging_bytes(st.geom)
+        assert nbytes > 0
+        staging = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        oh = torch.empty_like(qh).pin_memory()
+        for _ in range(2):   # twice in a row: the plans and the internal streams are reused
+            oh.fill_(float("nan"))
+            B.mv_decode_step_host_pipelined(slices, st.geom, qh, kh, vh, oh, kp, vp, staging)
+            torch.cuda.synchronize()
+            got = oh.float()
+            assert torch.isfinite(got).all()
+            assert (got - want).abs().max().item() <= 2e-2
+            assert ((got - want).norm() / want.norm()).item() <= 1e-2
+        with pytest.raises(B.MvError):   # too small for the slices
+            B.mv_decode_step_host_pipelined(slices, st.geom, qh, kh, vh, oh, kp, vp, staging[:nbytes // 2 // 256 * 256])
+        torch.cuda.synchronize()
+    with pytest.raises(B.MvError):       # more slices than requests
+        B.PlanSlices(st.plan, st.geom, 8)
+
+
 def test_error_statuses_on_kernel_calls():
     B, rt = _B(), _rt()
     wl = synth.config2(n_req=1, prefix=100, branches=2, branch_len=20)

@@ -179,3 +179,27 @@ def test_plan_without_geometry_then_bind_any_geometry():
     assert e.value.status == 4
     with pytest.raises(B.MvError):                            # 6 query heads over 4 KV heads
         B.Plan(wl.batch, geom=B.make_geom(6, 4, 128, wl.batch.num_pages, "bf16"))
+
+
+def test_sliced_step_plans_cover_the_batch():
+    """mv_decode_step_pipelined_plan cuts a batch between requests: the slices' position and slot tables, one after the
+    other, are the whole batch's (requests are planned independently of one another, Sec. 4.3), every slice keeps a
+    request, and no slice holds more than its even share of the new tokens plus one request's."""
+    for wl in (synth.config2(n_req=7, prefix=200, branches=3, branch_len=30), synth.config3(n_req=9, prefix=300)):
+        g = B.geom_of(wl)
+        plan = B.Plan(wl.batch, geom=g)
+        b = wl.batch
+        per_req = [int(b.node_new[b.node_off[r]:b.node_off[r + 1]].sum()) for r in range(b.n_req)]
+        for n in (1, 2, 3, min(b.n_req, 8)):
+            sl = B.PlanSlices(plan, g, n)
+            for name in ("pos_id", "slot"):
+                parts = [sl.table(i, name) for i in range(n)]
+                assert np.array_equal(np.concatenate(parts), plan.table(name))
+            rows = [len(sl.table(i, "pos_id")) for i in range(n)]
+            assert sum(rows) == sum(per_req) and min(rows) > 0
+            if n < b.n_req:
+                assert max(rows) <= sum(per_req) / n + max(per_req)
+        with pytest.raises(B.MvError):
+            B.PlanSlices(plan, g, b.n_req + 1)
+        with pytest.raises(B.MvError):
+            B.PlanSlices(plan, g, 0)
