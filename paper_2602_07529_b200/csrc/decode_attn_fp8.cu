@@ -259,11 +259,11 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
         }
       }
     }
+    // ordinary stores above, read by the tensor core (async proxy): every lane that wrote fences its own stores, then one
+    // lane signals (with the fence in the signalling lane alone, one run in some tens read a stale remainder tile)
+    mv::fence_proxy_async();
     __syncwarp();
-    if (lane == 0) {
-      mv::fence_proxy_async();  // ordinary stores above, read by the tensor core (async proxy)
-      mv::mbar_arrive(bar(&meta->q_full));
-    }
+    if (lane == 0) mv::mbar_arrive(bar(&meta->q_full));
     for (; s_next < wu.n_stages && ok; ++s_next) ok = issue_stage(s_next);
     wu = wu1; wu1 = wu2; ir0 = nir0; ir1 = nir1; win = nwin;
   }
