@@ -527,7 +527,7 @@ def run_ours(args):
     # the step, so the split-KV merge may round in another order (bf16 tolerance then)
     e2e_dev_err = float((oh.float() - st.out.float().cpu()).abs().max())
     same = bool(torch.equal(oh, st.out.cpu())) if e2e_slices == 1 else bool(e2e_dev_err <= BF16_TOL[0])
-    h2d = int(leg.plans[0].device_bytes() + qh.numel() * 2 + kh.numel() * 2 + vh.numel() * 2)
+    h2d = int((slices.device_bytes() if e2e_slices > 1 else leg.plans[0].device_bytes()) + qh.numel() * 2 + kh.numel() * 2 + vh.numel() * 2)
     d2h = int(oh.numel() * 2)
 
     # ---- host planner alone

@@ -340,6 +340,10 @@ class PlanSlices:
     def staging_bytes(self, geom: _Geom) -> int:
         return int(lib.mv_decode_step_pipelined_staging_bytes(self._hs, self.n, C.byref(geom)))
 
+    def device_bytes(self) -> int:
+        """Bytes of plan tables that a step uploads (all slices)."""
+        return sum(int(lib.mv_plan_device_bytes(C.c_void_p(self._hs[i]))) for i in range(self.n))
+
     def table(self, i: int, name: str) -> np.ndarray:
         """A canonical table of slice ``i``'s plan (a copy)."""
         view = Plan.__new__(Plan)
