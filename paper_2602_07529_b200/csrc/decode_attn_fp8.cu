@@ -224,7 +224,9 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
         const int r_lo = __shfl_sync(0xffffffffu, ir0.row, r & 31), r_hi = __shfl_sync(0xffffffffu, ir1.row, r & 31);
         const int row = r < 32 ? r_lo : r_hi;
         raw[i] = make_uint4(0, 0, 0, 0);
-        if (x < n_qv) raw[i] = __ldg(reinterpret_cast<const uint4*>(a.q + (int64_t(row) * a.Hq + wu.kvh * a.G + x % a.G) * D + c * 8));
+        // through L2, not the read-only path: the RoPE kernel writes q while this grid is already resident (programmatic
+        // stream serialisation), so q is not read-only for this kernel's lifetime
+        if (x < n_qv) raw[i] = __ldcg(reinterpret_cast<const uint4*>(a.q + (int64_t(row) * a.Hq + wu.kvh * a.G + x % a.G) * D + c * 8));
       }
 #pragma unroll
       for (int i = 0; i < QB; ++i) {
