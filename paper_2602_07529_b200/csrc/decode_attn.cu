@@ -584,14 +584,16 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const float* __restri
     for (int k = 0; k < 4; ++k) {
       const bool ok = pb + k < p1;
       const int64_t ps = int64_t(ok ? pb + k : pb) * G + g;
-      ml[k] = *reinterpret_cast<const float2*>(part_ml + ps * 2);
+      // through L2 (ld.global.cg), never the read-only path: the attention kernel writes the partials while this grid may
+      // already be resident, so they are not read-only for this kernel's lifetime
+      ml[k] = __ldcg(reinterpret_cast<const float2*>(part_ml + ps * 2));
       if (!ok) ml[k].x = -INFINITY;
       const float* po = part_o + ps * D + lane * E;
       if (E == 4) {
-        const float4 v = *reinterpret_cast<const float4*>(po);
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(po));
         t[k][0] = v.x; t[k][1] = v.y; t[k][2 % E] = v.z; t[k][3 % E] = v.w;
       } else {
-        const float2 v = *reinterpret_cast<const float2*>(po);
+        const float2 v = __ldcg(reinterpret_cast<const float2*>(po));
         t[k][0] = v.x; t[k][1] = v.y;
       }
     }
