@@ -92,8 +92,9 @@ __device__ __forceinline__ void rope_cos_sin(int pos, double theta, float& c, fl
 // FP8: the pools hold 8-bit floats (4 exponent, 3 mantissa bits), [pages][KV heads][16 tokens][head_dim bytes]; a value is
 // stored as round(x / scale[head]), saturating (kv_scale = the K scales of all heads, then the V scales).
 template <typename T, int D, int TPC, bool FP8 = false>
-__global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
-                                                            T* __restrict__ q_rot, T* __restrict__ k_rot, T* __restrict__ k_pages,
+// q_rot may be q and k_rot may be k (rotation in place), so those four carry no __restrict__.
+__global__ void __launch_bounds__(256) rope_write_kv_kernel(const T* q, const T* k, const T* __restrict__ v, T* q_rot, T* k_rot,
+                                                            T* __restrict__ k_pages,
                                                             T* __restrict__ v_pages, const int32_t* __restrict__ pos_id,
                                                             const int64_t* __restrict__ slot, int n_tok, int Hq, int Hkv,
                                                             const __grid_constant__ ThetaTable tt, const float* __restrict__ kv_scale = nullptr,
