@@ -367,6 +367,8 @@ mv_status mv_decode_step_host_batch(const mv_dag_batch* batch, mv_plan** plan, c
  *   n_slices 1 .. min(8, batch->n_req)
  *   staging  device, 256-byte aligned; mv_decode_step_pipelined_staging_bytes(plans, n_slices, geom) bytes after
  *            mv_decode_step_pipelined_plan on a batch of the same shape (0 if a plan is missing or invalid)
+ * The library's two streams and their events are shared by every call on a device: host threads must not run this
+ * call on the same device at the same time.
  * mv_decode_step_pipelined_plan plans the slices only (host work; for sizing the staging buffer).
  * Errors: MV_ERR_INVALID_ARG (n_slices out of range, a slice without a request, null pointers), MV_ERR_WORKSPACE,
  * MV_ERR_CUDA, and those of mv_plan_dag; after an error, work of earlier slices may already be enqueued. */
