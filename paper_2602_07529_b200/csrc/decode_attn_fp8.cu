@@ -262,7 +262,7 @@ __device__ __forceinline__ void producer(const TcArgs& a, const Half& h, const C
       }
     }
     // ordinary stores above, read by the tensor core (async proxy): every lane that wrote fences its own stores, then one
-    // lane signals (with the fence in the signalling lane alone, one run in some tens read a stale remainder tile)
+    // lane signals
     mv::fence_proxy_async();
     __syncwarp();
     if (lane == 0) mv::mbar_arrive(bar(&meta->q_full));
@@ -503,6 +503,14 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
             *reinterpret_cast<uint4*>(vt + (j * 16 + nt + (i >> 3)) * 128 + ((i & 7) << 4)) = make_uint4(0, 0, 0, 0);
         }
         mv::fence_proxy_async();  // ordinary stores, read next by the tensor core
+      }
+      // Keep in step with the products: the one before this stage's (issued while this stage's weights were computed) is
+      // confirmed here, before the arrival that lets the next one start.  The waits on o_done tell phases apart by
+      // parity, so a thread may never fall two phases behind; a warp that skipped the wait above would otherwise take
+      // the final wait of a unit for satisfied while two products were still in flight, and read O too early.
+      if (g > 0) {
+        ok = warp_wait(h, bar(&meta->o_done), (g - 1) & 1);
+        if (!ok) break;
       }
       mv::um::fence_before();
       mv::mbar_arrive(bar(&meta->p_full[pb]));
