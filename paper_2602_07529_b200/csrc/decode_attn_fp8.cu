@@ -504,11 +504,13 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, const Half& h) {
         }
         mv::fence_proxy_async();  // ordinary stores, read next by the tensor core
       }
-      // Keep in step with the products: the one before this stage's (issued while this stage's weights were computed) is
-      // confirmed here, before the arrival that lets the next one start.  The waits on o_done tell phases apart by
-      // parity, so a thread may never fall two phases behind; a warp that skipped the wait above would otherwise take
-      // the final wait of a unit for satisfied while two products were still in flight, and read O too early.
-      if (g > 0) {
+      // The waits on o_done tell phases apart by parity, so a thread may never be two phases behind when it waits.  At
+      // the wait above that holds: the scores of this stage were committed after the product two stages back.  At the
+      // unit's final wait it would not: a warp that skipped the wait above could get there while the product of the
+      // stage before the last was still in flight, take the wait for satisfied, and read O too early.  So on the last
+      // stage of a unit that product (issued while this stage's weights were computed) is confirmed here, before the
+      // arrival that lets the last one start.
+      if (s > 0 && s + 1 == n) {
         ok = warp_wait(h, bar(&meta->o_done), (g - 1) & 1);
         if (!ok) break;
       }
